@@ -1,0 +1,183 @@
+/*
+ * accept.h -- C ABI of the boundary-tensor codec (AccEPT bit-level compression, Sec. 3.3-3.4).
+ *
+ * The codec turns a flat fp32 tensor x_v (Sec. 3.3, "Forward Quantizer": the boundary tensor is
+ * vectorised to N = n*w*h*c values) into k-bit integer codes packed densely into 32-bit words plus
+ * fp32 side words, and back.  All compute runs in CUDA kernels built for sm_100a; there is no host
+ * fallback.  Every entry point is asynchronous on the stream it is given and allocates nothing.
+ *
+ * ---------------------------------------------------------------------------------------------
+ * Operation (per chunk of chunk_elems consecutive values; the paper's scheme is the case
+ * chunk_elems >= n_elems, one range for the whole tensor):
+ *
+ *   range   ABSMAX (Sec. 3.3 "Backward Quantizer"):  c = max|x|,  L = 2^(k-1)-1,  s = c/L,  o = 0
+ *           MINMAX (affine extension):               lo = min x, hi = max x, L = 2^k-1,
+ *                                                    s = (hi-lo)/L,  o = lo
+ *   scale   inv = L/c  (resp. L/(hi-lo)); one IEEE fp32 division per chunk.  If the range is 0,
+ *           or inv overflows, the chunk is degenerate: s = 0, inv = 0, every code is the zero point.
+ *   codes   t = x*inv           (MINMAX: t = (x-lo)*inv), each fp32 operation rounded separately
+ *           NEAREST:    q = rint(t)                      (ties to even)
+ *           STOCHASTIC: q = floor(t) + [U < t-floor(t)]  (Eq. 7), U from the counter-based
+ *                       generator described at accept_params.seed
+ *           ABSMAX: q clamped to [-2^(k-1), 2^(k-1)-1], stored code u = q + 2^(k-1)  ("+8" of the
+ *           "Backward Encoder" for k = 4);  MINMAX: u = q clamped to [0, 2^k-1]
+ *   pack    INTERLEAVED ("Backward Encoder"): code of element t of the chunk occupies bits
+ *           [k*t, k*t+k) of the chunk's little-endian bit string (k = 8: plain bytes).
+ *           BITPLANE ("Forward Encoder"): per group of 32 consecutive elements, k consecutive
+ *           32-bit words; bit t of word j is bit j of the code of element t of the group.
+ *   decode  ("Backward Decoder/Dequantizer", "Forward Decoder"): unpack u;
+ *           ABSMAX: xhat = float(u - 2^(k-1)) * s;   MINMAX: xhat = fl(fl(float(u)*s) + o)
+ *
+ * Stream layout (little-endian, byte offsets):
+ *   [0,32)    header, eight u32: magic 0x54504341 ("ACPT"), version 1, n_elems low, n_elems high,
+ *             chunk_elems, k, range | round<<8 | layout<<16, 0
+ *   [32, 32+8M)   M = ceil(n_elems/chunk_elems) records {float s; float o}, one per chunk
+ *   [P, ...)  payload, P = 32+8M rounded up to a multiple of 16.  Chunk m starts at word
+ *             m*chunk_elems*k/32 of the payload.  A partial last chunk holds ceil(valid/32)*k
+ *             words; codes of padding elements are 0 bits.
+ *   total     P + 4*k*ceil(n_elems/32) bytes  (= accept_compressed_size).
+ *
+ * Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  d_x, d_xhat and d_stream must be
+ * 16-byte aligned.  The caller owns every buffer and the stream.
+ */
+#ifndef ACCEPT_H_
+#define ACCEPT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ACCEPT_MAGIC 0x54504341u
+#define ACCEPT_VERSION 1u
+#define ACCEPT_HEADER_BYTES 32u
+
+/* Return codes of the host entry points (nothing was launched unless ACCEPT_OK). */
+typedef enum {
+  ACCEPT_OK = 0,
+  ACCEPT_ERR_NULL = 1,          /* a required pointer is NULL */
+  ACCEPT_ERR_BAD_K = 2,         /* k not in {2,3,4,8}, or k = 3 with INTERLEAVED */
+  ACCEPT_ERR_BAD_CHUNK = 3,     /* chunk_elems < 32 or not a multiple of 32 */
+  ACCEPT_ERR_BAD_ENUM = 4,      /* range / round / layout out of range */
+  ACCEPT_ERR_TOO_SMALL = 5,     /* a buffer is smaller than the size queries say */
+  ACCEPT_ERR_BAD_STREAM_HEADER = 6, /* header words do not match the parameters */
+  ACCEPT_ERR_CUDA = 7,          /* a CUDA runtime call failed */
+  ACCEPT_ERR_NONFINITE = 8,     /* reported through the device status word only */
+  ACCEPT_ERR_BAD_SIZE = 9,      /* n_elems = 0 */
+  ACCEPT_ERR_MISALIGNED = 10    /* a device pointer is not 16-byte aligned */
+} accept_status;
+
+/* Bits of the device status word (word 0 of the workspace); sticky until the caller clears it. */
+#define ACCEPT_DEV_NONFINITE 1u   /* some chunk held NaN/Inf (or an overflowing MINMAX range) */
+#define ACCEPT_DEV_BAD_HEADER 2u  /* accept_decompress: stream header differs from the parameters */
+
+typedef enum { ACCEPT_RANGE_ABSMAX = 0, ACCEPT_RANGE_MINMAX = 1 } accept_range;
+typedef enum { ACCEPT_ROUND_NEAREST = 0, ACCEPT_ROUND_STOCHASTIC = 1 } accept_round;
+typedef enum { ACCEPT_LAYOUT_INTERLEAVED = 0, ACCEPT_LAYOUT_BITPLANE = 1 } accept_layout;
+
+/*
+ * Parameters of one call.
+ *   n_elems      N >= 1, number of fp32 values.
+ *   chunk_elems  C, multiple of 32, >= 32: elements sharing one range.
+ *   k            bit width: 2, 3 (BITPLANE only), 4 or 8.
+ *   seed, rng_offset  STOCHASTIC only.  Element i draws
+ *                  U_i = (h >> 9) * 2^-23,
+ *                  h   = fmix32( lo32(ctr) ^ fmix32( hi32(ctr) ^ lo32(seed) ) ^ hi32(seed) ),
+ *                  ctr = rng_offset + i (mod 2^64),
+ *                fmix32 = the 32-bit finaliser of MurmurHash3:
+ *                  h ^= h>>16; h *= 0x85EBCA6B; h ^= h>>13; h *= 0xC2B2AE35; h ^= h>>16.
+ *                The same (seed, rng_offset) reproduces the same stream; advance rng_offset by
+ *                n_elems between calls to draw fresh numbers.
+ */
+typedef struct {
+  uint64_t n_elems;
+  uint32_t chunk_elems;
+  uint32_t k;
+  int32_t range;   /* accept_range  */
+  int32_t round;   /* accept_round  */
+  int32_t layout;  /* accept_layout */
+  uint32_t reserved; /* must be 0 */
+  uint64_t seed;
+  uint64_t rng_offset;
+} accept_params;
+
+/* Validates p as the compress/decompress entry points do (host only). */
+accept_status accept_check_params(const accept_params* p);
+
+/*
+ * Size in bytes of the compressed stream for p (layout above); 0 if p is invalid.
+ * Sec. 3.3 "Transmission Data Comparison", Eq. 8: payload of k bits per element plus fp32 side words.
+ */
+size_t accept_compressed_size(const accept_params* p);
+
+/* Byte offset of the payload inside the stream (P above); 0 if p is invalid. */
+size_t accept_payload_offset(const accept_params* p);
+
+/*
+ * Bytes of device workspace the kernels need: 16.  Word 0 is the device status word; the caller
+ * zeroes the workspace once (and whenever it wants to clear the status).  0 if p is invalid.
+ */
+size_t accept_workspace_size(const accept_params* p);
+
+/*
+ * Quantizer + encoder (Sec. 3.3): reads n_elems floats at d_x, writes accept_compressed_size(p)
+ * bytes at d_stream (header, per-chunk {s,o}, payload), in one kernel launch on cuda_stream
+ * (a cudaStream_t, may be NULL for the default stream).  Non-finite input does not fail the call:
+ * the chunk is written as degenerate and ACCEPT_DEV_NONFINITE is or-ed into the status word.
+ * d_x is only read; d_stream is fully overwritten up to the compressed size.
+ */
+accept_status accept_compress(const accept_params* p, const float* d_x, void* d_stream,
+                              size_t stream_bytes, void* d_ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Decoder + dequantizer (Sec. 3.4): reads the stream at d_stream, writes n_elems floats at d_xhat,
+ * in one kernel launch.  p carries what the receiver agreed on with the sender (n_elems,
+ * chunk_elems, k, range, layout; round/seed are ignored); the kernel compares it with the header
+ * words and or-s ACCEPT_DEV_BAD_HEADER into the status word on a mismatch (the output is then
+ * unspecified but every access stays inside the buffers as sized by p).
+ */
+accept_status accept_decompress(const accept_params* p, const void* d_stream, size_t stream_bytes,
+                                float* d_xhat, void* d_ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Host-buffer variants, for callers whose tensors live in host memory: copy h_x to the staging
+ * buffer d_x (host to device), run accept_compress, copy the stream back to h_stream (and the
+ * mirror image for decompress), all asynchronously on cuda_stream.  Staging buffers are the
+ * caller's; sizes as for the device entry points.  Pinned host memory makes the copies overlap
+ * nothing else but avoids a bounce buffer in the driver.
+ */
+accept_status accept_compress_host(const accept_params* p, const float* h_x, void* h_stream,
+                                   size_t stream_bytes, float* d_x, void* d_stream, void* d_ws,
+                                   size_t ws_bytes, void* cuda_stream);
+accept_status accept_decompress_host(const accept_params* p, const void* h_stream,
+                                     size_t stream_bytes, float* h_xhat, void* d_stream,
+                                     float* d_xhat, void* d_ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Synchronises cuda_stream, copies the status word to the host and returns it in *status_bits
+ * (ACCEPT_DEV_* bits).  Returns ACCEPT_ERR_CUDA if the stream reports an error.
+ */
+accept_status accept_last_device_status(const void* d_ws, void* cuda_stream, uint32_t* status_bits);
+
+/*
+ * Parses the 32 header bytes (a HOST copy) into *out; ACCEPT_ERR_BAD_STREAM_HEADER if the magic,
+ * version or any field is invalid.  For receivers that know nothing but the bytes they got (Sec. 3.4).
+ */
+accept_status accept_parse_header(const void* h_header, accept_params* out);
+
+/*
+ * Bit width the paper's schedule prescribes after n_lr_changes learning-rate changes:
+ * forward (Sec. 3.3 "Forward Quantizer"): starts at 2, +1 per change, at most 4;
+ * backward ("Backward Quantizer"): 8 until the first change, then 4.
+ */
+int accept_bitwidth_schedule(int is_backward, int n_lr_changes);
+
+/* Number of kernels the library has launched in this process (all entry points). */
+uint64_t accept_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ACCEPT_H_ */

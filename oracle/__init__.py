@@ -1,0 +1,170 @@
+"""TEST INFRASTRUCTURE: ctypes access to the CPU oracle (``accept_oracle.c``).
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg import this package.  It
+shares nothing with the CUDA library: its own C file, its own shared object, its own argument
+lists.  ``build()`` compiles the C file with gcc (no fast-math, no FMA contraction).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "accept_oracle.c")
+_LIB = os.path.join(_HERE, "libaccept_oracle.so")
+
+RANGE_ABSMAX, RANGE_MINMAX = 0, 1
+ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
+LAYOUT_INTERLEAVED, LAYOUT_BITPLANE = 0, 1
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle if its shared object is missing or older than the source."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared",
+           "-o", _LIB, _SRC, "-lm"]
+    subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    lib = ctypes.CDLL(build())
+    u64, u32, i32 = ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int
+    vp = ctypes.c_void_p
+    lib.oracle_payload_offset.restype = u64
+    lib.oracle_payload_offset.argtypes = [u64, u32]
+    lib.oracle_payload_bytes.restype = u64
+    lib.oracle_payload_bytes.argtypes = [u64, u32]
+    lib.oracle_stream_bytes.restype = u64
+    lib.oracle_stream_bytes.argtypes = [u64, u32, u32]
+    lib.oracle_rng_hash.restype = u32
+    lib.oracle_rng_hash.argtypes = [u64, u64]
+    lib.oracle_rng_uniform.restype = ctypes.c_float
+    lib.oracle_rng_uniform.argtypes = [u64, u64]
+    lib.oracle_quantize.restype = i32
+    lib.oracle_quantize.argtypes = [vp, u64, u32, u32, i32, i32, u64, u64, vp, vp]
+    lib.oracle_pack.restype = None
+    lib.oracle_pack.argtypes = [vp, u64, u32, u32, i32, vp]
+    lib.oracle_unpack.restype = None
+    lib.oracle_unpack.argtypes = [vp, u64, u32, u32, i32, vp]
+    lib.oracle_dequantize.restype = None
+    lib.oracle_dequantize.argtypes = [vp, vp, u64, u32, u32, i32, vp]
+    lib.oracle_compress.restype = i32
+    lib.oracle_compress.argtypes = [vp, u64, u32, u32, i32, i32, i32, u64, u64, vp]
+    lib.oracle_decompress.restype = i32
+    lib.oracle_decompress.argtypes = [vp, u64, u64, vp]
+    lib.oracle_bitwidth_schedule.restype = i32
+    lib.oracle_bitwidth_schedule.argtypes = [i32, i32]
+    _lib = lib
+    return lib
+
+
+def _f32(x) -> np.ndarray:
+    a = np.ascontiguousarray(x, dtype=np.float32).reshape(-1)
+    return a
+
+
+def _ptr(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def n_chunks(n: int, chunk: int) -> int:
+    return (n + chunk - 1) // chunk
+
+
+def payload_offset(n: int, chunk: int) -> int:
+    return int(_load().oracle_payload_offset(n, chunk))
+
+
+def payload_bytes(n: int, k: int) -> int:
+    return int(_load().oracle_payload_bytes(n, k))
+
+
+def stream_bytes(n: int, chunk: int, k: int) -> int:
+    return int(_load().oracle_stream_bytes(n, chunk, k))
+
+
+def rng_hash(seed: int, ctr: int) -> int:
+    return int(_load().oracle_rng_hash(seed & (2**64 - 1), ctr & (2**64 - 1)))
+
+
+def rng_uniform(seed: int, ctr: int) -> float:
+    return float(_load().oracle_rng_uniform(seed & (2**64 - 1), ctr & (2**64 - 1)))
+
+
+def quantize(x, chunk: int, k: int, range_: int = RANGE_ABSMAX, round_: int = ROUND_NEAREST,
+             seed: int = 0, rng_offset: int = 0):
+    """-> (codes uint8[n], meta float32[M,2], nonfinite flag)."""
+    x = _f32(x)
+    n = x.size
+    codes = np.empty(n, dtype=np.uint8)
+    meta = np.empty((n_chunks(n, chunk), 2), dtype=np.float32)
+    flag = _load().oracle_quantize(_ptr(x), n, chunk, k, range_, round_, seed, rng_offset,
+                                   _ptr(codes), _ptr(meta))
+    return codes, meta, int(flag)
+
+
+def pack(codes, chunk: int, k: int, layout: int) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8).reshape(-1)
+    out = np.empty(payload_bytes(codes.size, k) // 4, dtype=np.uint32)
+    _load().oracle_pack(_ptr(codes), codes.size, chunk, k, layout, _ptr(out))
+    return out
+
+
+def unpack(payload, n: int, chunk: int, k: int, layout: int) -> np.ndarray:
+    payload = np.ascontiguousarray(payload, dtype=np.uint32).reshape(-1)
+    assert payload.size * 4 >= payload_bytes(n, k)
+    codes = np.empty(n, dtype=np.uint8)
+    _load().oracle_unpack(_ptr(payload), n, chunk, k, layout, _ptr(codes))
+    return codes
+
+
+def dequantize(codes, meta, chunk: int, k: int, range_: int) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8).reshape(-1)
+    meta = np.ascontiguousarray(meta, dtype=np.float32)
+    xhat = np.empty(codes.size, dtype=np.float32)
+    _load().oracle_dequantize(_ptr(codes), _ptr(meta), codes.size, chunk, k, range_, _ptr(xhat))
+    return xhat
+
+
+def compress(x, chunk: int, k: int, range_: int = RANGE_ABSMAX, round_: int = ROUND_NEAREST,
+             layout: int = LAYOUT_INTERLEAVED, seed: int = 0, rng_offset: int = 0):
+    """-> (stream uint8[stream_bytes], nonfinite flag)."""
+    x = _f32(x)
+    out = np.empty(stream_bytes(x.size, chunk, k), dtype=np.uint8)
+    flag = _load().oracle_compress(_ptr(x), x.size, chunk, k, range_, round_, layout, seed,
+                                   rng_offset, _ptr(out))
+    return out, int(flag)
+
+
+def decompress(stream, n: int) -> np.ndarray:
+    stream = np.ascontiguousarray(stream, dtype=np.uint8).reshape(-1)
+    xhat = np.empty(n, dtype=np.float32)
+    rc = _load().oracle_decompress(_ptr(stream), stream.size, n, _ptr(xhat))
+    if rc != 0:
+        raise ValueError("oracle_decompress: invalid stream header")
+    return xhat
+
+
+def split_stream(stream, n: int, chunk: int):
+    """Views of a stream: (header uint32[8], meta float32[M,2], payload uint32[...])."""
+    stream = np.ascontiguousarray(stream, dtype=np.uint8).reshape(-1)
+    m = n_chunks(n, chunk)
+    header = stream[:32].view(np.uint32)
+    meta = stream[32:32 + 8 * m].view(np.float32).reshape(m, 2)
+    payload = stream[payload_offset(n, chunk):].view(np.uint32)
+    return header, meta, payload
+
+
+def bitwidth_schedule(is_backward: bool, n_lr_changes: int) -> int:
+    return int(_load().oracle_bitwidth_schedule(int(is_backward), n_lr_changes))
