@@ -1,0 +1,399 @@
+#!/usr/bin/env python
+"""Throughput of the boundary-tensor codec on one or more B200s (one process per GPU).
+
+A step is one pass of the whole hot path over one boundary tensor: accept_compress (range,
+quantize, pack) followed by accept_decompress (unpack, dequantize) of the stream just written.
+The metric is GB/s of fp32 input through that round trip; compress and decompress are also
+reported on their own, each with its achieved fraction of the measured HBM copy bandwidth.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--sweep]
+    python bench.py --impl reference ...      # the CPU oracle on the host cores
+
+With N > 1 (launched under torch.distributed.run) every rank codes its own replica of the tensor;
+the codec has no exchange step, so there is no data-path collective (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+import workloads
+
+METRIC = "compress+decompress round-trip throughput of fp32 boundary tensor"
+UNIT = "GB/s of fp32 input"
+DEFAULT_WORKLOAD = "cfg4_hidden"
+L2_BYTES = 126 << 20
+FALLBACK_HBM_GBS = 6650.0
+
+
+def mode_name(m) -> str:
+    return "k%d-%s-%s-%s" % (m.k, "absmax" if m.range == 0 else "minmax", "nearest" if m.round == 0 else "stochastic",
+                             "interleaved" if m.layout == 0 else "bitplane")
+
+
+def algorithmic_bytes(n: int, chunk: int, k: int) -> float:
+    """Bytes the method must move per call, either direction: 4 + k/8 + 8/C per element."""
+    return n * (4.0 + k / 8.0 + 8.0 / chunk)
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.out = None
+
+    def start(self):
+        try:
+            self.out = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.flush()
+        self.out.seek(0)
+        sm, smax, reasons = [], [], set()
+        for line in self.out.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.out.close()
+        os.unlink(self.out.name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------- GPU arm
+
+class Codec:
+    """Device buffers for one (tensor, mode): enough rotating copies that a step never finds its
+    inputs in L2."""
+
+    def __init__(self, A, torch, x_host: np.ndarray, chunk: int, mode, seed: int, min_footprint: int = 3 * L2_BYTES):
+        self.A, self.torch = A, torch
+        n = x_host.size
+        self.n, self.chunk, self.mode = n, chunk, mode
+        self.p = A.Params(n, chunk, mode.k, mode.range, mode.round, mode.layout, seed, 0)
+        self.stream_bytes = A.accept_compressed_size(self.p)
+        per_set = 8 * n + self.stream_bytes
+        self.copies = int(max(2, min(4096, -(-min_footprint // per_set))))
+        x0 = torch.from_numpy(x_host).cuda()
+        self.x = [x0] + [x0.clone() for _ in range(self.copies - 1)]
+        self.stream = [torch.empty(self.stream_bytes, dtype=torch.uint8, device="cuda") for _ in range(self.copies)]
+        self.xhat = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(self.copies)]
+        self.ws = A.new_workspace(self.p)
+        self.calls = 0
+
+    def step(self, i: int, events=None):
+        A, j = self.A, i % self.copies
+        if events is not None:
+            events[0].record()
+        A.accept_compress(self.p, self.x[j], self.stream[j], self.ws)
+        if events is not None:
+            events[1].record()
+        A.accept_decompress(self.p, self.stream[j], self.xhat[j], self.ws)
+        if events is not None:
+            events[2].record()
+        self.calls += 2
+
+    def run(self, steps: int, warmup: int):
+        """-> (ms per step, ms per compress, ms per decompress), device-timed."""
+        torch = self.torch
+        for i in range(warmup):
+            self.step(i)
+        torch.cuda.synchronize()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+        for i in range(steps):
+            self.step(warmup + i, ev[i])
+        torch.cuda.synchronize()
+        total = ev[0][0].elapsed_time(ev[-1][2])
+        tc = sum(e[0].elapsed_time(e[1]) for e in ev) / steps
+        td = sum(e[1].elapsed_time(e[2]) for e in ev) / steps
+        return total / steps, tc, td
+
+    def status(self) -> int:
+        return self.A.accept_last_device_status(self.ws)
+
+
+def e2e_run(A, torch, x_host, chunk, mode, seed, steps, warmup):
+    """Round trip through the host-buffer entry points: pinned host tensor in, stream to the host,
+    stream back to the device, reconstructed tensor to the host; copies inside the timed region."""
+    n = x_host.size
+    p = A.Params(n, chunk, mode.k, mode.range, mode.round, mode.layout, seed, 0)
+    sb = A.accept_compressed_size(p)
+    h_x = torch.from_numpy(x_host).pin_memory()
+    h_stream = torch.empty(sb, dtype=torch.uint8).pin_memory()
+    h_xhat = torch.empty(n, dtype=torch.float32).pin_memory()
+    d_x = torch.empty(n, dtype=torch.float32, device="cuda")
+    d_xhat = torch.empty(n, dtype=torch.float32, device="cuda")
+    d_stream, d_ws = A.new_stream_buffer(p), A.new_workspace(p)
+
+    def one():
+        A.accept_compress_host(p, h_x, h_stream, d_x, d_stream, d_ws)
+        A.accept_decompress_host(p, h_stream, h_xhat, d_stream, d_xhat, d_ws)
+
+    for _ in range(warmup):
+        one()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    assert A.accept_last_device_status(d_ws) == 0
+    return ms, 4 * n + sb, sb + 4 * n
+
+
+def time_oracle(x_host, chunk, mode, seed, budget_s=10.0, max_reps=50):
+    """The CPU oracle, as it stands, single-threaded, on x_host: seconds per round trip."""
+    import oracle
+    reps, t0 = 0, time.perf_counter()
+    tc = td = 0.0
+    while True:
+        a = time.perf_counter()
+        stream, _ = oracle.compress(x_host, chunk, mode.k, mode.range, mode.round, mode.layout, seed, 0)
+        b = time.perf_counter()
+        oracle.decompress(stream, x_host.size)
+        c = time.perf_counter()
+        tc += b - a
+        td += c - b
+        reps += 1
+        if time.perf_counter() - t0 >= budget_s or reps >= max_reps:
+            break
+    return tc / reps, td / reps, reps
+
+
+def run_gpu(args):
+    import torch
+    import paper_2311_05827_b200 as A
+    from paper_2311_05827_b200 import build as lib_build
+    lib_build.build()
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the codec has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    spec = workloads.TENSORS[args.workload]
+    mode = spec.headline[0]
+    x_host = workloads.generate(args.workload)
+    n = spec.n
+    peak, peak_src = measured_peak()
+
+    codec = Codec(A, torch, x_host, spec.chunk, mode, spec.seed)
+    launches0 = A.accept_launch_count()
+    sampler = ClockSampler(local_rank)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        codec.step(i)
+    barrier()
+    sampler.start()
+    launches_before = A.accept_launch_count()
+    ms_step, ms_c, ms_d = codec.run(args.steps, 0)
+    launches_timed = A.accept_launch_count() - launches_before
+    barrier()
+    clocks = sampler.stop()
+    assert codec.status() == 0
+
+    t = torch.tensor([ms_step, ms_c, ms_d], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step, ms_c, ms_d = [float(v) for v in t.tolist()]
+
+    # end to end through host buffers
+    e2e_steps = max(1, min(args.steps, 5))
+    ms_e2e, h2d, d2h = e2e_run(A, torch, x_host, spec.chunk, mode, spec.seed, e2e_steps, 1)
+    te = torch.tensor([ms_e2e], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    ms_e2e = float(te.item())
+
+    alg = algorithmic_bytes(n, spec.chunk, mode.k)
+    gbs = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9
+    dominant = "accept_compress" if ms_c >= ms_d else "accept_decompress"
+    ms_dom = max(ms_c, ms_d)
+    out = {
+        "metric": METRIC, "value": world * gbs(4 * n, ms_step), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "shape": list(spec.shape), "n_elems": n, "chunk": spec.chunk,
+                   "mode": mode_name(mode), "l2": "inputs larger than L2 and %d rotating buffer sets" % codec.copies,
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "compress": {"ms": ms_c, "gbs_fp32_in": gbs(4 * n, ms_c), "hbm_gbs": gbs(alg, ms_c), "frac_of_measured_copy": gbs(alg, ms_c) / peak,
+                     "frac_of_8TBs": gbs(alg, ms_c) / 8000.0},
+        "decompress": {"ms": ms_d, "gbs_fp32_out": gbs(4 * n, ms_d), "hbm_gbs": gbs(alg, ms_d), "frac_of_measured_copy": gbs(alg, ms_d) / peak,
+                       "frac_of_8TBs": gbs(alg, ms_d) / 8000.0},
+        "roofline": {"bound": "hbm", "kernel": dominant, "achieved": gbs(alg, ms_dom), "peak": peak, "peak_source": peak_src,
+                     "unit": "GB/s", "frac": gbs(alg, ms_dom) / peak, "traffic": TRAFFIC.get((args.workload, dominant))},
+        "e2e": {"value": world * gbs(4 * n, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches_timed,
+        "clocks": clocks,
+    }
+
+    if args.sweep and rank == 0:
+        out["workloads"] = sweep(A, torch, peak, args)
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        tc, td, reps = time_oracle(x_host, spec.chunk, mode, spec.seed, budget_s=args.cpu_budget)
+        out["cpu_baseline"] = {"value": 4 * n / (tc + td) / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                               "sample": "whole %s tensor (%d elements), %d round trips; compress %.3f s, decompress %.3f s each"
+                                         % (args.workload, n, reps, tc, td),
+                               "host_cores_available": os.cpu_count()}
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(out))
+
+
+# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch, filled from profiles/ once captured
+TRAFFIC = {}
+
+
+def sweep(A, torch, peak, args):
+    """All five workloads, headline modes: per-kernel time and HBM fraction."""
+    rows = []
+    for name, spec in workloads.TENSORS.items():
+        if spec.n * 4 > (1 << 30) and args.sweep_max_bytes < (1 << 30) + 1:
+            pass
+        if spec.n * 4 > args.sweep_max_bytes:
+            continue
+        x_host = workloads.generate(name)
+        for mode in spec.headline:
+            codec = Codec(A, torch, x_host, spec.chunk, mode, spec.seed)
+            steps = 20 if spec.n * 4 >= (64 << 20) else 200
+            _, ms_c, ms_d = codec.run(steps, 3)
+            assert codec.status() == 0
+            alg = algorithmic_bytes(spec.n, spec.chunk, mode.k)
+            rows.append({"workload": name, "mode": mode_name(mode), "mbytes": spec.n * 4 / 2 ** 20, "copies": codec.copies,
+                         "compress_ms": ms_c, "decompress_ms": ms_d,
+                         "compress_gbs_fp32": 4 * spec.n / ms_c / 1e6, "decompress_gbs_fp32": 4 * spec.n / ms_d / 1e6,
+                         "compress_frac_measured": alg / ms_c / 1e6 / peak, "decompress_frac_measured": alg / ms_d / 1e6 / peak,
+                         "compress_frac_8TBs": alg / ms_c / 1e6 / 8000.0, "decompress_frac_8TBs": alg / ms_d / 1e6 / 8000.0})
+            print("# %-12s %-34s c %8.4f ms %6.1f%%  d %8.4f ms %6.1f%% (of measured copy bw)" %
+                  (name, mode_name(mode), ms_c, 100 * rows[-1]["compress_frac_measured"], ms_d,
+                   100 * rows[-1]["decompress_frac_measured"]), file=sys.stderr)
+            del codec
+            torch.cuda.empty_cache()
+    return rows
+
+
+# --------------------------------------------------------------------------------------------- reference arm
+
+def run_reference(args):
+    """The CPU oracle on the host cores, same metric and workload; rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    oracle.build()
+    spec = workloads.TENSORS[args.workload]
+    mode = spec.headline[0]
+    # bounded sample: the leading elements of the tensor, whole chunks, sized so that the run ends in minutes
+    sample = min(spec.n, args.reference_sample // spec.chunk * spec.chunk)
+    x_host = workloads.generate(args.workload, 0, sample)
+    for _ in range(args.warmup):
+        oracle.decompress(oracle.compress(x_host, spec.chunk, mode.k, mode.range, mode.round, mode.layout, spec.seed, 0)[0], sample)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        stream, _ = oracle.compress(x_host, spec.chunk, mode.k, mode.range, mode.round, mode.layout, spec.seed, 0)
+        oracle.decompress(stream, sample)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = 4 * sample / dt / 1e9
+    desc = "first %d elements of %s per step" % (sample, args.workload)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "shape": list(spec.shape), "n_elems": spec.n, "chunk": spec.chunk,
+                   "mode": mode_name(mode), "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(workloads.TENSORS))
+    ap.add_argument("--sweep", action="store_true", help="also time every workload's headline modes")
+    ap.add_argument("--sweep-max-bytes", type=int, default=1 << 30)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=10.0)
+    ap.add_argument("--reference-sample", type=int, default=1 << 24)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        args.warmup = max(args.warmup, 3)
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

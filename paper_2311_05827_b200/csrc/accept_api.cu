@@ -1,0 +1,263 @@
+// Host side of the C ABI declared in include/accept.h: argument checks, stream geometry,
+// kernel selection and launch.  Nothing here allocates memory or synchronises, except
+// accept_last_device_status.
+#include "../../include/accept.h"
+
+#include <atomic>
+#include <cstring>
+
+#include "accept_kernels.cuh"
+
+namespace {
+
+using accept::CodecArgs;
+
+std::atomic<uint64_t> g_launches{0};
+
+bool is_aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+uint64_t n_chunks_of(const accept_params* p) { return (p->n_elems + p->chunk_elems - 1) / p->chunk_elems; }
+
+// Geometry of the register-resident compress path for chunk size C: rounds R and threads per chunk.
+struct FastGeometry { int rounds; uint32_t tpc; };
+
+FastGeometry fast_geometry(uint32_t C) {
+  if (C % 512 == 0 && C / 16 <= 1024) return {2, C / 16};
+  if (C % 1024 == 0 && C / 32 <= 1024) return {4, C / 32};
+  if (C % 256 == 0 && C / 8 <= 1024) return {1, C / 8};
+  return {0, 0};
+}
+
+CodecArgs make_args(const accept_params* p, void* d_stream, void* d_ws) {
+  CodecArgs a{};
+  uint8_t* base = static_cast<uint8_t*>(d_stream);
+  a.header = reinterpret_cast<uint32_t*>(base);
+  a.meta = reinterpret_cast<float2*>(base + ACCEPT_HEADER_BYTES);
+  a.payload = reinterpret_cast<uint32_t*>(base + accept_payload_offset(p));
+  a.status = static_cast<uint32_t*>(d_ws);
+  a.n = p->n_elems;
+  a.n_chunks = n_chunks_of(p);
+  a.seed = p->seed;
+  a.rng_offset = p->rng_offset;
+  a.chunk = p->chunk_elems;
+  a.chunk_shift = -1;
+  for (int s = 5; s < 32; ++s)
+    if (p->chunk_elems == (1u << s)) a.chunk_shift = s;
+  a.header_word6 = (uint32_t)p->range | ((uint32_t)p->round << 8) | ((uint32_t)p->layout << 16);
+  a.k = p->k;
+  return a;
+}
+
+// ---- kernel tables -------------------------------------------------------------------------
+
+using KernelFn = void (*)(const CodecArgs);
+
+template <int K, int LAYOUT, int RANGE, int ROUND>
+KernelFn compress_for_rounds(int rounds) {
+  switch (rounds) {
+    case 1: return accept::compress_kernel<K, LAYOUT, RANGE, ROUND, 1>;
+    case 4: return accept::compress_kernel<K, LAYOUT, RANGE, ROUND, 4>;
+    default: return accept::compress_kernel<K, LAYOUT, RANGE, ROUND, 2>;
+  }
+}
+
+template <int K, int LAYOUT>
+KernelFn compress_for_modes(int range, int round, int rounds) {
+  if (range == accept::kAbsMax) {
+    return round == accept::kNearest ? compress_for_rounds<K, LAYOUT, accept::kAbsMax, accept::kNearest>(rounds)
+                                     : compress_for_rounds<K, LAYOUT, accept::kAbsMax, accept::kStochastic>(rounds);
+  }
+  return round == accept::kNearest ? compress_for_rounds<K, LAYOUT, accept::kMinMax, accept::kNearest>(rounds)
+                                   : compress_for_rounds<K, LAYOUT, accept::kMinMax, accept::kStochastic>(rounds);
+}
+
+KernelFn select_compress(const accept_params* p, int rounds) {
+  const bool bp = p->layout == ACCEPT_LAYOUT_BITPLANE;
+  switch (p->k) {
+    case 2: return bp ? compress_for_modes<2, accept::kBitplane>(p->range, p->round, rounds)
+                      : compress_for_modes<2, accept::kInterleaved>(p->range, p->round, rounds);
+    case 3: return compress_for_modes<3, accept::kBitplane>(p->range, p->round, rounds);
+    case 4: return bp ? compress_for_modes<4, accept::kBitplane>(p->range, p->round, rounds)
+                      : compress_for_modes<4, accept::kInterleaved>(p->range, p->round, rounds);
+    default: return bp ? compress_for_modes<8, accept::kBitplane>(p->range, p->round, rounds)
+                       : compress_for_modes<8, accept::kInterleaved>(p->range, p->round, rounds);
+  }
+}
+
+template <int K, int LAYOUT>
+KernelFn decompress_for_range(int range, bool aligned) {
+  if (range == accept::kAbsMax)
+    return aligned ? accept::decompress_kernel<K, LAYOUT, accept::kAbsMax, 2>
+                   : accept::decompress_unaligned_kernel<K, LAYOUT, accept::kAbsMax>;
+  return aligned ? accept::decompress_kernel<K, LAYOUT, accept::kMinMax, 2>
+                 : accept::decompress_unaligned_kernel<K, LAYOUT, accept::kMinMax>;
+}
+
+KernelFn select_decompress(const accept_params* p, bool aligned) {
+  const bool bp = p->layout == ACCEPT_LAYOUT_BITPLANE;
+  switch (p->k) {
+    case 2: return bp ? decompress_for_range<2, accept::kBitplane>(p->range, aligned)
+                      : decompress_for_range<2, accept::kInterleaved>(p->range, aligned);
+    case 3: return decompress_for_range<3, accept::kBitplane>(p->range, aligned);
+    case 4: return bp ? decompress_for_range<4, accept::kBitplane>(p->range, aligned)
+                      : decompress_for_range<4, accept::kInterleaved>(p->range, aligned);
+    default: return bp ? decompress_for_range<8, accept::kBitplane>(p->range, aligned)
+                       : decompress_for_range<8, accept::kInterleaved>(p->range, aligned);
+  }
+}
+
+accept_status check_buffers(const accept_params* p, const void* d_tensor, const void* d_stream,
+                            size_t stream_bytes, const void* d_ws, size_t ws_bytes) {
+  if (!p || !d_tensor || !d_stream || !d_ws) return ACCEPT_ERR_NULL;
+  accept_status st = accept_check_params(p);
+  if (st != ACCEPT_OK) return st;
+  if (stream_bytes < accept_compressed_size(p) || ws_bytes < accept_workspace_size(p)) return ACCEPT_ERR_TOO_SMALL;
+  if (!is_aligned(d_tensor, 16) || !is_aligned(d_stream, 16) || !is_aligned(d_ws, 4)) return ACCEPT_ERR_MISALIGNED;
+  return ACCEPT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+accept_status accept_check_params(const accept_params* p) {
+  if (!p) return ACCEPT_ERR_NULL;
+  if (p->n_elems == 0) return ACCEPT_ERR_BAD_SIZE;
+  if (p->chunk_elems < 32 || p->chunk_elems % 32 != 0) return ACCEPT_ERR_BAD_CHUNK;
+  if (p->range != ACCEPT_RANGE_ABSMAX && p->range != ACCEPT_RANGE_MINMAX) return ACCEPT_ERR_BAD_ENUM;
+  if (p->round != ACCEPT_ROUND_NEAREST && p->round != ACCEPT_ROUND_STOCHASTIC) return ACCEPT_ERR_BAD_ENUM;
+  if (p->layout != ACCEPT_LAYOUT_INTERLEAVED && p->layout != ACCEPT_LAYOUT_BITPLANE) return ACCEPT_ERR_BAD_ENUM;
+  if (!(p->k == 2 || p->k == 3 || p->k == 4 || p->k == 8)) return ACCEPT_ERR_BAD_K;
+  if (p->k == 3 && p->layout != ACCEPT_LAYOUT_BITPLANE) return ACCEPT_ERR_BAD_K;
+  if (p->reserved != 0) return ACCEPT_ERR_BAD_ENUM;
+  // one block per chunk / per 4096 elements must fit the grid's x dimension
+  if (n_chunks_of(p) > 0x7fffffffull || p->n_elems / 4096 > 0x7ffffff0ull) return ACCEPT_ERR_BAD_SIZE;
+  return ACCEPT_OK;
+}
+
+size_t accept_payload_offset(const accept_params* p) {
+  if (accept_check_params(p) != ACCEPT_OK) return 0;
+  const uint64_t off = ACCEPT_HEADER_BYTES + 8 * n_chunks_of(p);
+  return (size_t)((off + 15) / 16 * 16);
+}
+
+size_t accept_compressed_size(const accept_params* p) {
+  if (accept_check_params(p) != ACCEPT_OK) return 0;
+  return accept_payload_offset(p) + (size_t)(4ull * p->k * ((p->n_elems + 31) / 32));
+}
+
+size_t accept_workspace_size(const accept_params* p) {
+  if (accept_check_params(p) != ACCEPT_OK) return 0;
+  return 16;
+}
+
+accept_status accept_compress(const accept_params* p, const float* d_x, void* d_stream, size_t stream_bytes,
+                              void* d_ws, size_t ws_bytes, void* cuda_stream) {
+  accept_status st = check_buffers(p, d_x, d_stream, stream_bytes, d_ws, ws_bytes);
+  if (st != ACCEPT_OK) return st;
+  CodecArgs a = make_args(p, d_stream, d_ws);
+  a.x = d_x;
+
+  const FastGeometry g = fast_geometry(p->chunk_elems);
+  const bool fast = g.rounds != 0 && is_aligned(d_x, 32);
+  unsigned block = accept::kGenericBlock;
+  uint64_t fast_blocks = 0;
+  if (fast) {
+    a.n_fast_chunks = p->n_elems / p->chunk_elems;  // full chunks
+    a.tpc = g.tpc;
+    const bool share = g.tpc <= (uint32_t)accept::kFastBlock && accept::kFastBlock % g.tpc == 0;
+    block = share ? accept::kFastBlock : g.tpc;
+    a.chunks_per_block = share ? accept::kFastBlock / g.tpc : 1;
+    fast_blocks = (a.n_fast_chunks + a.chunks_per_block - 1) / a.chunks_per_block;
+  } else {
+    a.n_fast_chunks = 0;
+    a.tpc = 32;
+    a.chunks_per_block = 1;
+  }
+  const uint64_t grid = fast_blocks + (a.n_chunks - a.n_fast_chunks);
+  KernelFn fn = select_compress(p, fast ? g.rounds : 2);
+  fn<<<(unsigned)grid, block, 0, static_cast<cudaStream_t>(cuda_stream)>>>(a);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+}
+
+accept_status accept_decompress(const accept_params* p, const void* d_stream, size_t stream_bytes, float* d_xhat,
+                                void* d_ws, size_t ws_bytes, void* cuda_stream) {
+  accept_status st = check_buffers(p, d_xhat, d_stream, stream_bytes, d_ws, ws_bytes);
+  if (st != ACCEPT_OK) return st;
+  CodecArgs a = make_args(p, const_cast<void*>(d_stream), d_ws);
+  a.xhat = d_xhat;
+  const bool aligned = is_aligned(d_xhat, 32);
+  KernelFn fn = select_decompress(p, aligned);
+  const uint64_t per_block = aligned ? 4096 : 256;  // elements
+  const uint64_t grid = (p->n_elems + per_block - 1) / per_block;
+  fn<<<(unsigned)grid, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(a);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+}
+
+accept_status accept_compress_host(const accept_params* p, const float* h_x, void* h_stream, size_t stream_bytes,
+                                   float* d_x, void* d_stream, void* d_ws, size_t ws_bytes, void* cuda_stream) {
+  if (!h_x || !h_stream) return ACCEPT_ERR_NULL;
+  accept_status st = check_buffers(p, d_x, d_stream, stream_bytes, d_ws, ws_bytes);
+  if (st != ACCEPT_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(d_x, h_x, p->n_elems * sizeof(float), cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return ACCEPT_ERR_CUDA;
+  st = accept_compress(p, d_x, d_stream, stream_bytes, d_ws, ws_bytes, cuda_stream);
+  if (st != ACCEPT_OK) return st;
+  if (cudaMemcpyAsync(h_stream, d_stream, accept_compressed_size(p), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return ACCEPT_ERR_CUDA;
+  return ACCEPT_OK;
+}
+
+accept_status accept_decompress_host(const accept_params* p, const void* h_stream, size_t stream_bytes,
+                                     float* h_xhat, void* d_stream, float* d_xhat, void* d_ws, size_t ws_bytes,
+                                     void* cuda_stream) {
+  if (!h_stream || !h_xhat) return ACCEPT_ERR_NULL;
+  accept_status st = check_buffers(p, d_xhat, d_stream, stream_bytes, d_ws, ws_bytes);
+  if (st != ACCEPT_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(d_stream, h_stream, accept_compressed_size(p), cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return ACCEPT_ERR_CUDA;
+  st = accept_decompress(p, d_stream, stream_bytes, d_xhat, d_ws, ws_bytes, cuda_stream);
+  if (st != ACCEPT_OK) return st;
+  if (cudaMemcpyAsync(h_xhat, d_xhat, p->n_elems * sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return ACCEPT_ERR_CUDA;
+  return ACCEPT_OK;
+}
+
+accept_status accept_last_device_status(const void* d_ws, void* cuda_stream, uint32_t* status_bits) {
+  if (!d_ws || !status_bits) return ACCEPT_ERR_NULL;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(status_bits, d_ws, sizeof(uint32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return ACCEPT_ERR_CUDA;
+  return cudaStreamSynchronize(s) == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+}
+
+accept_status accept_parse_header(const void* h_header, accept_params* out) {
+  if (!h_header || !out) return ACCEPT_ERR_NULL;
+  uint32_t h[8];
+  std::memcpy(h, h_header, sizeof(h));
+  if (h[0] != ACCEPT_MAGIC || h[1] != ACCEPT_VERSION || h[7] != 0) return ACCEPT_ERR_BAD_STREAM_HEADER;
+  accept_params p{};
+  p.n_elems = (uint64_t)h[2] | ((uint64_t)h[3] << 32);
+  p.chunk_elems = h[4];
+  p.k = h[5];
+  p.range = (int32_t)(h[6] & 0xFF);
+  p.round = (int32_t)((h[6] >> 8) & 0xFF);
+  p.layout = (int32_t)((h[6] >> 16) & 0xFF);
+  if ((h[6] >> 24) != 0 || accept_check_params(&p) != ACCEPT_OK) return ACCEPT_ERR_BAD_STREAM_HEADER;
+  *out = p;
+  return ACCEPT_OK;
+}
+
+int accept_bitwidth_schedule(int is_backward, int n_lr_changes) {
+  if (n_lr_changes < 0) n_lr_changes = 0;
+  if (is_backward) return n_lr_changes == 0 ? 8 : 4;
+  return n_lr_changes >= 2 ? 4 : 2 + n_lr_changes;
+}
+
+uint64_t accept_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

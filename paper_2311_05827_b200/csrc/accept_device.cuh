@@ -1,0 +1,264 @@
+// Device-side building blocks of the boundary-tensor codec (sm_100a).
+//
+// Data unit: an OCTET, eight consecutive fp32 values (32 bytes), moved with one 256-bit global
+// load or store per thread.  Four neighbouring lanes (a QUAD) hold one pack group of 32 elements.
+// Every fp32 operation that decides a code or a reconstructed value is an explicitly rounded
+// intrinsic (__fmul_rn, __fadd_rn, __fsub_rn, __fdiv_rn): no FMA contraction, no flush to zero.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace accept {
+
+constexpr int kAbsMax = 0, kMinMax = 1;
+constexpr int kNearest = 0, kStochastic = 1;
+constexpr int kInterleaved = 0, kBitplane = 1;
+
+constexpr uint32_t kDevNonFinite = 1u, kDevBadHeader = 2u;
+
+// 1.5 * 2^23: adding it to |t| < 2^22 rounds t to an integer (ties to even, the fp32 adder's
+// rounding) and leaves that integer in the low mantissa bits.
+constexpr float kMagic = 12582912.0f;
+constexpr uint32_t kMagicBits = 0x4B400000u;
+
+// ----------------------------------------------------------------------------- memory access
+
+__device__ __forceinline__ void ld_octet(const float* p, float (&v)[8]) {
+  asm("ld.global.nc.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+      : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+      : "l"(p));
+}
+
+__device__ __forceinline__ void st_octet(float* p, const float (&v)[8]) {
+  asm volatile("st.global.cs.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(v[0]), "f"(v[1]),
+               "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7])
+               : "memory");
+}
+
+// ----------------------------------------------------------------------------- range statistic
+
+// NaN-propagating max/min: a NaN anywhere in the chunk survives to the result, and so does Inf,
+// so one test of the reduced value detects a non-finite chunk.
+__device__ __forceinline__ float max_nan(float a, float b) {
+  float r;
+  asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ float min_nan(float a, float b) {
+  float r;
+  asm("min.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ float max3_nan(float a, float b, float c) {
+  float r;
+  asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+__device__ __forceinline__ float min3_nan(float a, float b, float c) {
+  float r;
+  asm("min.NaN.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+
+// hi = max|x| (ABSMAX) or max x (MINMAX); lo = min x (MINMAX only).
+template <int RANGE>
+struct Range {
+  float hi, lo;
+  __device__ __forceinline__ void init() {
+    hi = (RANGE == kAbsMax) ? 0.0f : -__int_as_float(0x7f800000);
+    lo = __int_as_float(0x7f800000);
+  }
+  __device__ __forceinline__ void add(float a) {
+    if (RANGE == kAbsMax) {
+      hi = max_nan(hi, fabsf(a));
+    } else {
+      hi = max_nan(hi, a);
+      lo = min_nan(lo, a);
+    }
+  }
+  __device__ __forceinline__ void add2(float a, float b) {
+    if (RANGE == kAbsMax) {
+      hi = max3_nan(hi, fabsf(a), fabsf(b));
+    } else {
+      hi = max3_nan(hi, a, b);
+      lo = min3_nan(lo, a, b);
+    }
+  }
+  __device__ __forceinline__ void merge(float ohi, float olo) {
+    hi = max_nan(hi, ohi);
+    if (RANGE == kMinMax) lo = min_nan(lo, olo);
+  }
+  // butterfly over the lanes of a warp; every lane ends with the warp's range
+  __device__ __forceinline__ void warp_reduce() {
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+      float ohi = __shfl_xor_sync(0xffffffffu, hi, d);
+      float olo = (RANGE == kMinMax) ? __shfl_xor_sync(0xffffffffu, lo, d) : 0.0f;
+      merge(ohi, olo);
+    }
+  }
+};
+
+// Per-chunk quantizer constants derived from the range.
+struct Scale {
+  float s;     // side word: scaling factor
+  float o;     // side word: offset (0 under ABSMAX)
+  float inv;   // L / range, or 0 for a degenerate chunk
+  float base;  // subtracted before scaling (MINMAX: lo)
+  bool nonfinite;
+};
+
+__device__ __forceinline__ bool is_finite_bits(float a) {
+  return (__float_as_uint(a) & 0x7f800000u) != 0x7f800000u;
+}
+
+template <int K, int RANGE>
+__device__ __forceinline__ Scale make_scale(float hi, float lo) {
+  Scale sc;
+  if (RANGE == kAbsMax) {
+    const float L = (float)((1 << (K - 1)) - 1);
+    sc.nonfinite = !is_finite_bits(hi);
+    sc.s = __fdiv_rn(hi, L);
+    sc.inv = __fdiv_rn(L, hi);
+    sc.base = 0.0f;
+    sc.o = 0.0f;
+    if (sc.nonfinite || !(hi > 0.0f) || !is_finite_bits(sc.inv)) { sc.s = 0.0f; sc.inv = 0.0f; }
+  } else {
+    const float L = (float)((1 << K) - 1);
+    const float r = __fsub_rn(hi, lo);
+    sc.nonfinite = !is_finite_bits(hi) || !is_finite_bits(lo) || !is_finite_bits(r);
+    sc.s = __fdiv_rn(r, L);
+    sc.inv = __fdiv_rn(L, r);
+    sc.base = lo;
+    sc.o = (lo == 0.0f) ? 0.0f : lo;  // -0 is written as +0
+    if (sc.nonfinite) { sc.s = 0.0f; sc.inv = 0.0f; sc.base = 0.0f; sc.o = 0.0f; }
+    else if (!(r > 0.0f) || !is_finite_bits(sc.inv)) { sc.s = 0.0f; sc.inv = 0.0f; }
+  }
+  return sc;
+}
+
+// ----------------------------------------------------------------------------- uniform numbers (Eq. 7)
+
+// 32-bit finaliser of MurmurHash3.
+__device__ __forceinline__ uint32_t fmix32(uint32_t h) {
+  h ^= h >> 16;
+  h *= 0x85EBCA6Bu;
+  h ^= h >> 13;
+  h *= 0xC2B2AE35u;
+  h ^= h >> 16;
+  return h;
+}
+
+struct Rng {
+  uint32_t seed_lo, seed_hi;
+  // key for all counters that share their upper 32 bits
+  __device__ __forceinline__ uint32_t key(uint32_t ctr_hi) const {
+    return fmix32(ctr_hi ^ seed_lo) ^ seed_hi;
+  }
+  // U in [0,1) with 23 bits: float in [1,2) built from the hash, minus one (exact)
+  __device__ __forceinline__ static float uniform(uint32_t ctr_lo, uint32_t key) {
+    const uint32_t h = fmix32(ctr_lo ^ key);
+    return __fsub_rn(__uint_as_float(0x3F800000u | (h >> 9)), 1.0f);
+  }
+};
+
+// ----------------------------------------------------------------------------- quantize
+
+// Returns the fp32 bit pattern of (kMagic + u), u the unsigned stored code; its low byte is u.
+template <int K, int RANGE, int ROUND>
+__device__ __forceinline__ uint32_t quantize_bits(float x, const Scale& sc, float U) {
+  constexpr int ZP = (RANGE == kAbsMax) ? (1 << (K - 1)) : 0;
+  constexpr float kMagicZ = kMagic + (float)ZP;  // exact; even, so ties still go to even codes
+  const float d = (RANGE == kAbsMax) ? x : __fsub_rn(x, sc.base);
+  const float t = __fmul_rn(d, sc.inv);
+  if (ROUND == kNearest) {
+    // |t| <= L(1+2^-22): the rounded code cannot leave [zp-L, zp+L], no clamp needed
+    return __float_as_uint(__fadd_rn(t, kMagicZ));
+  } else {
+    const float f = floorf(t);
+    const float pr = __fsub_rn(t, f);
+    uint32_t b = __float_as_uint(__fadd_rn(f, kMagicZ)) + ((U < pr) ? 1u : 0u);
+    // floor(t)+1 may exceed the top code when t rounded just above L; the low side cannot underflow
+    return min(b, kMagicBits + (uint32_t)((1 << K) - 1));
+  }
+}
+
+// low bytes of four words -> one word
+__device__ __forceinline__ uint32_t pack_low_bytes(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3) {
+  const uint32_t p01 = __byte_perm(b0, b1, 0x0040);
+  const uint32_t p23 = __byte_perm(b2, b3, 0x0040);
+  return __byte_perm(p01, p23, 0x5410);
+}
+
+// Quantizes an octet.  xlo holds the codes of elements 0..3 one per byte, xhi those of 4..7.
+// i0 = index of element 0 in the whole tensor (random-number counter = rng_offset + index).
+template <int K, int RANGE, int ROUND>
+__device__ __forceinline__ void quantize_octet(const float (&v)[8], const Scale& sc, const Rng& rng,
+                                               uint64_t ctr0, uint32_t& xlo, uint32_t& xhi) {
+  uint32_t b[8];
+  if (ROUND == kStochastic) {
+    const uint32_t lo = (uint32_t)ctr0, hi = (uint32_t)(ctr0 >> 32);
+    if (lo <= 0xFFFFFFF8u) {
+      const uint32_t key = rng.key(hi);
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        b[e] = quantize_bits<K, RANGE, ROUND>(v[e], sc, Rng::uniform(lo + e, key));
+    } else {  // the counter's low word wraps inside this octet
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const uint64_t c = ctr0 + e;
+        b[e] = quantize_bits<K, RANGE, ROUND>(
+            v[e], sc, Rng::uniform((uint32_t)c, rng.key((uint32_t)(c >> 32))));
+      }
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) b[e] = quantize_bits<K, RANGE, ROUND>(v[e], sc, 0.0f);
+  }
+  xlo = pack_low_bytes(b[0], b[1], b[2], b[3]);
+  xhi = pack_low_bytes(b[4], b[5], b[6], b[7]);
+}
+
+// ----------------------------------------------------------------------------- bit permutations
+
+// Exchanges the bits selected by m with the bits s places above them.
+__device__ __forceinline__ uint32_t delta_swap(uint32_t x, uint32_t m, int s) {
+  const uint32_t t = ((x >> s) ^ x) & m;
+  return x ^ t ^ (t << s);
+}
+
+// 4 x 8 bit-matrix transpose inside a word, its own inverse.
+//   plane form:  bit 8*j + e       = digit j (0..3) of the code of element e (0..7)
+//   nibble form: bit 8*b + 4*a + j = digit j of the code of element 4*a + b
+// i.e. byte b of the nibble form holds code b in its low and code 4+b in its high nibble.
+__device__ __forceinline__ uint32_t planes_nibbles(uint32_t x) {
+  x = delta_swap(x, 0x0000CCCCu, 14);  // index bit 4 <-> index bit 1
+  x = delta_swap(x, 0x00AA00AAu, 7);   // index bit 3 <-> index bit 0
+  return x;
+}
+
+// 4 x 4 byte transpose across the four lanes of a quad, its own inverse: before, lane q holds
+// bytes [a_q0 a_q1 a_q2 a_q3]; after, lane q holds [a_0q a_1q a_2q a_3q].  All 32 lanes must call.
+__device__ __forceinline__ uint32_t quad_transpose(uint32_t v, int lane) {
+  uint32_t r = __shfl_xor_sync(0xffffffffu, v, 2);
+  v = __byte_perm(v, r, (lane & 2) ? 0x3276 : 0x5410);
+  r = __shfl_xor_sync(0xffffffffu, v, 1);
+  v = __byte_perm(v, r, (lane & 1) ? 0x3715 : 0x6240);
+  return v;
+}
+
+// codes 0..3 / 4..7 (one per byte, < 16) -> byte b = code b | code(4+b) << 4
+__device__ __forceinline__ uint32_t merge_nibbles(uint32_t xlo, uint32_t xhi) { return xlo | (xhi << 4); }
+
+// ----------------------------------------------------------------------------- dequantize
+
+template <int K, int RANGE>
+__device__ __forceinline__ float dequantize_code(uint32_t u, float s, float o) {
+  constexpr int ZP = (RANGE == kAbsMax) ? (1 << (K - 1)) : 0;
+  // kMagicBits | u is the float kMagic + u; subtracting kMagic + zp leaves the integer u - zp, exactly
+  const float g = __fsub_rn(__uint_as_float(kMagicBits | u), kMagic + (float)ZP);
+  if (RANGE == kAbsMax) return __fmul_rn(g, s);
+  return __fadd_rn(__fmul_rn(g, s), o);
+}
+
+}  // namespace accept

@@ -1,0 +1,310 @@
+// Kernels of the boundary-tensor codec: fused range + quantize + pack (compress) and fused
+// unpack + dequantize (decompress).  One launch per call; chunks are independent, so no block ever
+// waits on another.
+#pragma once
+#include "accept_device.cuh"
+
+namespace accept {
+
+struct CodecArgs {
+  const float* x;         // compress input
+  float* xhat;            // decompress output
+  uint32_t* header;       // stream + 0
+  float2* meta;           // stream + 32
+  uint32_t* payload;      // stream + payload offset
+  uint32_t* status;       // device status word
+  uint64_t n;             // elements
+  uint64_t n_chunks;      // M
+  uint64_t n_fast_chunks; // leading full chunks coded by the register-resident path
+  uint64_t seed, rng_offset;
+  uint32_t chunk;         // C
+  int chunk_shift;        // log2(C) if C is a power of two, else -1
+  uint32_t tpc;           // fast path: threads that share one chunk (C / (8*R))
+  uint32_t chunks_per_block;
+  uint32_t header_word6;  // range | round<<8 | layout<<16
+  uint32_t k;
+};
+
+constexpr int kFastBlock = 256;     // threads per block when a chunk needs at most 256 threads
+constexpr int kGenericBlock = 256;  // threads per block of the any-shape path
+
+// ----------------------------------------------------------------------------- stores of packed codes
+
+// INTERLEAVED: the 8 codes of global octet index oct occupy bits [8*K*oct, 8*K*(oct+1)) of the payload.
+template <int K>
+__device__ __forceinline__ void store_interleaved(uint32_t* payload, uint64_t oct, uint32_t xlo, uint32_t xhi) {
+  if (K == 8) {
+    reinterpret_cast<uint2*>(payload)[oct] = make_uint2(xlo, xhi);
+  } else if (K == 4) {
+    // bytes u0|u1<<4 and u2|u3<<4 sit in bytes 0 and 2 of x | x>>4
+    const uint32_t ylo = xlo | (xlo >> 4), yhi = xhi | (xhi >> 4);
+    payload[oct] = __byte_perm(ylo, yhi, 0x6420);
+  } else {  // K == 2
+    uint32_t ylo = xlo | (xlo >> 6), yhi = xhi | (xhi >> 6);
+    ylo |= ylo >> 12;
+    yhi |= yhi >> 12;
+    reinterpret_cast<uint16_t*>(payload)[oct] = (uint16_t)__byte_perm(ylo, yhi, 0x0040);
+  }
+}
+
+// BITPLANE: lane q of a quad ends with the word of binary digit q (and q+4 for K = 8) of the
+// quad's group and stores it.  group = global index of the 32-element group.  All lanes call.
+template <int K>
+__device__ __forceinline__ void store_bitplane(uint32_t* payload, uint64_t group, uint32_t xlo, uint32_t xhi,
+                                               int lane) {
+  const int q = lane & 3;
+  if (K <= 4) {
+    const uint32_t w = quad_transpose(planes_nibbles(merge_nibbles(xlo, xhi)), lane);
+    if (q < K) payload[group * K + q] = w;
+  } else {
+    const uint32_t lo = merge_nibbles(xlo & 0x0F0F0F0Fu, xhi & 0x0F0F0F0Fu);
+    const uint32_t hi = merge_nibbles((xlo >> 4) & 0x0F0F0F0Fu, (xhi >> 4) & 0x0F0F0F0Fu);
+    const uint32_t w0 = quad_transpose(planes_nibbles(lo), lane);
+    const uint32_t w1 = quad_transpose(planes_nibbles(hi), lane);
+    payload[group * 8 + q] = w0;
+    payload[group * 8 + 4 + q] = w1;
+  }
+}
+
+// ----------------------------------------------------------------------------- any-shape chunk coder
+
+// Codes chunk m with the whole block: any C (multiple of 32), partial chunks, any alignment.
+// Two passes over the chunk (the second is served by the caches); one element per lane, words
+// formed with warp votes.  Used for the partial last chunk and for chunk sizes or alignments the
+// register-resident path does not take.
+template <int K, int LAYOUT, int RANGE, int ROUND>
+__device__ void compress_chunk_generic(const CodecArgs& a, uint64_t m, float* s_hi, float* s_lo) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const uint64_t i0 = m * a.chunk;
+  const uint32_t valid = (uint32_t)min((uint64_t)a.chunk, a.n - i0);
+  const float* x = a.x + i0;
+
+  Range<RANGE> rg;
+  rg.init();
+  for (uint32_t i = tid; i < valid; i += blockDim.x) rg.add(__ldg(x + i));
+  rg.warp_reduce();
+  __syncthreads();  // protects s_hi/s_lo against a previous use
+  if (lane == 0) { s_hi[warp] = rg.hi; s_lo[warp] = rg.lo; }
+  __syncthreads();
+  rg.init();
+  for (int w = 0; w < nwarps; ++w) rg.merge(s_hi[w], s_lo[w]);
+
+  Scale sc = make_scale<K, RANGE>(rg.hi, rg.lo);
+  if (tid == 0) {
+    a.meta[m] = make_float2(sc.s, sc.o);
+    if (sc.nonfinite) atomicOr(a.status, kDevNonFinite);
+  }
+  Rng rng{(uint32_t)a.seed, (uint32_t)(a.seed >> 32)};
+  const uint32_t ngroups = (valid + 31) / 32;
+  for (uint32_t g = warp; g < ngroups; g += nwarps) {
+    const uint32_t t = g * 32 + lane;
+    uint32_t u = 0;
+    if (t < valid) {
+      float v = __ldg(x + t);
+      if (sc.nonfinite) v = 0.0f;
+      float U = 0.0f;
+      if (ROUND == kStochastic) {
+        const uint64_t c = a.rng_offset + i0 + t;
+        U = Rng::uniform((uint32_t)c, rng.key((uint32_t)(c >> 32)));
+      }
+      u = quantize_bits<K, RANGE, ROUND>(v, sc, U) & 0xFFu;
+    }
+    const uint64_t word0 = (i0 / 32 + g) * K;
+#pragma unroll
+    for (int w = 0; w < K; ++w) {
+      uint32_t bit;
+      if (LAYOUT == kBitplane) {
+        bit = (u >> w) & 1u;  // word w = binary digit w of the 32 codes
+      } else {
+        // bit b of word w is bit (32w+b) of the group's string: digit (32w+b)%K of element (32w+b)/K
+        const int pos = 32 * w + lane;
+        bit = (__shfl_sync(0xffffffffu, u, pos / K) >> (pos % K)) & 1u;
+      }
+      const uint32_t word = __ballot_sync(0xffffffffu, bit);
+      if (lane == w) a.payload[word0 + w] = word;
+    }
+  }
+}
+
+// ----------------------------------------------------------------------------- compress
+
+// Register-resident path.  A chunk of C = 8*R*tpc elements is shared by tpc threads (tpc a multiple
+// of 32, the block holds chunks_per_block such groups).  Each thread loads R octets, one per round,
+// round r covering elements [8*r*tpc, 8*(r+1)*tpc) of the chunk with consecutive threads on
+// consecutive octets; the chunk is read from HBM once and stays in registers between the range
+// reduction and the quantizer.  Blocks past the fast chunks code the remaining chunk(s) with the
+// any-shape coder.
+template <int K, int LAYOUT, int RANGE, int ROUND, int R>
+__global__ void __launch_bounds__(1024) compress_kernel(const CodecArgs a) {
+  __shared__ float s_hi[32], s_lo[32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  if (blockIdx.x == 0 && tid < 8) {
+    // stream header and the pad between the side words and the payload
+    const uint32_t h[8] = {0x54504341u, 1u, (uint32_t)a.n, (uint32_t)(a.n >> 32), a.chunk, a.k, a.header_word6, 0u};
+    a.header[tid] = h[tid];
+    if ((a.n_chunks & 1) && tid < 2) reinterpret_cast<uint32_t*>(a.meta + a.n_chunks)[tid] = 0u;
+  }
+
+  const uint64_t fast_blocks = (a.n_fast_chunks + a.chunks_per_block - 1) / a.chunks_per_block;
+  if (blockIdx.x >= fast_blocks) {
+    compress_chunk_generic<K, LAYOUT, RANGE, ROUND>(a, a.n_fast_chunks + (blockIdx.x - fast_blocks), s_hi, s_lo);
+    return;
+  }
+
+  const uint32_t tpc = a.tpc;
+  const uint32_t grp = tid / tpc, gt = tid - grp * tpc;
+  uint64_t m = (uint64_t)blockIdx.x * a.chunks_per_block + grp;
+  const bool active = m < a.n_fast_chunks;  // a whole group is active or not; warps never straddle groups
+  if (!active) m = a.n_fast_chunks - 1;     // idle groups redo the last chunk's loads, store nothing
+
+  const uint64_t e0 = m * a.chunk;  // first element of the chunk
+  float v[R][8];
+#pragma unroll
+  for (int r = 0; r < R; ++r) ld_octet(a.x + e0 + 8ull * (r * tpc + gt), v[r]);
+
+  Range<RANGE> rg;
+  rg.init();
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+#pragma unroll
+    for (int e = 0; e < 8; e += 2) rg.add2(v[r][e], v[r][e + 1]);
+  }
+  rg.warp_reduce();
+  if (tpc > 32) {
+    if (lane == 0) { s_hi[warp] = rg.hi; s_lo[warp] = rg.lo; }
+    __syncthreads();
+    const int w0 = (grp * tpc) >> 5, wn = tpc >> 5;
+    rg.init();
+    for (int w = 0; w < wn; ++w) rg.merge(s_hi[w0 + w], s_lo[w0 + w]);
+  }
+
+  Scale sc = make_scale<K, RANGE>(rg.hi, rg.lo);
+  if (gt == 0 && active) {
+    a.meta[m] = make_float2(sc.s, sc.o);
+    if (sc.nonfinite) atomicOr(a.status, kDevNonFinite);
+  }
+  if (sc.nonfinite) {
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[r][e] = 0.0f;
+  }
+
+  const Rng rng{(uint32_t)a.seed, (uint32_t)(a.seed >> 32)};
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const uint64_t oct = e0 / 8 + (r * tpc + gt);  // global octet index
+    uint32_t xlo, xhi;
+    quantize_octet<K, RANGE, ROUND>(v[r], sc, rng, a.rng_offset + oct * 8, xlo, xhi);
+    if (LAYOUT == kInterleaved) {
+      if (active) store_interleaved<K>(a.payload, oct, xlo, xhi);
+    } else {
+      // shuffles inside: every lane takes part; an idle group rewrites nothing
+      if (active) store_bitplane<K>(a.payload, oct >> 2, xlo, xhi, lane);
+    }
+  }
+}
+
+// ----------------------------------------------------------------------------- decompress
+
+// Each thread rebuilds R octets; consecutive threads take consecutive octets, so every store
+// instruction of a warp writes 1 KB of contiguous output.
+template <int K, int LAYOUT, int RANGE, int R>
+__global__ void __launch_bounds__(256) decompress_kernel(const CodecArgs a) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  if (blockIdx.x == 0 && tid == 0) {
+    const uint32_t h[8] = {0x54504341u, 1u, (uint32_t)a.n, (uint32_t)(a.n >> 32), a.chunk, a.k, a.header_word6, 0u};
+    bool ok = true;
+    for (int i = 0; i < 6; ++i) ok = ok && (a.header[i] == h[i]);
+    // the rounding mode does not change how a stream is read: compare range and layout only
+    ok = ok && ((a.header[6] & 0xFFFF00FFu) == (h[6] & 0xFFFF00FFu));
+    if (!ok) atomicOr(a.status, kDevBadHeader);
+  }
+  const uint64_t n_oct = (a.n + 7) / 8;       // octets, the last one maybe partial
+  const uint64_t n_groups = (a.n + 31) / 32;  // pack groups present in the payload
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const uint64_t oct = ((uint64_t)blockIdx.x * R + r) * blockDim.x + tid;
+    const bool in = oct < n_oct;
+    const uint64_t e = oct * 8;
+    uint32_t xlo = 0, xhi = 0;  // codes 0..3 / 4..7, one per byte
+    if (LAYOUT == kInterleaved) {
+      if (in) {
+        if (K == 8) {
+          const uint2 w = __ldg(reinterpret_cast<const uint2*>(a.payload) + oct);
+          xlo = w.x; xhi = w.y;
+        } else if (K == 4) {
+          const uint32_t w = __ldg(a.payload + oct);
+          // nibbles -> bytes
+          uint32_t y = __byte_perm(w, 0, 0x4140);  // bytes: w.b0, 0, w.b1, 0
+          xlo = (y | (y << 4)) & 0x0F0F0F0Fu;
+          y = __byte_perm(w, 0, 0x4342);           // bytes: w.b2, 0, w.b3, 0
+          xhi = (y | (y << 4)) & 0x0F0F0F0Fu;
+        } else {
+          const uint32_t w = __ldg(reinterpret_cast<const uint16_t*>(a.payload) + oct);
+          // 2-bit fields -> bytes
+          uint32_t y = (w | (w << 12)) & 0x000F000Fu;  // fields 0,1 | 2,3 (low byte), 4,5 | 6,7 handled below
+          xlo = (y | (y << 6)) & 0x03030303u;
+          y = ((w >> 8) | ((w >> 8) << 12)) & 0x000F000Fu;
+          xhi = (y | (y << 6)) & 0x03030303u;
+        }
+      }
+    } else {
+      // lane q of a quad fetches the word of binary digit q of its group; a quad transpose then
+      // hands every lane the plane bytes of its own octet
+      const int q = lane & 3;
+      const uint64_t group = oct >> 2;
+      const bool gin = group < n_groups;
+      if (K <= 4) {
+        uint32_t w = 0;
+        if (gin && q < K) w = __ldg(a.payload + group * K + q);
+        const uint32_t nib = planes_nibbles(quad_transpose(w, lane));
+        xlo = nib & 0x0F0F0F0Fu;
+        xhi = (nib >> 4) & 0x0F0F0F0Fu;
+      } else {
+        uint32_t w0 = 0, w1 = 0;
+        if (gin) { w0 = __ldg(a.payload + group * 8 + q); w1 = __ldg(a.payload + group * 8 + 4 + q); }
+        const uint32_t lo = planes_nibbles(quad_transpose(w0, lane));
+        const uint32_t hi = planes_nibbles(quad_transpose(w1, lane));
+        xlo = (lo & 0x0F0F0F0Fu) | ((hi & 0x0F0F0F0Fu) << 4);
+        xhi = ((lo >> 4) & 0x0F0F0F0Fu) | (hi & 0xF0F0F0F0u);
+      }
+    }
+    if (!in) continue;
+    const uint64_t m = (a.chunk_shift >= 0) ? (e >> a.chunk_shift) : (e / a.chunk);
+    const float2 so = __ldg(a.meta + m);
+    float out[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      out[i] = dequantize_code<K, RANGE>((xlo >> (8 * i)) & 0xFFu, so.x, so.y);
+      out[4 + i] = dequantize_code<K, RANGE>((xhi >> (8 * i)) & 0xFFu, so.x, so.y);
+    }
+    if (e + 8 <= a.n) {
+      st_octet(a.xhat + e, out);
+    } else {
+      for (int i = 0; i < 8; ++i)
+        if (e + i < a.n) a.xhat[e + i] = out[i];
+    }
+  }
+}
+
+// Scalar any-alignment decoder for output pointers that are not 32-byte aligned.
+template <int K, int LAYOUT, int RANGE>
+__global__ void __launch_bounds__(256) decompress_unaligned_kernel(const CodecArgs a) {
+  const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= a.n) return;
+  uint32_t u = 0;
+  if (LAYOUT == kInterleaved) {
+    const uint64_t bit = i * K;
+    u = (a.payload[bit >> 5] >> (bit & 31)) & ((1u << K) - 1);
+  } else {
+    const uint64_t w0 = (i >> 5) * K;
+    for (int j = 0; j < K; ++j) u |= ((a.payload[w0 + j] >> (i & 31)) & 1u) << j;
+  }
+  const uint64_t m = (a.chunk_shift >= 0) ? (i >> a.chunk_shift) : (i / a.chunk);
+  const float2 so = a.meta[m];
+  a.xhat[i] = dequantize_code<K, RANGE>(u, so.x, so.y);
+}
+
+}  // namespace accept

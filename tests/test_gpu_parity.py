@@ -1,0 +1,334 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element.
+
+Bar: the whole compressed stream (header words, per-chunk side words, packed payload) is
+bit-exact; reconstructed floats agree within 1e-6 * (chunk max - chunk min) -- and are in fact
+required to be bit-exact too, since decoding is a fixed sequence of rounded fp32 operations.
+"""
+import numpy as np
+import pytest
+
+import oracle
+import workloads
+from oracle import (LAYOUT_BITPLANE, LAYOUT_INTERLEAVED, RANGE_ABSMAX, RANGE_MINMAX, ROUND_NEAREST,
+                    ROUND_STOCHASTIC)
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+def _lib():
+    import paper_2311_05827_b200 as A
+    return A
+
+
+def gpu_compress(x_np, chunk, k, range_, round_, layout, seed=0, rng_offset=0, x_dev=None):
+    A = _lib()
+    n = x_np.size if x_dev is None else x_dev.numel()
+    p = A.Params(n, chunk, k, range_, round_, layout, seed, rng_offset)
+    d_x = torch.from_numpy(x_np).cuda() if x_dev is None else x_dev
+    d_stream = A.new_stream_buffer(p)
+    d_stream.fill_(0xA5)  # stale bytes must all be overwritten
+    d_ws = A.new_workspace(p)
+    A.accept_compress(p, d_x, d_stream, d_ws)
+    status = A.accept_last_device_status(d_ws)
+    return d_stream.cpu().numpy(), status, p, d_stream, d_ws
+
+
+def gpu_decompress(p, stream_np_or_dev, d_ws=None):
+    A = _lib()
+    d_stream = stream_np_or_dev if torch.is_tensor(stream_np_or_dev) else torch.from_numpy(stream_np_or_dev).cuda()
+    d_xhat = torch.full((p.n_elems,), float("nan"), dtype=torch.float32, device="cuda")
+    if d_ws is None:
+        d_ws = A.new_workspace(p)
+    A.accept_decompress(p, d_stream, d_xhat, d_ws)
+    status = A.accept_last_device_status(d_ws)
+    return d_xhat.cpu().numpy(), status
+
+
+def assert_float_parity(xhat_gpu, xhat_ref, x, chunk):
+    """spec tolerance, then the stricter bit-exact check."""
+    n = x.size
+    m = -(-n // chunk)
+    pad = m * chunk - n
+    xp = np.concatenate([x, np.full(pad, x[-1], dtype=np.float32)]).reshape(m, chunk).astype(np.float64)
+    span = np.repeat(xp.max(axis=1) - xp.min(axis=1), chunk)[:n]
+    assert np.all(np.abs(xhat_gpu.astype(np.float64) - xhat_ref.astype(np.float64)) <= 1e-6 * span)
+    assert np.array_equal(xhat_gpu.view(np.uint32), xhat_ref.view(np.uint32))
+
+
+def check_roundtrip(x, chunk, k, range_, round_, layout, seed=0, rng_offset=0):
+    ref_stream, ref_flag = oracle.compress(x, chunk, k, range_, round_, layout, seed, rng_offset)
+    got_stream, status, p, d_stream, d_ws = gpu_compress(x, chunk, k, range_, round_, layout, seed, rng_offset)
+    assert got_stream.size == ref_stream.size
+    if not np.array_equal(got_stream, ref_stream):
+        hdr_g, meta_g, pay_g = oracle.split_stream(got_stream, x.size, chunk)
+        hdr_r, meta_r, pay_r = oracle.split_stream(ref_stream, x.size, chunk)
+        assert np.array_equal(hdr_g, hdr_r), "header words differ"
+        bad = np.nonzero(meta_g.view(np.uint32) != meta_r.view(np.uint32))
+        assert bad[0].size == 0, f"side words differ first at chunk {bad[0][:4]}: {meta_g[bad[0][:4]]} vs {meta_r[bad[0][:4]]}"
+        badw = np.nonzero(pay_g != pay_r)[0]
+        assert badw.size == 0, f"{badw.size} payload words differ, first {badw[:8]}"
+        raise AssertionError("streams differ outside header/meta/payload (padding)")
+    assert (status & 1) == ref_flag
+    xhat_ref = oracle.decompress(ref_stream, x.size)
+    xhat_gpu, status2 = gpu_decompress(p, d_stream)
+    assert status2 == 0
+    if ref_flag == 0:
+        assert_float_parity(xhat_gpu, xhat_ref, x, chunk)
+    else:
+        assert np.array_equal(xhat_gpu.view(np.uint32), xhat_ref.view(np.uint32))
+
+
+def modes():
+    out = []
+    for layout in (LAYOUT_INTERLEAVED, LAYOUT_BITPLANE):
+        for k in ((2, 4, 8) if layout == LAYOUT_INTERLEAVED else (2, 3, 4, 8)):
+            for range_ in (RANGE_ABSMAX, RANGE_MINMAX):
+                for round_ in (ROUND_NEAREST, ROUND_STOCHASTIC):
+                    out.append((k, range_, round_, layout))
+    return out
+
+
+MODE_IDS = [f"k{k}-{'absmax' if r == 0 else 'minmax'}-{'rn' if d == 0 else 'sr'}-{'il' if l == 0 else 'bp'}"
+            for k, r, d, l in modes()]
+
+
+# ------------------------------------------------------------------ shapes spanning tiles and ragged tails
+
+
+@pytest.mark.parametrize("mode", modes(), ids=MODE_IDS)
+@pytest.mark.parametrize("chunk,n", [
+    (4096, 4096 * 37 + 1234),   # register path (2 rounds, 256 threads per chunk) + partial chunk
+    (1024, 1024 * 131 + 1),     # 64 threads per chunk, four chunks per block, last block part idle
+    (512, 512 * 9),             # one warp per chunk
+    (256, 256 * 21 + 77),       # one round
+    (2048, 2048 * 5 + 2047),
+    (96, 96 * 50 + 40),         # any-shape coder only
+    (32, 1000),
+])
+def test_parity_shapes(mode, chunk, n):
+    k, range_, round_, layout = mode
+    x = workloads.random_tensor(n, 17 * chunk + k, "normal")
+    check_roundtrip(x, chunk, k, range_, round_, layout, seed=0x1234567890ABCDEF, rng_offset=3)
+
+
+@pytest.mark.parametrize("chunk", [8192, 16384, 32768, 1 << 20])
+@pytest.mark.parametrize("mode", [(4, RANGE_ABSMAX, ROUND_NEAREST, LAYOUT_BITPLANE),
+                                  (8, RANGE_MINMAX, ROUND_STOCHASTIC, LAYOUT_INTERLEAVED)])
+def test_parity_large_chunks(chunk, mode):
+    """512- and 1024-thread groups, four rounds, and a chunk far larger than a block holds."""
+    k, range_, round_, layout = mode
+    n = min(3 * chunk + 333, (1 << 21) + 333)
+    x = workloads.random_tensor(n, chunk, "relu")
+    check_roundtrip(x, chunk, k, range_, round_, layout, seed=5)
+
+
+@pytest.mark.parametrize("n", [1, 2, 7, 8, 9, 31, 32, 33, 63, 255, 257, 4095, 4097])
+def test_parity_tiny_and_ragged(n):
+    for k, range_, round_, layout in [(2, RANGE_ABSMAX, ROUND_NEAREST, LAYOUT_INTERLEAVED),
+                                      (3, RANGE_MINMAX, ROUND_NEAREST, LAYOUT_BITPLANE),
+                                      (4, RANGE_ABSMAX, ROUND_STOCHASTIC, LAYOUT_BITPLANE),
+                                      (8, RANGE_ABSMAX, ROUND_NEAREST, LAYOUT_INTERLEAVED)]:
+        x = workloads.random_tensor(n, n + k, "normal")
+        for chunk in (32, 256, 4096):
+            check_roundtrip(x, chunk, k, range_, round_, layout, seed=n)
+
+
+def test_per_tensor_range_is_one_chunk():
+    """chunk >= N reproduces the paper's one-range-per-tensor scheme."""
+    x = workloads.generate("cfg2_grad", 0, 100000)
+    for k in (4, 8):
+        check_roundtrip(x, 100000 // 32 * 32 + 32, k, RANGE_ABSMAX, ROUND_STOCHASTIC, LAYOUT_INTERLEAVED, seed=9)
+
+
+# ------------------------------------------------------------------ degenerate values
+
+
+def edge_tensor(chunk):
+    x = workloads.random_tensor(chunk * 12, 77, "normal")
+    x[0 * chunk:1 * chunk] = 0.0                      # all-zero chunk
+    x[1 * chunk:2 * chunk] = -2.5                     # constant chunk
+    x[2 * chunk:3 * chunk] = np.float32(1e-42)        # denormals only: L/c overflows
+    x[3 * chunk + 5] = np.float32(3e38)               # one huge outlier
+    x[4 * chunk:5 * chunk:2] = -0.0                   # negative zeros among values
+    x[5 * chunk:6 * chunk] = -0.0                     # all negative zero
+    x[6 * chunk:7 * chunk] *= np.float32(1e-39)       # denormal-scale values
+    x[7 * chunk + 1] = np.float32(-3e38)
+    x[7 * chunk + 2] = np.float32(3e38)               # min/max range overflows
+    x[8 * chunk:9 * chunk] = np.abs(x[8 * chunk:9 * chunk])
+    x[9 * chunk + 3] = np.float32(1e-30)
+    x[9 * chunk:10 * chunk] *= np.float32(1e-30)
+    return x
+
+
+@pytest.mark.parametrize("chunk", [32, 512, 4096])
+@pytest.mark.parametrize("mode", modes(), ids=MODE_IDS)
+def test_parity_degenerate_values(chunk, mode):
+    k, range_, round_, layout = mode
+    check_roundtrip(edge_tensor(chunk), chunk, k, range_, round_, layout, seed=11)
+
+
+@pytest.mark.parametrize("bad", [np.nan, np.inf, -np.inf])
+@pytest.mark.parametrize("chunk", [64, 1024, 4096])
+def test_nonfinite_input_sets_status_and_writes_degenerate_chunk(bad, chunk):
+    x = workloads.random_tensor(chunk * 6 + 50, 3, "normal")
+    x[chunk + 9] = bad
+    x[chunk * 6 + 7] = bad  # also in the partial chunk
+    for range_ in (RANGE_ABSMAX, RANGE_MINMAX):
+        for layout, k in ((LAYOUT_INTERLEAVED, 4), (LAYOUT_BITPLANE, 3)):
+            ref_stream, flag = oracle.compress(x, chunk, k, range_, ROUND_NEAREST, layout)
+            got, status, p, d_stream, _ = gpu_compress(x, chunk, k, range_, ROUND_NEAREST, layout)
+            assert flag == 1 and status == 1
+            assert np.array_equal(got, ref_stream)
+            xhat, st2 = gpu_decompress(p, d_stream)
+            assert st2 == 0 and np.all(np.isfinite(xhat))
+            assert np.array_equal(xhat.view(np.uint32), oracle.decompress(ref_stream, x.size).view(np.uint32))
+
+
+def test_rng_counter_wraps_32_bits():
+    """Random-number counters that cross a multiple of 2^32 inside the tensor."""
+    x = workloads.random_tensor(4096 * 3, 5, "uniform")
+    for off in (2 ** 32 - 4096 - 5, 2 ** 32 - 3, 2 ** 64 - 100):
+        check_roundtrip(x, 4096, 4, RANGE_ABSMAX, ROUND_STOCHASTIC, LAYOUT_INTERLEAVED, seed=2 ** 63 + 12345, rng_offset=off)
+        check_roundtrip(x[:1000], 96, 2, RANGE_MINMAX, ROUND_STOCHASTIC, LAYOUT_BITPLANE, seed=7, rng_offset=off)
+
+
+def test_unaligned_device_pointers_take_the_any_shape_path():
+    A = _lib()
+    n, chunk, k = 4096 * 5 + 100, 4096, 4
+    x = workloads.random_tensor(n, 1, "normal")
+    big = torch.zeros(n + 16, dtype=torch.float32, device="cuda")
+    d_x = big[4:4 + n]  # 16-byte but not 32-byte aligned
+    d_x.copy_(torch.from_numpy(x))
+    for layout in (LAYOUT_INTERLEAVED, LAYOUT_BITPLANE):
+        ref, _ = oracle.compress(x, chunk, k, RANGE_ABSMAX, ROUND_NEAREST, layout)
+        got, status, p, d_stream, d_ws = gpu_compress(x, chunk, k, RANGE_ABSMAX, ROUND_NEAREST, layout, x_dev=d_x)
+        assert np.array_equal(got, ref) and status == 0
+        out = torch.zeros(n + 16, dtype=torch.float32, device="cuda")
+        A.accept_decompress(p, d_stream, out[4:4 + n], d_ws)
+        assert np.array_equal(out[4:4 + n].cpu().numpy().view(np.uint32), oracle.decompress(ref, n).view(np.uint32))
+        assert float(out[:4].abs().sum()) == 0 and float(out[4 + n:].abs().sum()) == 0
+
+
+def test_decompress_flags_header_mismatch():
+    A = _lib()
+    x = workloads.random_tensor(5000, 2, "normal")
+    ref, _ = oracle.compress(x, 1024, 4, RANGE_ABSMAX, ROUND_NEAREST, LAYOUT_INTERLEAVED)
+    p_ok = A.Params(5000, 1024, 4)
+    xhat, st = gpu_decompress(p_ok, ref)
+    assert st == 0
+    # same sizes, other layout: the kernel reads inside the buffers and reports the mismatch
+    p_bad = A.Params(5000, 1024, 4, layout=LAYOUT_BITPLANE)
+    _, st = gpu_decompress(p_bad, ref)
+    assert st == A.DEV_BAD_HEADER
+    # a stream coded with stochastic rounding decodes under parameters that say nearest
+    ref_sr, _ = oracle.compress(x, 1024, 4, RANGE_ABSMAX, ROUND_STOCHASTIC, LAYOUT_INTERLEAVED, 3, 0)
+    _, st = gpu_decompress(p_ok, ref_sr)
+    assert st == 0
+    # the host parser recovers the parameters from the 32 header bytes
+    got = A.accept_parse_header(bytes(ref_sr[:32]))
+    assert (got.n_elems, got.chunk_elems, got.k, got.range, got.round, got.layout) == (5000, 1024, 4, 0, 1, 0)
+
+
+def test_output_canaries_untouched():
+    """Nothing is written past the compressed size or the N floats."""
+    A = _lib()
+    n, chunk, k = 4096 * 3 + 1001, 4096, 3
+    x = workloads.random_tensor(n, 8, "normal")
+    p = A.Params(n, chunk, k, layout=LAYOUT_BITPLANE)
+    size = A.accept_compressed_size(p)
+    d_stream = torch.full((size + 256,), 0x5A, dtype=torch.uint8, device="cuda")
+    d_ws = A.new_workspace(p)
+    A.accept_compress(p, torch.from_numpy(x).cuda(), d_stream, d_ws)
+    host = d_stream.cpu().numpy()
+    assert np.all(host[size:] == 0x5A)
+    assert np.array_equal(host[:size], oracle.compress(x, chunk, k, RANGE_ABSMAX, ROUND_NEAREST, LAYOUT_BITPLANE)[0])
+    d_out = torch.full((n + 64,), 7.0, dtype=torch.float32, device="cuda")
+    A.accept_decompress(p, d_stream, d_out, d_ws)
+    assert A.accept_last_device_status(d_ws) == 0
+    assert bool((d_out[n:] == 7.0).all())
+
+
+def test_host_buffer_entry_points():
+    A = _lib()
+    n, chunk, k = 1 << 18, 4096, 8
+    x = workloads.generate("cfg1_act", 0, n)
+    p = A.Params(n, chunk, k)
+    h_x = torch.from_numpy(x).pin_memory()
+    h_stream = torch.empty(A.accept_compressed_size(p), dtype=torch.uint8).pin_memory()
+    h_xhat = torch.empty(n, dtype=torch.float32).pin_memory()
+    d_x = torch.empty(n, dtype=torch.float32, device="cuda")
+    d_xhat = torch.empty(n, dtype=torch.float32, device="cuda")
+    d_stream, d_ws = A.new_stream_buffer(p), A.new_workspace(p)
+    A.accept_compress_host(p, h_x, h_stream, d_x, d_stream, d_ws)
+    A.accept_decompress_host(p, h_stream, h_xhat, d_stream, d_xhat, d_ws)
+    assert A.accept_last_device_status(d_ws) == 0
+    ref, _ = oracle.compress(x, chunk, k)
+    assert np.array_equal(h_stream.numpy(), ref)
+    assert np.array_equal(h_xhat.numpy().view(np.uint32), oracle.decompress(ref, n).view(np.uint32))
+
+
+# ------------------------------------------------------------------ the five workloads
+
+
+def _modes_of(spec):
+    return [(m.k, m.range, m.round, m.layout) for m in spec.headline + spec.also]
+
+
+@pytest.mark.parametrize("name", ["cfg1_act", "cfg2_grad", "cfg5_64KB", "cfg5_1MB", "cfg5_16MB"])
+def test_workloads_full_parity_small(name):
+    spec = workloads.TENSORS[name]
+    x = workloads.generate(name)
+    for k, range_, round_, layout in _modes_of(spec):
+        check_roundtrip(x, spec.chunk, k, range_, round_, layout, seed=spec.seed)
+
+
+@pytest.mark.parametrize("name", ["cfg3_act", "cfg3_grad", "cfg4_hidden"])
+def test_workloads_full_parity_large(name):
+    """Full-size tensors in the launch configuration the benchmark times; every element compared."""
+    spec = workloads.TENSORS[name]
+    x = workloads.generate(name)
+    for m in spec.headline:
+        check_roundtrip(x, spec.chunk, m.k, m.range, m.round, m.layout, seed=spec.seed)
+
+
+@pytest.mark.parametrize("name", ["cfg5_256MB", "cfg5_1GB"])
+def test_workloads_sampled_parity_sweep(name):
+    """Full-size launch; the oracle recomputes sampled runs of chunks (chunks are independent and
+    the random-number counter is the element index, so a slice can be coded on its own)."""
+    A = _lib()
+    spec = workloads.TENSORS[name]
+    n, chunk = spec.n, spec.chunk
+    d_x = torch.empty(n, dtype=torch.float32, device="cuda")
+    step = 1 << 24
+    for s in range(0, n, step):
+        d_x[s:s + step].copy_(torch.from_numpy(workloads.generate(name, s, min(step, n - s))))
+    n_chunks = n // chunk
+    rng = np.random.default_rng(123)
+    starts = sorted({0, n_chunks - 8, *rng.integers(0, n_chunks - 8, 6).tolist()})
+    for m in spec.headline:
+        p = A.Params(n, chunk, m.k, m.range, m.round, m.layout, spec.seed, 0)
+        d_stream, d_ws = A.new_stream_buffer(p), A.new_workspace(p)
+        A.accept_compress(p, d_x, d_stream, d_ws)
+        d_xhat = torch.empty(n, dtype=torch.float32, device="cuda")
+        A.accept_decompress(p, d_stream, d_xhat, d_ws)
+        assert A.accept_last_device_status(d_ws) == 0
+        off = A.accept_payload_offset(p)
+        words_per_chunk = chunk * m.k // 32
+        for c0 in starts:
+            xs = workloads.generate(name, c0 * chunk, 8 * chunk)
+            ref, _ = oracle.compress(xs, chunk, m.k, m.range, m.round, m.layout, spec.seed, c0 * chunk)
+            _, meta_r, pay_r = oracle.split_stream(ref, xs.size, chunk)
+            meta_g = d_stream[32 + 8 * c0:32 + 8 * (c0 + 8)].cpu().numpy().view(np.float32).reshape(8, 2)
+            b0 = off + 4 * words_per_chunk * c0
+            pay_g = d_stream[b0:b0 + 4 * words_per_chunk * 8].cpu().numpy().view(np.uint32)
+            assert np.array_equal(meta_g.view(np.uint32), meta_r.view(np.uint32))
+            assert np.array_equal(pay_g, pay_r[:pay_g.size])
+            xhat_g = d_xhat[c0 * chunk:(c0 + 8) * chunk].cpu().numpy()
+            assert_float_parity(xhat_g, oracle.decompress(ref, xs.size), xs, chunk)
+        # properties that hold at any size: header, total size, every reconstructed value finite
+        hdr = d_stream[:32].cpu().numpy().view(np.uint32)
+        assert [int(v) for v in hdr[:6]] == [0x54504341, 1, n & 0xFFFFFFFF, n >> 32, chunk, m.k]
+        assert bool(torch.isfinite(d_xhat).all())
+        del d_stream, d_xhat

@@ -1,0 +1,129 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, validates arguments before touching CUDA, and sizes streams like the oracle."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def A():
+    from paper_2311_05827_b200 import build
+    build.build()
+    import paper_2311_05827_b200 as pkg
+    return pkg
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "accept.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(accept_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(A):
+    from paper_2311_05827_b200 import binding
+    names = declared_functions()
+    assert len(names) >= 12
+    lib = binding.lib()
+    for name in names:
+        assert hasattr(lib, name), f"{name} declared in accept.h but not exported"
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_params_struct_matches_header_layout(A):
+    from paper_2311_05827_b200.binding import CParams
+    assert ctypes.sizeof(CParams) == 48
+    assert CParams.seed.offset == 32 and CParams.rng_offset.offset == 40 and CParams.range.offset == 16
+
+
+@pytest.mark.parametrize("n,chunk,k", [(1, 32, 2), (100, 32, 3), (5000, 1024, 4), (4096, 4096, 8),
+                                       (1 << 20, 1 << 20, 2), (51380224, 4096, 4), (268435456, 4096, 8),
+                                       (2 ** 33 + 5, 4096, 2)])
+def test_size_queries_match_oracle(A, n, chunk, k):
+    layout = A.LAYOUT_BITPLANE if k == 3 else A.LAYOUT_INTERLEAVED
+    p = A.Params(n, chunk, k, layout=layout)
+    assert A.accept_check_params(p) == 0
+    assert A.accept_compressed_size(p) == oracle.stream_bytes(n, chunk, k)
+    assert A.accept_payload_offset(p) == oracle.payload_offset(n, chunk)
+    assert A.accept_workspace_size(p) == 16
+
+
+def test_invalid_params_are_rejected(A):
+    P = A.Params
+    assert A.accept_check_params(P(0, 32, 4)) == 9
+    assert A.accept_check_params(P(10, 0, 4)) == 3
+    assert A.accept_check_params(P(10, 48, 4)) == 3
+    assert A.accept_check_params(P(10, 32, 5)) == 2
+    assert A.accept_check_params(P(10, 32, 3)) == 2                       # k = 3 needs BITPLANE
+    assert A.accept_check_params(P(10, 32, 3, layout=A.LAYOUT_BITPLANE)) == 0
+    assert A.accept_check_params(P(10, 32, 4, range=2)) == 4
+    assert A.accept_check_params(P(10, 32, 4, round=-1)) == 4
+    assert A.accept_check_params(P(10, 32, 4, layout=7)) == 4
+    for bad in (P(0, 32, 4), P(10, 33, 4), P(10, 32, 1)):
+        assert A.accept_compressed_size(bad) == 0 and A.accept_workspace_size(bad) == 0
+
+
+def test_entry_points_validate_before_launching(A):
+    """Bad arguments return an error code without any CUDA call (this machine has no GPU)."""
+    from paper_2311_05827_b200 import binding
+    lib = binding.lib()
+    before = A.accept_launch_count()
+    p = A.Params(1000, 32, 4).c()
+    size = oracle.stream_bytes(1000, 32, 4)
+    good = 0x10000  # never dereferenced on the host
+    assert lib.accept_compress(ctypes.byref(p), None, good, size, good, 16, None) == 1
+    assert lib.accept_compress(ctypes.byref(p), good, None, size, good, 16, None) == 1
+    assert lib.accept_compress(ctypes.byref(p), good, good, size, None, 16, None) == 1
+    assert lib.accept_compress(ctypes.byref(p), good, good, size - 1, good, 16, None) == 5
+    assert lib.accept_compress(ctypes.byref(p), good, good, size, good, 15, None) == 5
+    assert lib.accept_compress(ctypes.byref(p), good + 4, good, size, good, 16, None) == 10
+    assert lib.accept_decompress(ctypes.byref(p), good, size, None, good, 16, None) == 1
+    assert lib.accept_decompress(ctypes.byref(p), good, size - 1, good, good, 16, None) == 5
+    bad = A.Params(1000, 32, 7).c()
+    assert lib.accept_compress(ctypes.byref(bad), good, good, size, good, 16, None) == 2
+    assert lib.accept_compress_host(ctypes.byref(p), None, good, size, good, good, good, 16, None) == 1
+    assert lib.accept_decompress_host(ctypes.byref(p), good, size, None, good, good, good, 16, None) == 1
+    assert A.accept_launch_count() == before
+
+
+def test_parse_header_reads_an_oracle_stream(A):
+    x = workloads.random_tensor(777, 4, "normal")
+    stream, _ = oracle.compress(x, 96, 3, oracle.RANGE_MINMAX, oracle.ROUND_STOCHASTIC, oracle.LAYOUT_BITPLANE, 5, 6)
+    p = A.accept_parse_header(bytes(stream[:32]))
+    assert (p.n_elems, p.chunk_elems, p.k, p.range, p.round, p.layout) == (777, 96, 3, 1, 1, 1)
+    broken = stream[:32].copy()
+    broken[1] ^= 0x40
+    with pytest.raises(A.AcceptError):
+        A.accept_parse_header(bytes(broken))
+    broken = stream[:32].copy()
+    broken[20] = 6  # k = 6
+    with pytest.raises(A.AcceptError):
+        A.accept_parse_header(bytes(broken))
+
+
+def test_bitwidth_schedule_matches_the_paper(A):
+    assert [A.accept_bitwidth_schedule(False, c) for c in range(5)] == [2, 3, 4, 4, 4]
+    assert [A.accept_bitwidth_schedule(True, c) for c in range(4)] == [8, 4, 4, 4]
+    for back in (False, True):
+        for c in range(-1, 6):
+            assert A.accept_bitwidth_schedule(back, c) == oracle.bitwidth_schedule(back, c)
+
+
+def test_workload_generator_is_sliceable_and_seeded():
+    a = workloads.generate("cfg3_act", (1 << 20) - 100, 300)
+    b = workloads.generate("cfg3_act", (1 << 20) - 100, 300)
+    whole = workloads.generate("cfg3_act", 0, (1 << 20) + 500)
+    assert np.array_equal(a, b) and np.array_equal(a, whole[(1 << 20) - 100:(1 << 20) + 200])
+    x = workloads.generate("cfg1_act")
+    assert x.size == 32 * 64 * 32 * 32 and 0.45 < (x == 0).mean() < 0.55 and x.min() >= 0
+    g = workloads.generate("cfg2_grad")
+    assert abs(np.abs(g).max() - 0.05) < 1e-6 and 0.0005 < (np.abs(g) == np.float32(0.05)).mean() < 0.002
+    h = workloads.generate("cfg4_hidden", 0, 4096 * 4)
+    assert np.allclose(h[:4096].std() / h[4096:8192].std(), 1, atol=0.2)
