@@ -20,7 +20,6 @@ import os
 import subprocess
 import sys
 import tempfile
-import threading
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -75,7 +74,7 @@ class ClockSampler:
             self.out = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+                 "-lms", "20"], stdout=self.out, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -159,6 +158,27 @@ class Codec:
         td = sum(e[1].elapsed_time(e[2]) for e in ev) / steps
         return total / steps, tc, td
 
+    def run_isolated(self, steps: int, warmup: int = 3):
+        """Each kernel in a loop of its own (rotating buffers): -> (ms per compress, ms per decompress).
+        Inside a step the compress kernel also pays for the write-back of the dirty output lines the
+        previous decompress left in L2; these loops charge every kernel with its own traffic only."""
+        torch, A = self.torch, self.A
+        out = []
+        for fn in (lambda j: A.accept_compress(self.p, self.x[j], self.stream[j], self.ws),
+                   lambda j: A.accept_decompress(self.p, self.stream[j], self.xhat[j], self.ws)):
+            for i in range(warmup):
+                fn(i % self.copies)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(steps):
+                fn((warmup + i) % self.copies)
+            e1.record()
+            torch.cuda.synchronize()
+            out.append(e0.elapsed_time(e1) / steps)
+            self.calls += steps + warmup
+        return out[0], out[1]
+
     def status(self) -> int:
         return self.A.accept_last_device_status(self.ws)
 
@@ -232,7 +252,7 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     spec = workloads.TENSORS[args.workload]
-    mode = spec.headline[0]
+    mode = (spec.headline + spec.also)[args.mode_index]
     x_host = workloads.generate(args.workload)
     n = spec.n
     peak, peak_src = measured_peak()
@@ -254,17 +274,21 @@ def run_gpu(args):
     ms_step, ms_c, ms_d = codec.run(args.steps, 0)
     launches_timed = A.accept_launch_count() - launches_before
     barrier()
+    iso_c, iso_d = codec.run_isolated(args.steps)
     clocks = sampler.stop()
     assert codec.status() == 0
 
-    t = torch.tensor([ms_step, ms_c, ms_d], dtype=torch.float64, device="cuda")
+    t = torch.tensor([ms_step, ms_c, ms_d, iso_c, iso_d], dtype=torch.float64, device="cuda")
     if dist is not None:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step, ms_c, ms_d = [float(v) for v in t.tolist()]
+    ms_step, ms_c, ms_d, iso_c, iso_d = [float(v) for v in t.tolist()]
 
     # end to end through host buffers
     e2e_steps = max(1, min(args.steps, 5))
-    ms_e2e, h2d, d2h = e2e_run(A, torch, x_host, spec.chunk, mode, spec.seed, e2e_steps, 1)
+    if args.kernels_only:
+        ms_e2e, h2d, d2h = float("nan"), 0, 0
+    else:
+        ms_e2e, h2d, d2h = e2e_run(A, torch, x_host, spec.chunk, mode, spec.seed, e2e_steps, 1)
     te = torch.tensor([ms_e2e], dtype=torch.float64, device="cuda")
     if dist is not None:
         dist.all_reduce(te, op=dist.ReduceOp.MAX)
@@ -281,10 +305,12 @@ def run_gpu(args):
         "config": {"workload": args.workload, "shape": list(spec.shape), "n_elems": n, "chunk": spec.chunk,
                    "mode": mode_name(mode), "l2": "inputs larger than L2 and %d rotating buffer sets" % codec.copies,
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
-        "compress": {"ms": ms_c, "gbs_fp32_in": gbs(4 * n, ms_c), "hbm_gbs": gbs(alg, ms_c), "frac_of_measured_copy": gbs(alg, ms_c) / peak,
-                     "frac_of_8TBs": gbs(alg, ms_c) / 8000.0},
-        "decompress": {"ms": ms_d, "gbs_fp32_out": gbs(4 * n, ms_d), "hbm_gbs": gbs(alg, ms_d), "frac_of_measured_copy": gbs(alg, ms_d) / peak,
-                       "frac_of_8TBs": gbs(alg, ms_d) / 8000.0},
+        "step_hbm": {"algorithmic_bytes": 2 * alg, "gbs": gbs(2 * alg, ms_step), "frac_of_measured_copy": gbs(2 * alg, ms_step) / peak,
+                     "frac_of_8TBs": gbs(2 * alg, ms_step) / 8000.0},
+        "compress": {"ms_in_step": ms_c, "ms_alone": iso_c, "gbs_fp32_in": gbs(4 * n, iso_c), "hbm_gbs": gbs(alg, iso_c),
+                     "frac_of_measured_copy": gbs(alg, iso_c) / peak, "frac_of_8TBs": gbs(alg, iso_c) / 8000.0},
+        "decompress": {"ms_in_step": ms_d, "ms_alone": iso_d, "gbs_fp32_out": gbs(4 * n, iso_d), "hbm_gbs": gbs(alg, iso_d),
+                       "frac_of_measured_copy": gbs(alg, iso_d) / peak, "frac_of_8TBs": gbs(alg, iso_d) / 8000.0},
         "roofline": {"bound": "hbm", "kernel": dominant, "achieved": gbs(alg, ms_dom), "peak": peak, "peak_source": peak_src,
                      "unit": "GB/s", "frac": gbs(alg, ms_dom) / peak, "traffic": TRAFFIC.get((args.workload, dominant))},
         "e2e": {"value": world * gbs(4 * n, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d,
@@ -296,7 +322,7 @@ def run_gpu(args):
     if args.sweep and rank == 0:
         out["workloads"] = sweep(A, torch, peak, args)
 
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not (args.no_cpu_baseline or args.kernels_only):
         tc, td, reps = time_oracle(x_host, spec.chunk, mode, spec.seed, budget_s=args.cpu_budget)
         out["cpu_baseline"] = {"value": 4 * n / (tc + td) / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
                                "sample": "whole %s tensor (%d elements), %d round trips; compress %.3f s, decompress %.3f s each"
@@ -325,7 +351,7 @@ def sweep(A, torch, peak, args):
         for mode in spec.headline:
             codec = Codec(A, torch, x_host, spec.chunk, mode, spec.seed)
             steps = 20 if spec.n * 4 >= (64 << 20) else 200
-            _, ms_c, ms_d = codec.run(steps, 3)
+            ms_c, ms_d = codec.run_isolated(steps)
             assert codec.status() == 0
             alg = algorithmic_bytes(spec.n, spec.chunk, mode.k)
             rows.append({"workload": name, "mode": mode_name(mode), "mbytes": spec.n * 4 / 2 ** 20, "copies": codec.copies,
@@ -385,6 +411,9 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="also time every workload's headline modes")
     ap.add_argument("--sweep-max-bytes", type=int, default=1 << 30)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernels-only", action="store_true",
+                    help="profiling runs: skip the host-buffer and CPU-oracle legs (the line is then not a bench result)")
+    ap.add_argument("--mode-index", type=int, default=0, help="which of the workload's headline modes to run")
     ap.add_argument("--cpu-budget", type=float, default=10.0)
     ap.add_argument("--reference-sample", type=int, default=1 << 24)
     args = ap.parse_args()

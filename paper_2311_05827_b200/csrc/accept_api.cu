@@ -21,9 +21,11 @@ uint64_t n_chunks_of(const accept_params* p) { return (p->n_elems + p->chunk_ele
 // Geometry of the register-resident compress path for chunk size C: rounds R and threads per chunk.
 struct FastGeometry { int rounds; uint32_t tpc; };
 
+// Four octets per thread measured fastest (fewest per-thread fixed costs per element); fewer
+// rounds serve chunk sizes that four rounds of whole warps do not divide.
 FastGeometry fast_geometry(uint32_t C) {
-  if (C % 512 == 0 && C / 16 <= 1024) return {2, C / 16};
   if (C % 1024 == 0 && C / 32 <= 1024) return {4, C / 32};
+  if (C % 512 == 0 && C / 16 <= 1024) return {2, C / 16};
   if (C % 256 == 0 && C / 8 <= 1024) return {1, C / 8};
   return {0, 0};
 }
@@ -53,56 +55,67 @@ CodecArgs make_args(const accept_params* p, void* d_stream, void* d_ws) {
 using KernelFn = void (*)(const CodecArgs);
 
 template <int K, int LAYOUT, int RANGE, int ROUND>
-KernelFn compress_for_rounds(int rounds) {
+KernelFn compress_for_rounds(int rounds, bool small_block) {
+  if (small_block) {
+    switch (rounds) {
+      case 1: return accept::compress_kernel<K, LAYOUT, RANGE, ROUND, 1, 256>;
+      case 4: return accept::compress_kernel<K, LAYOUT, RANGE, ROUND, 4, 256>;
+      default: return accept::compress_kernel<K, LAYOUT, RANGE, ROUND, 2, 256>;
+    }
+  }
   switch (rounds) {
-    case 1: return accept::compress_kernel<K, LAYOUT, RANGE, ROUND, 1>;
-    case 4: return accept::compress_kernel<K, LAYOUT, RANGE, ROUND, 4>;
-    default: return accept::compress_kernel<K, LAYOUT, RANGE, ROUND, 2>;
+    case 1: return accept::compress_kernel<K, LAYOUT, RANGE, ROUND, 1, 1024>;
+    case 4: return accept::compress_kernel<K, LAYOUT, RANGE, ROUND, 4, 1024>;
+    default: return accept::compress_kernel<K, LAYOUT, RANGE, ROUND, 2, 1024>;
   }
 }
 
 template <int K, int LAYOUT>
-KernelFn compress_for_modes(int range, int round, int rounds) {
+KernelFn compress_for_modes(int range, int round, int rounds, bool sb) {
   if (range == accept::kAbsMax) {
-    return round == accept::kNearest ? compress_for_rounds<K, LAYOUT, accept::kAbsMax, accept::kNearest>(rounds)
-                                     : compress_for_rounds<K, LAYOUT, accept::kAbsMax, accept::kStochastic>(rounds);
+    return round == accept::kNearest ? compress_for_rounds<K, LAYOUT, accept::kAbsMax, accept::kNearest>(rounds, sb)
+                                     : compress_for_rounds<K, LAYOUT, accept::kAbsMax, accept::kStochastic>(rounds, sb);
   }
-  return round == accept::kNearest ? compress_for_rounds<K, LAYOUT, accept::kMinMax, accept::kNearest>(rounds)
-                                   : compress_for_rounds<K, LAYOUT, accept::kMinMax, accept::kStochastic>(rounds);
+  return round == accept::kNearest ? compress_for_rounds<K, LAYOUT, accept::kMinMax, accept::kNearest>(rounds, sb)
+                                   : compress_for_rounds<K, LAYOUT, accept::kMinMax, accept::kStochastic>(rounds, sb);
 }
 
-KernelFn select_compress(const accept_params* p, int rounds) {
+KernelFn select_compress(const accept_params* p, int rounds, bool sb) {
   const bool bp = p->layout == ACCEPT_LAYOUT_BITPLANE;
   switch (p->k) {
-    case 2: return bp ? compress_for_modes<2, accept::kBitplane>(p->range, p->round, rounds)
-                      : compress_for_modes<2, accept::kInterleaved>(p->range, p->round, rounds);
-    case 3: return compress_for_modes<3, accept::kBitplane>(p->range, p->round, rounds);
-    case 4: return bp ? compress_for_modes<4, accept::kBitplane>(p->range, p->round, rounds)
-                      : compress_for_modes<4, accept::kInterleaved>(p->range, p->round, rounds);
-    default: return bp ? compress_for_modes<8, accept::kBitplane>(p->range, p->round, rounds)
-                       : compress_for_modes<8, accept::kInterleaved>(p->range, p->round, rounds);
+    case 2: return bp ? compress_for_modes<2, accept::kBitplane>(p->range, p->round, rounds, sb)
+                      : compress_for_modes<2, accept::kInterleaved>(p->range, p->round, rounds, sb);
+    case 3: return compress_for_modes<3, accept::kBitplane>(p->range, p->round, rounds, sb);
+    case 4: return bp ? compress_for_modes<4, accept::kBitplane>(p->range, p->round, rounds, sb)
+                      : compress_for_modes<4, accept::kInterleaved>(p->range, p->round, rounds, sb);
+    default: return bp ? compress_for_modes<8, accept::kBitplane>(p->range, p->round, rounds, sb)
+                       : compress_for_modes<8, accept::kInterleaved>(p->range, p->round, rounds, sb);
   }
+}
+
+template <int K, int LAYOUT, int RANGE>
+KernelFn decompress_for_rounds(bool aligned, int rounds) {
+  if (!aligned) return accept::decompress_unaligned_kernel<K, LAYOUT, RANGE>;
+  (void)rounds;
+  return accept::decompress_kernel<K, LAYOUT, RANGE, 2>;
 }
 
 template <int K, int LAYOUT>
-KernelFn decompress_for_range(int range, bool aligned) {
-  if (range == accept::kAbsMax)
-    return aligned ? accept::decompress_kernel<K, LAYOUT, accept::kAbsMax, 2>
-                   : accept::decompress_unaligned_kernel<K, LAYOUT, accept::kAbsMax>;
-  return aligned ? accept::decompress_kernel<K, LAYOUT, accept::kMinMax, 2>
-                 : accept::decompress_unaligned_kernel<K, LAYOUT, accept::kMinMax>;
+KernelFn decompress_for_range(int range, bool aligned, int rounds) {
+  if (range == accept::kAbsMax) return decompress_for_rounds<K, LAYOUT, accept::kAbsMax>(aligned, rounds);
+  return decompress_for_rounds<K, LAYOUT, accept::kMinMax>(aligned, rounds);
 }
 
-KernelFn select_decompress(const accept_params* p, bool aligned) {
+KernelFn select_decompress(const accept_params* p, bool aligned, int rounds) {
   const bool bp = p->layout == ACCEPT_LAYOUT_BITPLANE;
   switch (p->k) {
-    case 2: return bp ? decompress_for_range<2, accept::kBitplane>(p->range, aligned)
-                      : decompress_for_range<2, accept::kInterleaved>(p->range, aligned);
-    case 3: return decompress_for_range<3, accept::kBitplane>(p->range, aligned);
-    case 4: return bp ? decompress_for_range<4, accept::kBitplane>(p->range, aligned)
-                      : decompress_for_range<4, accept::kInterleaved>(p->range, aligned);
-    default: return bp ? decompress_for_range<8, accept::kBitplane>(p->range, aligned)
-                       : decompress_for_range<8, accept::kInterleaved>(p->range, aligned);
+    case 2: return bp ? decompress_for_range<2, accept::kBitplane>(p->range, aligned, rounds)
+                      : decompress_for_range<2, accept::kInterleaved>(p->range, aligned, rounds);
+    case 3: return decompress_for_range<3, accept::kBitplane>(p->range, aligned, rounds);
+    case 4: return bp ? decompress_for_range<4, accept::kBitplane>(p->range, aligned, rounds)
+                      : decompress_for_range<4, accept::kInterleaved>(p->range, aligned, rounds);
+    default: return bp ? decompress_for_range<8, accept::kBitplane>(p->range, aligned, rounds)
+                       : decompress_for_range<8, accept::kInterleaved>(p->range, aligned, rounds);
   }
 }
 
@@ -168,14 +181,17 @@ accept_status accept_compress(const accept_params* p, const float* d_x, void* d_
     const bool share = g.tpc <= (uint32_t)accept::kFastBlock && accept::kFastBlock % g.tpc == 0;
     block = share ? accept::kFastBlock : g.tpc;
     a.chunks_per_block = share ? accept::kFastBlock / g.tpc : 1;
+    a.tpc_shift = 0;
+    while ((1u << a.tpc_shift) < g.tpc) ++a.tpc_shift;  // exact when share: tpc is then a power of two
     fast_blocks = (a.n_fast_chunks + a.chunks_per_block - 1) / a.chunks_per_block;
   } else {
     a.n_fast_chunks = 0;
     a.tpc = 32;
     a.chunks_per_block = 1;
   }
+  a.fast_blocks = (uint32_t)fast_blocks;
   const uint64_t grid = fast_blocks + (a.n_chunks - a.n_fast_chunks);
-  KernelFn fn = select_compress(p, fast ? g.rounds : 2);
+  KernelFn fn = select_compress(p, fast ? g.rounds : 2, block <= 256);
   fn<<<(unsigned)grid, block, 0, static_cast<cudaStream_t>(cuda_stream)>>>(a);
   g_launches.fetch_add(1, std::memory_order_relaxed);
   return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
@@ -188,8 +204,9 @@ accept_status accept_decompress(const accept_params* p, const void* d_stream, si
   CodecArgs a = make_args(p, const_cast<void*>(d_stream), d_ws);
   a.xhat = d_xhat;
   const bool aligned = is_aligned(d_xhat, 32);
-  KernelFn fn = select_decompress(p, aligned);
-  const uint64_t per_block = aligned ? 4096 : 256;  // elements
+  const int rounds = 2;  // octets per thread
+  KernelFn fn = select_decompress(p, aligned, rounds);
+  const uint64_t per_block = aligned ? 2048ull * rounds : 256;  // elements per block
   const uint64_t grid = (p->n_elems + per_block - 1) / per_block;
   fn<<<(unsigned)grid, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(a);
   g_launches.fetch_add(1, std::memory_order_relaxed);

@@ -20,10 +20,26 @@ struct CodecArgs {
   uint32_t chunk;         // C
   int chunk_shift;        // log2(C) if C is a power of two, else -1
   uint32_t tpc;           // fast path: threads that share one chunk (C / (8*R))
+  int tpc_shift;          // log2(tpc) when a block holds several chunks (tpc divides 256), else unused
   uint32_t chunks_per_block;
+  uint32_t fast_blocks;   // blocks of the register-resident path; later blocks take the any-shape coder
   uint32_t header_word6;  // range | round<<8 | layout<<16
   uint32_t k;
 };
+
+// Word i of the 32-byte stream header.
+__device__ __forceinline__ uint32_t header_word(const CodecArgs& a, int i) {
+  switch (i) {
+    case 0: return 0x54504341u;
+    case 1: return 1u;
+    case 2: return (uint32_t)a.n;
+    case 3: return (uint32_t)(a.n >> 32);
+    case 4: return a.chunk;
+    case 5: return a.k;
+    case 6: return a.header_word6;
+    default: return 0u;
+  }
+}
 
 constexpr int kFastBlock = 256;     // threads per block when a chunk needs at most 256 threads
 constexpr int kGenericBlock = 256;  // threads per block of the any-shape path
@@ -134,26 +150,26 @@ __device__ void compress_chunk_generic(const CodecArgs& a, uint64_t m, float* s_
 // consecutive octets; the chunk is read from HBM once and stays in registers between the range
 // reduction and the quantizer.  Blocks past the fast chunks code the remaining chunk(s) with the
 // any-shape coder.
-template <int K, int LAYOUT, int RANGE, int ROUND, int R>
-__global__ void __launch_bounds__(1024) compress_kernel(const CodecArgs a) {
+// BLOCK_MAX is the largest block the instantiation is launched with (256 or 1024); the smaller
+// bound lets the compiler keep six (R <= 2) or four (R = 4) blocks resident per SM.
+template <int K, int LAYOUT, int RANGE, int ROUND, int R, int BLOCK_MAX>
+__global__ void __launch_bounds__(BLOCK_MAX, BLOCK_MAX == 256 ? (R <= 2 ? 6 : 4) : 1) compress_kernel(const CodecArgs a) {
   __shared__ float s_hi[32], s_lo[32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   if (blockIdx.x == 0 && tid < 8) {
     // stream header and the pad between the side words and the payload
-    const uint32_t h[8] = {0x54504341u, 1u, (uint32_t)a.n, (uint32_t)(a.n >> 32), a.chunk, a.k, a.header_word6, 0u};
-    a.header[tid] = h[tid];
+    a.header[tid] = header_word(a, tid);
     if ((a.n_chunks & 1) && tid < 2) reinterpret_cast<uint32_t*>(a.meta + a.n_chunks)[tid] = 0u;
   }
 
-  const uint64_t fast_blocks = (a.n_fast_chunks + a.chunks_per_block - 1) / a.chunks_per_block;
-  if (blockIdx.x >= fast_blocks) {
-    compress_chunk_generic<K, LAYOUT, RANGE, ROUND>(a, a.n_fast_chunks + (blockIdx.x - fast_blocks), s_hi, s_lo);
+  if (blockIdx.x >= a.fast_blocks) {
+    compress_chunk_generic<K, LAYOUT, RANGE, ROUND>(a, a.n_fast_chunks + (blockIdx.x - a.fast_blocks), s_hi, s_lo);
     return;
   }
 
   const uint32_t tpc = a.tpc;
-  const uint32_t grp = tid / tpc, gt = tid - grp * tpc;
+  const uint32_t grp = (a.chunks_per_block > 1) ? (tid >> a.tpc_shift) : 0u, gt = tid - grp * tpc;
   uint64_t m = (uint64_t)blockIdx.x * a.chunks_per_block + grp;
   const bool active = m < a.n_fast_chunks;  // a whole group is active or not; warps never straddle groups
   if (!active) m = a.n_fast_chunks - 1;     // idle groups redo the last chunk's loads, store nothing
@@ -174,9 +190,12 @@ __global__ void __launch_bounds__(1024) compress_kernel(const CodecArgs a) {
   if (tpc > 32) {
     if (lane == 0) { s_hi[warp] = rg.hi; s_lo[warp] = rg.lo; }
     __syncthreads();
+    // lane w of every warp picks up the partial of the group's warp w; a second butterfly
+    // leaves the chunk's range in every lane
     const int w0 = (grp * tpc) >> 5, wn = tpc >> 5;
     rg.init();
-    for (int w = 0; w < wn; ++w) rg.merge(s_hi[w0 + w], s_lo[w0 + w]);
+    if (lane < wn) { rg.hi = s_hi[w0 + lane]; rg.lo = s_lo[w0 + lane]; }
+    rg.warp_reduce();
   }
 
   Scale sc = make_scale<K, RANGE>(rg.hi, rg.lo);
@@ -208,85 +227,129 @@ __global__ void __launch_bounds__(1024) compress_kernel(const CodecArgs a) {
 
 // ----------------------------------------------------------------------------- decompress
 
-// Each thread rebuilds R octets; consecutive threads take consecutive octets, so every store
-// instruction of a warp writes 1 KB of contiguous output.
+// What one thread fetches for one octet: its slice of the payload and the chunk's side words.
+struct RawOctet {
+  uint32_t w0, w1;
+  float2 so;
+};
+
+template <int K, int LAYOUT>
+__device__ __forceinline__ RawOctet load_raw(const CodecArgs& a, uint64_t oct, uint64_t n_oct, uint64_t n_groups,
+                                             int lane) {
+  RawOctet raw;
+  raw.w0 = 0; raw.w1 = 0; raw.so = make_float2(0.0f, 0.0f);
+  if (LAYOUT == kInterleaved) {
+    if (oct < n_oct) {
+      if (K == 8) {
+        const uint2 w = __ldg(reinterpret_cast<const uint2*>(a.payload) + oct);
+        raw.w0 = w.x; raw.w1 = w.y;
+      } else if (K == 4) {
+        raw.w0 = __ldg(a.payload + oct);
+      } else {
+        raw.w0 = __ldg(reinterpret_cast<const uint16_t*>(a.payload) + oct);
+      }
+    }
+  } else {
+    // lane q of a quad fetches the word of binary digit q (and q+4) of the quad's group
+    const int q = lane & 3;
+    const uint64_t group = oct >> 2;
+    if (group < n_groups) {
+      if (K <= 4) {
+        if (q < K) raw.w0 = __ldg(a.payload + group * K + q);
+      } else {
+        raw.w0 = __ldg(a.payload + group * 8 + q);
+        raw.w1 = __ldg(a.payload + group * 8 + 4 + q);
+      }
+    }
+  }
+  if (oct < n_oct) {
+    const uint64_t e = oct * 8;
+    const uint64_t m = (a.chunk_shift >= 0) ? (e >> a.chunk_shift) : (e / a.chunk);
+    raw.so = __ldg(a.meta + m);
+  }
+  return raw;
+}
+
+// Payload slice -> the codes of the octet, one per byte (xlo: elements 0..3, xhi: 4..7).
+// BITPLANE shuffles inside a quad: all 32 lanes call.
+template <int K, int LAYOUT>
+__device__ __forceinline__ void unpack_octet(const RawOctet& raw, int lane, uint32_t& xlo, uint32_t& xhi) {
+  if (LAYOUT == kInterleaved) {
+    if (K == 8) {
+      xlo = raw.w0; xhi = raw.w1;
+    } else if (K == 4) {
+      uint32_t y = __byte_perm(raw.w0, 0, 0x4140);  // bytes: w.b0, 0, w.b1, 0
+      xlo = (y | (y << 4)) & 0x0F0F0F0Fu;           // nibbles -> bytes
+      y = __byte_perm(raw.w0, 0, 0x4342);           // bytes: w.b2, 0, w.b3, 0
+      xhi = (y | (y << 4)) & 0x0F0F0F0Fu;
+    } else {
+      const uint32_t w = raw.w0;                    // eight 2-bit fields
+      uint32_t y = (w | (w << 12)) & 0x000F000Fu;
+      xlo = (y | (y << 6)) & 0x03030303u;
+      y = ((w >> 8) | ((w >> 8) << 12)) & 0x000F000Fu;
+      xhi = (y | (y << 6)) & 0x03030303u;
+    }
+  } else {
+    // a quad transpose hands every lane the plane bytes of its own octet
+    if (K <= 4) {
+      const uint32_t nib = planes_nibbles(quad_transpose(raw.w0, lane));
+      xlo = nib & 0x0F0F0F0Fu;
+      xhi = (nib >> 4) & 0x0F0F0F0Fu;
+    } else {
+      const uint32_t lo = planes_nibbles(quad_transpose(raw.w0, lane));
+      const uint32_t hi = planes_nibbles(quad_transpose(raw.w1, lane));
+      xlo = (lo & 0x0F0F0F0Fu) | ((hi & 0x0F0F0F0Fu) << 4);
+      xhi = ((lo >> 4) & 0x0F0F0F0Fu) | (hi & 0xF0F0F0F0u);
+    }
+  }
+}
+
+// Decodes and stores the R octets of one tile from the slices fetched earlier.
 template <int K, int LAYOUT, int RANGE, int R>
-__global__ void __launch_bounds__(256) decompress_kernel(const CodecArgs a) {
+__device__ __forceinline__ void decode_tile(const CodecArgs& a, const RawOctet (&raw)[R], uint64_t first_oct,
+                                            uint64_t n_oct, int lane) {
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const uint64_t oct = first_oct + r * 256;
+    uint32_t xlo, xhi;
+    unpack_octet<K, LAYOUT>(raw[r], lane, xlo, xhi);
+    if (oct < n_oct) {
+      const uint64_t e = oct * 8;
+      float out[8];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        out[i] = dequantize_code<K, RANGE>((xlo >> (8 * i)) & 0xFFu, raw[r].so.x, raw[r].so.y);
+        out[4 + i] = dequantize_code<K, RANGE>((xhi >> (8 * i)) & 0xFFu, raw[r].so.x, raw[r].so.y);
+      }
+      if (e + 8 <= a.n) {
+        st_octet(a.xhat + e, out);
+      } else {
+        for (int i = 0; i < 8; ++i)
+          if (e + i < a.n) a.xhat[e + i] = out[i];
+      }
+    }
+  }
+}
+
+// One tile of R*256 octets per block: every thread requests its R payload slices first, then
+// decodes and stores them; consecutive threads take consecutive octets, so each store instruction
+// of a warp writes 1 KB of contiguous output.  (Grid-stride variants of this kernel that prefetch
+// the next tile measured slower than one short-lived block per tile.)
+template <int K, int LAYOUT, int RANGE, int R>
+__global__ void __launch_bounds__(256, R <= 2 ? 8 : 6) decompress_kernel(const CodecArgs a) {
   const int tid = threadIdx.x, lane = tid & 31;
-  if (blockIdx.x == 0 && tid == 0) {
-    const uint32_t h[8] = {0x54504341u, 1u, (uint32_t)a.n, (uint32_t)(a.n >> 32), a.chunk, a.k, a.header_word6, 0u};
-    bool ok = true;
-    for (int i = 0; i < 6; ++i) ok = ok && (a.header[i] == h[i]);
-    // the rounding mode does not change how a stream is read: compare range and layout only
-    ok = ok && ((a.header[6] & 0xFFFF00FFu) == (h[6] & 0xFFFF00FFu));
-    if (!ok) atomicOr(a.status, kDevBadHeader);
+  if (blockIdx.x == 0 && tid < 8) {
+    // the rounding mode (bits 8..15 of word 6) does not change how a stream is read
+    const uint32_t mask = (tid == 6) ? 0xFFFF00FFu : 0xFFFFFFFFu;
+    if ((a.header[tid] & mask) != (header_word(a, tid) & mask)) atomicOr(a.status, kDevBadHeader);
   }
   const uint64_t n_oct = (a.n + 7) / 8;       // octets, the last one maybe partial
   const uint64_t n_groups = (a.n + 31) / 32;  // pack groups present in the payload
+  const uint64_t first_oct = (uint64_t)blockIdx.x * (R * 256) + tid;
+  RawOctet raw[R];
 #pragma unroll
-  for (int r = 0; r < R; ++r) {
-    const uint64_t oct = ((uint64_t)blockIdx.x * R + r) * blockDim.x + tid;
-    const bool in = oct < n_oct;
-    const uint64_t e = oct * 8;
-    uint32_t xlo = 0, xhi = 0;  // codes 0..3 / 4..7, one per byte
-    if (LAYOUT == kInterleaved) {
-      if (in) {
-        if (K == 8) {
-          const uint2 w = __ldg(reinterpret_cast<const uint2*>(a.payload) + oct);
-          xlo = w.x; xhi = w.y;
-        } else if (K == 4) {
-          const uint32_t w = __ldg(a.payload + oct);
-          // nibbles -> bytes
-          uint32_t y = __byte_perm(w, 0, 0x4140);  // bytes: w.b0, 0, w.b1, 0
-          xlo = (y | (y << 4)) & 0x0F0F0F0Fu;
-          y = __byte_perm(w, 0, 0x4342);           // bytes: w.b2, 0, w.b3, 0
-          xhi = (y | (y << 4)) & 0x0F0F0F0Fu;
-        } else {
-          const uint32_t w = __ldg(reinterpret_cast<const uint16_t*>(a.payload) + oct);
-          // 2-bit fields -> bytes
-          uint32_t y = (w | (w << 12)) & 0x000F000Fu;  // fields 0,1 | 2,3 (low byte), 4,5 | 6,7 handled below
-          xlo = (y | (y << 6)) & 0x03030303u;
-          y = ((w >> 8) | ((w >> 8) << 12)) & 0x000F000Fu;
-          xhi = (y | (y << 6)) & 0x03030303u;
-        }
-      }
-    } else {
-      // lane q of a quad fetches the word of binary digit q of its group; a quad transpose then
-      // hands every lane the plane bytes of its own octet
-      const int q = lane & 3;
-      const uint64_t group = oct >> 2;
-      const bool gin = group < n_groups;
-      if (K <= 4) {
-        uint32_t w = 0;
-        if (gin && q < K) w = __ldg(a.payload + group * K + q);
-        const uint32_t nib = planes_nibbles(quad_transpose(w, lane));
-        xlo = nib & 0x0F0F0F0Fu;
-        xhi = (nib >> 4) & 0x0F0F0F0Fu;
-      } else {
-        uint32_t w0 = 0, w1 = 0;
-        if (gin) { w0 = __ldg(a.payload + group * 8 + q); w1 = __ldg(a.payload + group * 8 + 4 + q); }
-        const uint32_t lo = planes_nibbles(quad_transpose(w0, lane));
-        const uint32_t hi = planes_nibbles(quad_transpose(w1, lane));
-        xlo = (lo & 0x0F0F0F0Fu) | ((hi & 0x0F0F0F0Fu) << 4);
-        xhi = ((lo >> 4) & 0x0F0F0F0Fu) | (hi & 0xF0F0F0F0u);
-      }
-    }
-    if (!in) continue;
-    const uint64_t m = (a.chunk_shift >= 0) ? (e >> a.chunk_shift) : (e / a.chunk);
-    const float2 so = __ldg(a.meta + m);
-    float out[8];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      out[i] = dequantize_code<K, RANGE>((xlo >> (8 * i)) & 0xFFu, so.x, so.y);
-      out[4 + i] = dequantize_code<K, RANGE>((xhi >> (8 * i)) & 0xFFu, so.x, so.y);
-    }
-    if (e + 8 <= a.n) {
-      st_octet(a.xhat + e, out);
-    } else {
-      for (int i = 0; i < 8; ++i)
-        if (e + i < a.n) a.xhat[e + i] = out[i];
-    }
-  }
+  for (int r = 0; r < R; ++r) raw[r] = load_raw<K, LAYOUT>(a, first_oct + r * 256, n_oct, n_groups, lane);
+  decode_tile<K, LAYOUT, RANGE, R>(a, raw, first_oct, n_oct, lane);
 }
 
 // Scalar any-alignment decoder for output pointers that are not 32-byte aligned.
