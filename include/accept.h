@@ -66,7 +66,8 @@ typedef enum {
   ACCEPT_ERR_CUDA = 7,          /* a CUDA runtime call failed */
   ACCEPT_ERR_NONFINITE = 8,     /* reported through the device status word only */
   ACCEPT_ERR_BAD_SIZE = 9,      /* n_elems = 0 */
-  ACCEPT_ERR_MISALIGNED = 10    /* a device pointer is not 16-byte aligned */
+  ACCEPT_ERR_MISALIGNED = 10,   /* a device pointer is not 16-byte aligned */
+  ACCEPT_ERR_SCRATCH_LIMIT = 11 /* accept_compress_static: the call needs more scratch than the built-in array holds */
 } accept_status;
 
 /* Bits of the device status word (word 0 of the workspace); sticky until the caller clears it. */
@@ -140,6 +141,34 @@ accept_status accept_compress(const accept_params* p, const float* d_x, void* d_
  */
 accept_status accept_decompress(const accept_params* p, const void* d_stream, size_t stream_bytes,
                                 float* d_xhat, void* d_ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * accept_compress for callers that cannot allocate device memory at all.  (The paper has no counterpart:
+ * this is a packaging variant of the quantizer + encoder above, same kernel, same stream.)
+ *
+ * Who needs it: a pipeline stage on a device whose memory budget is sealed after start-up, or a plug-in
+ * living inside a host framework that owns every byte of device memory, has no way to obtain the
+ * workspace accept_compress asks for -- cudaMalloc (or the framework's allocator) is off limits to it.
+ * Here the workspace is a fixed array of ACCEPT_STATIC_SCRATCH_BYTES (256) bytes that is part of the
+ * library image: every GPU that loads the library holds it until the process exits, and the entry point
+ * calls no cudaMalloc, cudaFree or any other allocating routine.  The caller still passes the input and
+ * the output stream, sized as for accept_compress.
+ *
+ *   d_status_out  optional DEVICE pointer (4-byte aligned) that receives the ACCEPT_DEV_* status bits of
+ *                 THIS call (copied on cuda_stream after the kernel); NULL if not wanted.
+ *
+ * Limits and rules:
+ *   - a call whose workspace need (accept_workspace_size) exceeds ACCEPT_STATIC_SCRATCH_BYTES is rejected
+ *     with ACCEPT_ERR_SCRATCH_LIMIT and nothing is launched;
+ *   - the first call on each device looks up the array's device address (with that device current); make
+ *     that first call before any stream capture begins on that device;
+ *   - all calls on a device share the one array.  The status word in it is cleared at the start of every
+ *     call (so it does not accumulate across calls as a caller-owned workspace does), and two calls that
+ *     overlap on the GPU (different streams) race on it: issue them on one stream, or order them.
+ */
+#define ACCEPT_STATIC_SCRATCH_BYTES 256u
+accept_status accept_compress_static(const accept_params* p, const float* d_x, void* d_stream,
+                                     size_t stream_bytes, uint32_t* d_status_out, void* cuda_stream);
 
 /*
  * Host-buffer variants, for callers whose tensors live in host memory: copy h_x to the staging

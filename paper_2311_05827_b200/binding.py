@@ -25,12 +25,14 @@ STATUS_NAMES = {
     0: "ACCEPT_OK", 1: "ACCEPT_ERR_NULL", 2: "ACCEPT_ERR_BAD_K", 3: "ACCEPT_ERR_BAD_CHUNK",
     4: "ACCEPT_ERR_BAD_ENUM", 5: "ACCEPT_ERR_TOO_SMALL", 6: "ACCEPT_ERR_BAD_STREAM_HEADER",
     7: "ACCEPT_ERR_CUDA", 8: "ACCEPT_ERR_NONFINITE", 9: "ACCEPT_ERR_BAD_SIZE", 10: "ACCEPT_ERR_MISALIGNED",
+    11: "ACCEPT_ERR_SCRATCH_LIMIT",
 }
 
 EXPORTS = [
     "accept_check_params", "accept_compressed_size", "accept_payload_offset", "accept_workspace_size",
     "accept_compress", "accept_decompress", "accept_compress_host", "accept_decompress_host",
     "accept_last_device_status", "accept_parse_header", "accept_bitwidth_schedule", "accept_launch_count",
+    "accept_compress_static",
 ]
 
 
@@ -93,6 +95,8 @@ def lib() -> ctypes.CDLL:
     L.accept_parse_header.argtypes = [vp, P]
     L.accept_bitwidth_schedule.restype = ctypes.c_int
     L.accept_bitwidth_schedule.argtypes = [ctypes.c_int, ctypes.c_int]
+    L.accept_compress_static.restype = ctypes.c_int
+    L.accept_compress_static.argtypes = [P, vp, vp, sz, vp, vp]
     L.accept_launch_count.restype = u64
     L.accept_launch_count.argtypes = []
     _lib = L
@@ -150,6 +154,15 @@ def accept_compress(p: Params, d_x, d_stream, d_ws, stream=None) -> None:
     _check(lib().accept_compress(ctypes.byref(p.c()), d_x.data_ptr(), d_stream.data_ptr(),
                                  d_stream.numel() * d_stream.element_size(), d_ws.data_ptr(),
                                  d_ws.numel() * d_ws.element_size(), _stream_handle(stream)), "accept_compress")
+
+
+def accept_compress_static(p: Params, d_x, d_stream, d_status_out=None, stream=None) -> None:
+    """accept_compress with the library's built-in scratch: for callers that cannot allocate a workspace.
+    d_status_out: optional int32/uint32 CUDA tensor (>= 1 element) that receives this call's status bits."""
+    _check(lib().accept_compress_static(ctypes.byref(p.c()), d_x.data_ptr(), d_stream.data_ptr(),
+                                        d_stream.numel() * d_stream.element_size(),
+                                        None if d_status_out is None else d_status_out.data_ptr(),
+                                        _stream_handle(stream)), "accept_compress_static")
 
 
 def accept_decompress(p: Params, d_stream, d_xhat, d_ws, stream=None) -> None:

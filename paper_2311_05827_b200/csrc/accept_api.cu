@@ -5,6 +5,7 @@
 
 #include <atomic>
 #include <cstring>
+#include <mutex>
 
 #include "accept_kernels.cuh"
 
@@ -117,6 +118,30 @@ KernelFn select_decompress(const accept_params* p, bool aligned, int rounds) {
     default: return bp ? decompress_for_range<8, accept::kBitplane>(p->range, aligned, rounds)
                        : decompress_for_range<8, accept::kInterleaved>(p->range, aligned, rounds);
   }
+}
+
+// ---- built-in scratch for accept_compress_static ------------------------------------------------
+//
+// The workspace of callers that cannot allocate.  In host code the name g_static_scratch is only a
+// stand-in for the symbol, not a device address: the address a kernel can use comes from
+// cudaGetSymbolAddress, asked once per device with that device current.
+static __device__ __align__(256) unsigned char g_static_scratch[ACCEPT_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_address[kMaxDevices] = {};
+
+// Device address of the built-in scratch on the current device, or nullptr on a CUDA error.
+void* static_scratch_address() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_address[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) return nullptr;
+    g_scratch_address[dev] = ptr;
+  }
+  return g_scratch_address[dev];
 }
 
 accept_status check_buffers(const accept_params* p, const void* d_tensor, const void* d_stream,
@@ -276,5 +301,28 @@ int accept_bitwidth_schedule(int is_backward, int n_lr_changes) {
 }
 
 uint64_t accept_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+accept_status accept_compress_static(const accept_params* p, const float* d_x, void* d_stream, size_t stream_bytes,
+                                     uint32_t* d_status_out, void* cuda_stream) {
+  // everything that can be refused on the host is refused before CUDA is touched
+  if (!p || !d_x || !d_stream) return ACCEPT_ERR_NULL;
+  accept_status st = accept_check_params(p);
+  if (st != ACCEPT_OK) return st;
+  if (accept_workspace_size(p) > ACCEPT_STATIC_SCRATCH_BYTES) return ACCEPT_ERR_SCRATCH_LIMIT;
+  if (stream_bytes < accept_compressed_size(p)) return ACCEPT_ERR_TOO_SMALL;
+  if (!is_aligned(d_x, 16) || !is_aligned(d_stream, 16) || !is_aligned(d_status_out, 4)) return ACCEPT_ERR_MISALIGNED;
+
+  void* scratch = static_scratch_address();
+  if (!scratch) return ACCEPT_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  // the array keeps what the previous call left: the status word must start at zero
+  if (cudaMemsetAsync(scratch, 0, 16, s) != cudaSuccess) return ACCEPT_ERR_CUDA;
+  st = accept_compress(p, d_x, d_stream, stream_bytes, scratch, ACCEPT_STATIC_SCRATCH_BYTES, cuda_stream);
+  if (st != ACCEPT_OK) return st;
+  if (d_status_out &&
+      cudaMemcpyAsync(d_status_out, scratch, sizeof(uint32_t), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return ACCEPT_ERR_CUDA;
+  return ACCEPT_OK;
+}
 
 }  // extern "C"
