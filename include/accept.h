@@ -18,7 +18,8 @@
  *   codes   t = x*inv           (MINMAX: t = (x-lo)*inv), each fp32 operation rounded separately
  *           NEAREST:    q = rint(t)                      (ties to even)
  *           STOCHASTIC: q = floor(t) + [U < t-floor(t)]  (Eq. 7), U from the counter-based
- *                       generator described at accept_params.seed
+ *                       generator described at accept_params.seed; the fraction t-floor(t) and
+ *                       the comparison are exact (no rounding of the difference)
  *           ABSMAX: q clamped to [-2^(k-1), 2^(k-1)-1], stored code u = q + 2^(k-1)  ("+8" of the
  *           "Backward Encoder" for k = 4);  MINMAX: u = q clamped to [0, 2^k-1]
  *   pack    INTERLEAVED ("Backward Encoder"): code of element t of the chunk occupies bits
@@ -84,9 +85,10 @@ typedef enum { ACCEPT_LAYOUT_INTERLEAVED = 0, ACCEPT_LAYOUT_BITPLANE = 1 } accep
  *   chunk_elems  C, multiple of 32, >= 32: elements sharing one range.
  *   k            bit width: 2, 3 (BITPLANE only), 4 or 8.
  *   seed, rng_offset  STOCHASTIC only.  Element i draws
- *                  U_i = (h >> 9) * 2^-23,
- *                  h   = fmix32( lo32(ctr) ^ fmix32( hi32(ctr) ^ lo32(seed) ) ^ hi32(seed) ),
- *                  ctr = rng_offset + i (mod 2^64),
+ *                  U_i = (g >> 8) * 2^-24,
+ *                  g   = h if ctr is even, h * 0x9E3779B1 (mod 2^32) if ctr is odd,
+ *                  h   = fmix32( lo32(j) ^ fmix32( hi32(j) ^ lo32(seed) ^ 0x9E3779B9 ) ^ hi32(seed) ),
+ *                  j   = ctr >> 1,  ctr = rng_offset + i (mod 2^64),
  *                fmix32 = the 32-bit finaliser of MurmurHash3:
  *                  h ^= h>>16; h *= 0x85EBCA6B; h ^= h>>13; h *= 0xC2B2AE35; h ^= h>>16.
  *                The same (seed, rng_offset) reproduces the same stream; advance rng_offset by

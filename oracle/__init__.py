@@ -49,7 +49,7 @@ def _load():
     lib.oracle_stream_bytes.argtypes = [u64, u32, u32]
     lib.oracle_rng_hash.restype = u32
     lib.oracle_rng_hash.argtypes = [u64, u64]
-    lib.oracle_rng_uniform.restype = ctypes.c_float
+    lib.oracle_rng_uniform.restype = ctypes.c_double
     lib.oracle_rng_uniform.argtypes = [u64, u64]
     lib.oracle_quantize.restype = i32
     lib.oracle_quantize.argtypes = [vp, u64, u32, u32, i32, i32, u64, u64, vp, vp]

@@ -17,8 +17,9 @@
  *   - "dividing by the scaling factor" is computed as a product with inv = L/c (one division per
  *     chunk); pinned against true division in the tests;
  *   - nearest rounding is IEEE round-half-to-even;
- *   - the uniform generator of Eq. 7 is counter based (MurmurHash3's 32-bit finaliser, see
- *     oracle_rng_hash below);
+ *   - the uniform generator of Eq. 7 is counter based (MurmurHash3's 32-bit finaliser, one hash per
+ *     pair of counters, see oracle_rng_hash below); U has 24 bits; pr = t - floor(t) and the test
+ *     U < pr are exact;
  *   - bit order in a packed word is LSB first (element t of a group <-> bit t).  The paper's only
  *     worked example, (00110110)_2 = 54, fixes the value of a word, not which element is the MSB:
  *     PARITY UNPINNED for the bit order and for which elements share a word (the figure that
@@ -68,15 +69,19 @@ static uint32_t fmix32(uint32_t h) {
   return h;
 }
 
-/* 32 hashed bits for counter ctr under seed. */
+/* 32 random bits for counter ctr under seed.  Counters 2j and 2j+1 share the hash of their pair
+ * index j; the odd one multiplies it by an odd constant (a bijection of the 32-bit word). */
 uint32_t oracle_rng_hash(uint64_t seed, uint64_t ctr) {
-  uint32_t inner = fmix32((uint32_t)(ctr >> 32) ^ (uint32_t)seed);
-  return fmix32((uint32_t)ctr ^ inner ^ (uint32_t)(seed >> 32));
+  uint64_t pair = ctr >> 1;
+  /* the constant keeps seed 0, pair 0 off the fixed point fmix32(0) = 0 */
+  uint32_t inner = fmix32((uint32_t)(pair >> 32) ^ (uint32_t)seed ^ 0x9E3779B9u);
+  uint32_t h = fmix32((uint32_t)pair ^ inner ^ (uint32_t)(seed >> 32));
+  return (ctr & 1) ? h * 0x9E3779B1u : h;
 }
 
-/* U in [0,1) with 23 random bits; exact in fp32. */
-float oracle_rng_uniform(uint64_t seed, uint64_t ctr) {
-  return (float)(oracle_rng_hash(seed, ctr) >> 9) * (1.0f / 8388608.0f);
+/* U in [0,1) on a grid of 2^-24: the top 24 random bits. */
+double oracle_rng_uniform(uint64_t seed, uint64_t ctr) {
+  return (double)(oracle_rng_hash(seed, ctr) >> 8) / 16777216.0;
 }
 
 /* ---------------------------------------------------------------- quantizer ("Backward Quantizer", Eq. 7) */
@@ -142,10 +147,12 @@ static int quantize_chunk(const float* x, uint32_t valid, uint32_t k, int range,
       if (round_mode == ROUND_NEAREST) {
         q = (int)rintf(t); /* default rounding mode: to nearest, ties to even */
       } else {
-        /* Eq. 7: floor(t) with probability 1-pr, floor(t)+1 with probability pr = t - floor(t). */
-        float f = floorf(t);
-        float pr = t - f;
-        float U = oracle_rng_uniform(seed, rng_offset + i0 + i);
+        /* Eq. 7: floor(t) with probability 1-pr, floor(t)+1 with probability pr = t - floor(t).
+         * pr is a real number in the paper: it is held in double here, where the difference of an
+         * fp32 value and its floor cannot cross a multiple of 2^-24, so U < pr is decided exactly. */
+        double f = floor((double)t);
+        double pr = (double)t - f;
+        double U = oracle_rng_uniform(seed, rng_offset + i0 + i);
         q = (int)f + ((U < pr) ? 1 : 0);
       }
       if (q < qmin) q = qmin;

@@ -149,74 +149,129 @@ __device__ __forceinline__ uint32_t fmix32(uint32_t h) {
   return h;
 }
 
+// Two neighbouring counters share one hash: the element with the even counter takes the hashed
+// word as it is, the odd one takes it times kPairMul (an odd constant, so a bijection of the word).
+// This halves the per-element cost of the integer hash, which runs on the half-rate ALU pipe and
+// is what bounds stochastic rounding.
+constexpr uint32_t kPairMul = 0x9E3779B1u;
+
 struct Rng {
   uint32_t seed_lo, seed_hi;
-  // key for all counters that share their upper 32 bits
-  __device__ __forceinline__ uint32_t key(uint32_t ctr_hi) const {
-    return fmix32(ctr_hi ^ seed_lo) ^ seed_hi;
+  // key for all pairs that share the upper 32 bits of their pair index; the constant keeps
+  // seed 0 / pair 0 off the fixed point fmix32(0) = 0
+  __device__ __forceinline__ uint32_t key(uint32_t pair_hi) const {
+    return fmix32(pair_hi ^ seed_lo ^ 0x9E3779B9u) ^ seed_hi;
   }
-  // U in [0,1) with 23 bits: float in [1,2) built from the hash, minus one (exact)
-  __device__ __forceinline__ static float uniform(uint32_t ctr_lo, uint32_t key) {
-    const uint32_t h = fmix32(ctr_lo ^ key);
-    return __fsub_rn(__uint_as_float(0x3F800000u | (h >> 9)), 1.0f);
+  // hashed word of a pair
+  __device__ __forceinline__ static uint32_t pair_hash(uint32_t pair_lo, uint32_t key) { return fmix32(pair_lo ^ key); }
+  // 32 random bits of any counter (the octet path below shares the pair hashes instead)
+  __device__ __forceinline__ uint32_t word(uint64_t ctr) const {
+    const uint64_t pair = ctr >> 1;
+    const uint32_t h = pair_hash((uint32_t)pair, key((uint32_t)(pair >> 32)));
+    return (ctr & 1) ? h * kPairMul : h;
+  }
+};
+
+// What a thread works out once for all the octets it quantizes stochastically: the pair index and
+// key of its first counter, the counter's parity (the same for every octet, octets start 8 apart)
+// and whether the low word of the pair index stays clear of a wrap over the thread's whole span.
+struct RngThread {
+  uint64_t ctr_first;
+  uint32_t pair_lo, key;
+  bool odd, fast;
+  // span = distance, in counters, from the thread's first counter to one past its last
+  __device__ __forceinline__ void init(const Rng& rng, uint64_t ctr, uint32_t span) {
+    ctr_first = ctr;
+    const uint64_t pair = ctr >> 1;
+    pair_lo = (uint32_t)pair;
+    key = rng.key((uint32_t)(pair >> 32));
+    odd = ctr & 1;
+    fast = pair_lo <= 0xFFFFFFFFu - (span / 2 + 1);
   }
 };
 
 // ----------------------------------------------------------------------------- quantize
 
-// Returns the fp32 bit pattern of (kMagic + u), u the unsigned stored code; its low byte is u.
-template <int K, int RANGE, int ROUND>
-__device__ __forceinline__ uint32_t quantize_bits(float x, const Scale& sc, float U) {
+// NEAREST.  Returns the fp32 bit pattern of (kMagic + u), u the unsigned stored code: its byte 0 is u.
+template <int K, int RANGE>
+__device__ __forceinline__ uint32_t quantize_nearest_word(float x, const Scale& sc) {
   constexpr int ZP = (RANGE == kAbsMax) ? (1 << (K - 1)) : 0;
   constexpr float kMagicZ = kMagic + (float)ZP;  // exact; even, so ties still go to even codes
   const float d = (RANGE == kAbsMax) ? x : __fsub_rn(x, sc.base);
   const float t = __fmul_rn(d, sc.inv);
-  if (ROUND == kNearest) {
-    // |t| <= L(1+2^-22): the rounded code cannot leave [zp-L, zp+L], no clamp needed
-    return __float_as_uint(__fadd_rn(t, kMagicZ));
-  } else {
-    const float f = floorf(t);
-    const float pr = __fsub_rn(t, f);
-    uint32_t b = __float_as_uint(__fadd_rn(f, kMagicZ)) + ((U < pr) ? 1u : 0u);
-    // floor(t)+1 may exceed the top code when t rounded just above L; the low side cannot underflow
-    return min(b, kMagicBits + (uint32_t)((1 << K) - 1));
-  }
+  // |t| <= L(1+2^-22): the rounded code cannot leave [zp-L, zp+L], no clamp needed
+  return __float_as_uint(__fadd_rn(t, kMagicZ));
 }
 
-// low bytes of four words -> one word
-__device__ __forceinline__ uint32_t pack_low_bytes(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3) {
-  const uint32_t p01 = __byte_perm(b0, b1, 0x0040);
-  const uint32_t p23 = __byte_perm(b2, b3, 0x0040);
+// STOCHASTIC (Eq. 7) in exact fixed point.  With r = h >> 8 (U = r * 2^-24) and n = floor(t):
+//   U < t - n   <=>   r < ceil((t - n) * 2^24)          (r is an integer)
+// so  n + [U < t - n] = floor((ceil(t * 2^24) + (2^24 - 1 - r)) / 2^24), and 2^24 - 1 - r = (~h) >> 8.
+// Adding zero_point << 24 makes the sum non-negative; byte 3 of the 32-bit sum is the stored code u.
+// t is clamped to the top level first (a quotient that rounded just above L must not reach L + 1),
+// which also keeps the sum below 2^32; the low side cannot pass the lowest code.
+template <int K, int RANGE>
+__device__ __forceinline__ uint32_t quantize_stochastic_word(float x, const Scale& sc, uint32_t h) {
+  constexpr int ZP = (RANGE == kAbsMax) ? (1 << (K - 1)) : 0;
+  constexpr float kTop = (RANGE == kAbsMax) ? (float)((1 << (K - 1)) - 1) : (float)((1 << K) - 1);
+  const float d = (RANGE == kAbsMax) ? x : __fsub_rn(x, sc.base);
+  const float t = fminf(__fmul_rn(d, sc.inv), kTop);
+  const float t24 = __fmul_rn(t, 16777216.0f);  // exact scaling
+  const uint32_t tc = (RANGE == kAbsMax) ? (uint32_t)__float2int_ru(t24) : __float2uint_ru(t24);
+  return tc + ((uint32_t)ZP << 24) + ((~h) >> 8);
+}
+
+// The stored code of one element (any-shape path).
+template <int K, int RANGE, int ROUND>
+__device__ __forceinline__ uint32_t quantize_code(float x, const Scale& sc, uint32_t h) {
+  if (ROUND == kNearest) return quantize_nearest_word<K, RANGE>(x, sc) & 0xFFu;
+  return quantize_stochastic_word<K, RANGE>(x, sc, h) >> 24;
+}
+
+// byte BYTE of four words -> one word
+template <int BYTE>
+__device__ __forceinline__ uint32_t pack_bytes(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3) {
+  constexpr uint32_t sel = (uint32_t)BYTE | ((uint32_t)(BYTE + 4) << 4);
+  const uint32_t p01 = __byte_perm(b0, b1, sel);
+  const uint32_t p23 = __byte_perm(b2, b3, sel);
   return __byte_perm(p01, p23, 0x5410);
 }
 
+// Stochastic codes of an octet whose first counter has parity ODD; pair_lo/key address its first pair.
+template <int K, int RANGE, int ODD>
+__device__ __forceinline__ void quantize_octet_stochastic(const float (&v)[8], const Scale& sc, uint32_t pair_lo,
+                                                          uint32_t key, uint32_t (&b)[8]) {
+  uint32_t h[4 + ODD];
+#pragma unroll
+  for (int p = 0; p < 4 + ODD; ++p) h[p] = Rng::pair_hash(pair_lo + p, key);
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const uint32_t w = h[(e + ODD) >> 1];
+    b[e] = quantize_stochastic_word<K, RANGE>(v[e], sc, ((e + ODD) & 1) ? w * kPairMul : w);
+  }
+}
+
 // Quantizes an octet.  xlo holds the codes of elements 0..3 one per byte, xhi those of 4..7.
-// i0 = index of element 0 in the whole tensor (random-number counter = rng_offset + index).
+// delta = distance of the octet's first counter from the thread's first one (a multiple of 8).
 template <int K, int RANGE, int ROUND>
 __device__ __forceinline__ void quantize_octet(const float (&v)[8], const Scale& sc, const Rng& rng,
-                                               uint64_t ctr0, uint32_t& xlo, uint32_t& xhi) {
+                                               const RngThread& rt, uint32_t delta, uint32_t& xlo, uint32_t& xhi) {
   uint32_t b[8];
   if (ROUND == kStochastic) {
-    const uint32_t lo = (uint32_t)ctr0, hi = (uint32_t)(ctr0 >> 32);
-    if (lo <= 0xFFFFFFF8u) {
-      const uint32_t key = rng.key(hi);
+    if (rt.fast) {
+      if (rt.odd) quantize_octet_stochastic<K, RANGE, 1>(v, sc, rt.pair_lo + delta / 2, rt.key, b);
+      else quantize_octet_stochastic<K, RANGE, 0>(v, sc, rt.pair_lo + delta / 2, rt.key, b);
+    } else {  // the pair index's low word (or the counter itself) wraps somewhere in this thread's span
 #pragma unroll
-      for (int e = 0; e < 8; ++e)
-        b[e] = quantize_bits<K, RANGE, ROUND>(v[e], sc, Rng::uniform(lo + e, key));
-    } else {  // the counter's low word wraps inside this octet
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const uint64_t c = ctr0 + e;
-        b[e] = quantize_bits<K, RANGE, ROUND>(
-            v[e], sc, Rng::uniform((uint32_t)c, rng.key((uint32_t)(c >> 32))));
-      }
+      for (int e = 0; e < 8; ++e) b[e] = quantize_stochastic_word<K, RANGE>(v[e], sc, rng.word(rt.ctr_first + delta + e));
     }
+    xlo = pack_bytes<3>(b[0], b[1], b[2], b[3]);
+    xhi = pack_bytes<3>(b[4], b[5], b[6], b[7]);
   } else {
 #pragma unroll
-    for (int e = 0; e < 8; ++e) b[e] = quantize_bits<K, RANGE, ROUND>(v[e], sc, 0.0f);
+    for (int e = 0; e < 8; ++e) b[e] = quantize_nearest_word<K, RANGE>(v[e], sc);
+    xlo = pack_bytes<0>(b[0], b[1], b[2], b[3]);
+    xhi = pack_bytes<0>(b[4], b[5], b[6], b[7]);
   }
-  xlo = pack_low_bytes(b[0], b[1], b[2], b[3]);
-  xhi = pack_low_bytes(b[4], b[5], b[6], b[7]);
 }
 
 // ----------------------------------------------------------------------------- bit permutations

@@ -118,12 +118,9 @@ __device__ void compress_chunk_generic(const CodecArgs& a, uint64_t m, float* s_
     if (t < valid) {
       float v = __ldg(x + t);
       if (sc.nonfinite) v = 0.0f;
-      float U = 0.0f;
-      if (ROUND == kStochastic) {
-        const uint64_t c = a.rng_offset + i0 + t;
-        U = Rng::uniform((uint32_t)c, rng.key((uint32_t)(c >> 32)));
-      }
-      u = quantize_bits<K, RANGE, ROUND>(v, sc, U) & 0xFFu;
+      uint32_t h = 0;
+      if (ROUND == kStochastic) h = rng.word(a.rng_offset + i0 + t);
+      u = quantize_code<K, RANGE, ROUND>(v, sc, h);
     }
     const uint64_t word0 = (i0 / 32 + g) * K;
 #pragma unroll
@@ -211,11 +208,13 @@ __global__ void __launch_bounds__(BLOCK_MAX, BLOCK_MAX == 256 ? (R <= 2 ? 6 : 4)
   }
 
   const Rng rng{(uint32_t)a.seed, (uint32_t)(a.seed >> 32)};
+  RngThread rt;
+  if (ROUND == kStochastic) rt.init(rng, a.rng_offset + e0 + 8ull * gt, 8u * (R - 1) * tpc + 8u);
 #pragma unroll
   for (int r = 0; r < R; ++r) {
     const uint64_t oct = e0 / 8 + (r * tpc + gt);  // global octet index
     uint32_t xlo, xhi;
-    quantize_octet<K, RANGE, ROUND>(v[r], sc, rng, a.rng_offset + oct * 8, xlo, xhi);
+    quantize_octet<K, RANGE, ROUND>(v[r], sc, rng, rt, 8u * r * tpc, xlo, xhi);
     if (LAYOUT == kInterleaved) {
       if (active) store_interleaved<K>(a.payload, oct, xlo, xhi);
     } else {

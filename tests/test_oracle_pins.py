@@ -313,12 +313,12 @@ def test_stochastic_is_deterministic_and_counter_based():
 
 
 def test_rng_uniformity():
-    """Chi-square over 64 bins for consecutive counters, a few seeds; U in [0,1) on a 2^-23 grid."""
+    """Chi-square over 64 bins for consecutive counters, a few seeds; U in [0,1) on a 2^-24 grid."""
     n, bins = 1 << 16, 64
     for seed in (0, 1, 2 ** 40 + 12345):
         u = np.array([oracle.rng_uniform(seed, 7 * 2 ** 32 - n // 2 + i) for i in range(n)])
         assert u.min() >= 0 and u.max() < 1
-        assert np.all(u * 2 ** 23 == np.floor(u * 2 ** 23))
+        assert np.all(u * 2 ** 24 == np.floor(u * 2 ** 24))
         hist = np.bincount((u * bins).astype(int), minlength=bins)
         chi2 = ((hist - n / bins) ** 2 / (n / bins)).sum()
         assert chi2 < 120  # 63 dof: mean 63, sd 11.2; 120 is > 5 sd
@@ -331,10 +331,41 @@ def test_rng_uniformity():
         assert abs(((h >> np.uint64(b)) & np.uint64(1)).mean() - 0.5) < 0.03
 
 
-def test_rng_hash_known_fixed_point():
-    """fmix32(0) = 0, so seed 0 / counter 0 hashes to 0 (a property of the published finaliser)."""
-    assert oracle.rng_hash(0, 0) == 0
-    assert oracle.rng_hash(0, 1) != 0 and oracle.rng_hash(1, 0) != 0
+def fmix32_py(h):
+    """MurmurHash3's 32-bit finaliser as published (two multiplies, three xor-shifts)."""
+    h ^= h >> 16
+    h = (h * 0x85EBCA6B) & 0xFFFFFFFF
+    h ^= h >> 13
+    h = (h * 0xC2B2AE35) & 0xFFFFFFFF
+    h ^= h >> 16
+    return h
+
+
+def test_rng_pair_structure_and_finaliser():
+    """Counters 2j, 2j+1 share one finaliser output; the odd one is that word times an odd constant
+    (a bijection, so each stays uniform); seed 0 / counter 0 does not sit on fmix32(0) = 0."""
+    assert fmix32_py(0) == 0 and fmix32_py(1) == 0x514E28B7  # published finaliser: fixed point and one value
+    for seed, j in [(0, 0), (5, 77), (2 ** 63 + 9, 2 ** 40 + 3)]:
+        even, odd = oracle.rng_hash(seed, 2 * j), oracle.rng_hash(seed, 2 * j + 1)
+        assert odd == (even * 0x9E3779B1) & 0xFFFFFFFF
+        inner = fmix32_py(((j >> 32) ^ (seed & 0xFFFFFFFF) ^ 0x9E3779B9) & 0xFFFFFFFF)
+        assert even == fmix32_py(((j & 0xFFFFFFFF) ^ inner ^ (seed >> 32)) & 0xFFFFFFFF)
+    assert oracle.rng_hash(0, 0) != 0 and oracle.rng_hash(0, 1) != 0
+
+
+def test_rng_pairs_are_jointly_uniform():
+    """The two numbers of a pair: no correlation, and a 16 x 16 chi-square of (U_even, U_odd)."""
+    n = 1 << 16
+    u = np.array([oracle.rng_uniform(3, i) for i in range(2 * n)]).reshape(n, 2)
+    assert abs(np.corrcoef(u[:, 0], u[:, 1])[0, 1]) < 0.02
+    cells = (u[:, 0] * 16).astype(int) * 16 + (u[:, 1] * 16).astype(int)
+    hist = np.bincount(cells, minlength=256)
+    chi2 = ((hist - n / 256) ** 2 / (n / 256)).sum()
+    assert chi2 < 360  # 255 dof: mean 255, sd 22.6
+    # the low bits of the 24 used are as balanced as the high ones
+    r = (u * 2 ** 24).astype(np.int64)
+    for b in range(24):
+        assert abs(((r >> b) & 1).mean() - 0.5) < 0.01
 
 
 # ------------------------------------------------------------------ packing: round trip and brute force
