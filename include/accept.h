@@ -119,14 +119,18 @@ size_t accept_compressed_size(const accept_params* p);
 size_t accept_payload_offset(const accept_params* p);
 
 /*
- * Bytes of device workspace the kernels need: 16.  Word 0 is the device status word; the caller
- * zeroes the workspace once (and whenever it wants to clear the status).  0 if p is invalid.
+ * Bytes of device workspace the kernels need: 16, plus 16 per chunk when chunk_elems > 32768
+ * (such chunks do not fit on chip: their ranges are gathered in the workspace first, and the input
+ * is read twice).  Word 0 is the device status word; the caller zeroes the workspace once (and
+ * whenever it wants to clear the status); the workspace must be 16-byte aligned.  0 if p is invalid.
  */
 size_t accept_workspace_size(const accept_params* p);
 
 /*
  * Quantizer + encoder (Sec. 3.3): reads n_elems floats at d_x, writes accept_compressed_size(p)
- * bytes at d_stream (header, per-chunk {s,o}, payload), in one kernel launch on cuda_stream
+ * bytes at d_stream (header, per-chunk {s,o}, payload), in one kernel launch (three launches and a
+ * memset of the workspace records when chunk_elems > 32768, e.g. one range for the whole tensor as
+ * in the paper) on cuda_stream
  * (a cudaStream_t, may be NULL for the default stream).  Non-finite input does not fail the call:
  * the chunk is written as degenerate and ACCEPT_DEV_NONFINITE is or-ed into the status word.
  * d_x is only read; d_stream is fully overwritten up to the compressed size.

@@ -8,6 +8,7 @@
 #include <mutex>
 
 #include "accept_kernels.cuh"
+#include "accept_wide.cuh"
 
 namespace {
 
@@ -18,6 +19,11 @@ std::atomic<uint64_t> g_launches{0};
 bool is_aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 uint64_t n_chunks_of(const accept_params* p) { return (p->n_elems + p->chunk_elems - 1) / p->chunk_elems; }
+
+// Chunks above this size are coded by the three-launch wide path (accept_wide.cuh).
+constexpr uint32_t kWideChunk = 32768;
+
+bool is_wide(const accept_params* p) { return p->chunk_elems > kWideChunk; }
 
 // Geometry of the register-resident compress path for chunk size C: rounds R and threads per chunk.
 struct FastGeometry { int rounds; uint32_t tpc; };
@@ -120,6 +126,50 @@ KernelFn select_decompress(const accept_params* p, bool aligned, int rounds) {
   }
 }
 
+// ---- wide chunks: ranges, constants, encode ------------------------------------------------------
+
+template <int K, int LAYOUT, int RANGE>
+void launch_wide_encode(int round, const CodecArgs& a, const accept::ChunkRecord* rec, unsigned grid, cudaStream_t s) {
+  if (round == accept::kNearest) accept::wide_encode_kernel<K, LAYOUT, RANGE, accept::kNearest, 2><<<grid, 256, 0, s>>>(a, rec);
+  else accept::wide_encode_kernel<K, LAYOUT, RANGE, accept::kStochastic, 2><<<grid, 256, 0, s>>>(a, rec);
+}
+
+template <int RANGE>
+void launch_wide_encode_for(const accept_params* p, const CodecArgs& a, const accept::ChunkRecord* rec, unsigned grid,
+                            cudaStream_t s) {
+  const bool bp = p->layout == ACCEPT_LAYOUT_BITPLANE;
+  switch (p->k) {
+    case 2: bp ? launch_wide_encode<2, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
+               : launch_wide_encode<2, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s); break;
+    case 3: launch_wide_encode<3, accept::kBitplane, RANGE>(p->round, a, rec, grid, s); break;
+    case 4: bp ? launch_wide_encode<4, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
+               : launch_wide_encode<4, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s); break;
+    default: bp ? launch_wide_encode<8, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
+                : launch_wide_encode<8, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s); break;
+  }
+}
+
+// rec_bytes = the workspace past its first 16 bytes: one record per chunk, cleared here.
+accept_status launch_wide(const accept_params* p, const CodecArgs& a, uint8_t* rec_bytes, cudaStream_t s) {
+  accept::ChunkRecord* rec = reinterpret_cast<accept::ChunkRecord*>(rec_bytes);
+  if (cudaMemsetAsync(rec, 0, sizeof(accept::ChunkRecord) * a.n_chunks, s) != cudaSuccess) return ACCEPT_ERR_CUDA;
+  const uint64_t n_oct = (p->n_elems + 7) / 8;
+  const unsigned range_grid = (unsigned)((n_oct + 4 * 256 - 1) / (4 * 256));
+  const unsigned fin_grid = (unsigned)((a.n_chunks + 255) / 256);
+  const unsigned enc_grid = (unsigned)((((p->n_elems + 31) / 32) * 4 + 2 * 256 - 1) / (2 * 256));
+  if (p->range == ACCEPT_RANGE_ABSMAX) {
+    accept::wide_range_kernel<accept::kAbsMax, 4><<<range_grid, 256, 0, s>>>(a, rec);
+    accept::wide_finalize_kernel<accept::kAbsMax><<<fin_grid, 256, 0, s>>>(a, rec);
+    launch_wide_encode_for<accept::kAbsMax>(p, a, rec, enc_grid, s);
+  } else {
+    accept::wide_range_kernel<accept::kMinMax, 4><<<range_grid, 256, 0, s>>>(a, rec);
+    accept::wide_finalize_kernel<accept::kMinMax><<<fin_grid, 256, 0, s>>>(a, rec);
+    launch_wide_encode_for<accept::kMinMax>(p, a, rec, enc_grid, s);
+  }
+  g_launches.fetch_add(3, std::memory_order_relaxed);
+  return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+}
+
 // ---- built-in scratch for accept_compress_static ------------------------------------------------
 //
 // The workspace of callers that cannot allocate.  In host code the name g_static_scratch is only a
@@ -186,7 +236,8 @@ size_t accept_compressed_size(const accept_params* p) {
 
 size_t accept_workspace_size(const accept_params* p) {
   if (accept_check_params(p) != ACCEPT_OK) return 0;
-  return 16;
+  // status word (+ pad); chunks wider than 32768 elements also need one 16-byte record each
+  return 16 + (is_wide(p) ? 16 * (size_t)n_chunks_of(p) : 0);
 }
 
 accept_status accept_compress(const accept_params* p, const float* d_x, void* d_stream, size_t stream_bytes,
@@ -195,6 +246,11 @@ accept_status accept_compress(const accept_params* p, const float* d_x, void* d_
   if (st != ACCEPT_OK) return st;
   CodecArgs a = make_args(p, d_stream, d_ws);
   a.x = d_x;
+
+  if (is_wide(p) && is_aligned(d_x, 32)) {
+    if (!is_aligned(d_ws, 16)) return ACCEPT_ERR_MISALIGNED;
+    return launch_wide(p, a, static_cast<uint8_t*>(d_ws) + 16, static_cast<cudaStream_t>(cuda_stream));
+  }
 
   const FastGeometry g = fast_geometry(p->chunk_elems);
   const bool fast = g.rounds != 0 && is_aligned(d_x, 32);

@@ -124,6 +124,46 @@ def test_parity_large_chunks(chunk, mode):
     check_roundtrip(x, chunk, k, range_, round_, layout, seed=5)
 
 
+@pytest.mark.parametrize("mode", modes(), ids=MODE_IDS)
+@pytest.mark.parametrize("chunk,n", [
+    (32800, 32800 * 5 + 12345),      # not a power of two: blocks of the range pass straddle chunk boundaries
+    (65536, 65536 * 3 + 8191),       # n not a multiple of 8: a partly filled last octet
+    (1 << 18, (1 << 18) + 33),
+    (1 << 21, 1500003),              # one range for the whole tensor (chunk >= n)
+])
+def test_parity_wide_chunks(mode, chunk, n):
+    """Chunks above 32768 elements: ranges gathered in the workspace, constants, then encode."""
+    k, range_, round_, layout = mode
+    x = workloads.random_tensor(n, chunk + k, "normal")
+    check_roundtrip(x, chunk, k, range_, round_, layout, seed=77, rng_offset=2 ** 32 - 70000)
+
+
+@pytest.mark.parametrize("bad", [np.nan, -np.inf])
+def test_wide_chunks_degenerate_and_nonfinite(bad):
+    chunk = 40000 // 32 * 32
+    x = workloads.random_tensor(chunk * 6 + 5, 3, "normal")
+    x[:chunk] = 0.0                  # all-zero chunk
+    x[chunk:2 * chunk] = 1e-42       # L/c overflows
+    x[2 * chunk:3 * chunk] = -7.0    # constant chunk
+    for range_ in (RANGE_ABSMAX, RANGE_MINMAX):
+        check_roundtrip(x, chunk, 4, range_, ROUND_NEAREST, LAYOUT_BITPLANE)
+        check_roundtrip(x, chunk, 8, range_, ROUND_STOCHASTIC, LAYOUT_INTERLEAVED, seed=3)
+    x[4 * chunk + 17] = bad
+    x[-1] = bad                      # also in the partial last chunk
+    for range_ in (RANGE_ABSMAX, RANGE_MINMAX):
+        check_roundtrip(x, chunk, 4, range_, ROUND_NEAREST, LAYOUT_INTERLEAVED)
+        check_roundtrip(x, chunk, 2, range_, ROUND_STOCHASTIC, LAYOUT_BITPLANE, seed=4)
+
+
+def test_per_tensor_range_on_a_large_tensor():
+    """The paper's granularity (one scaling factor per tensor) on the 205 MB gradient, every element."""
+    spec = workloads.TENSORS["cfg3_grad"]
+    x = workloads.generate("cfg3_grad")
+    chunk = (x.size + 31) // 32 * 32
+    check_roundtrip(x, chunk, 4, RANGE_ABSMAX, ROUND_STOCHASTIC, LAYOUT_INTERLEAVED, seed=spec.seed)
+    check_roundtrip(x, chunk, 8, RANGE_ABSMAX, ROUND_NEAREST, LAYOUT_INTERLEAVED)
+
+
 @pytest.mark.parametrize("n", [1, 2, 7, 8, 9, 31, 32, 33, 63, 255, 257, 4095, 4097])
 def test_parity_tiny_and_ragged(n):
     for k, range_, round_, layout in [(2, RANGE_ABSMAX, ROUND_NEAREST, LAYOUT_INTERLEAVED),

@@ -52,7 +52,23 @@ def test_size_queries_match_oracle(A, n, chunk, k):
     assert A.accept_check_params(p) == 0
     assert A.accept_compressed_size(p) == oracle.stream_bytes(n, chunk, k)
     assert A.accept_payload_offset(p) == oracle.payload_offset(n, chunk)
-    assert A.accept_workspace_size(p) == 16
+    assert A.accept_workspace_size(p) == 16 + (16 * -(-n // chunk) if chunk > 32768 else 0)
+
+
+def test_workspace_grows_with_wide_chunks_and_static_scratch_refuses_them(A):
+    """16 bytes, plus a 16-byte record per chunk once chunks exceed 32768 elements; the built-in
+    256-byte scratch of accept_compress_static holds 15 such records and refuses more."""
+    from paper_2311_05827_b200 import binding
+    assert A.accept_workspace_size(A.Params(10 ** 6, 32768, 4)) == 16
+    assert A.accept_workspace_size(A.Params(10 ** 6, 32800, 4)) == 16 + 16 * 31
+    assert A.accept_workspace_size(A.Params(10 ** 6, 1 << 20, 4)) == 32
+    lib = binding.lib()
+    good = 0x10000
+    for n, chunk, want in [(10 ** 6, 32800, 11), (15 * 65536, 65536, 1)]:  # 31 records: refused; 15 fit (then NULL input)
+        p = A.Params(n, chunk, 4)
+        size = A.accept_compressed_size(p)
+        x_ptr = good if want == 11 else None
+        assert lib.accept_compress_static(ctypes.byref(p.c()), x_ptr, good, size, None, None) == want
 
 
 def test_invalid_params_are_rejected(A):
