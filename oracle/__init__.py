@@ -65,6 +65,25 @@ def _load():
     lib.oracle_decompress.argtypes = [vp, u64, u64, vp]
     lib.oracle_bitwidth_schedule.restype = i32
     lib.oracle_bitwidth_schedule.argtypes = [i32, i32]
+    f32p = vp
+    lib.oracle_mbq_payload_offset.restype = u64
+    lib.oracle_mbq_payload_offset.argtypes = [u32]
+    lib.oracle_mbq_stream_bytes.restype = u64
+    lib.oracle_mbq_stream_bytes.argtypes = [u64, u32]
+    lib.oracle_mbq_levels.restype = None
+    lib.oracle_mbq_levels.argtypes = [f32p, u32, f32p]
+    lib.oracle_mbq_assign_nearest.restype = None
+    lib.oracle_mbq_assign_nearest.argtypes = [vp, u64, f32p, u32, vp]
+    lib.oracle_mbq_assign_residue.restype = None
+    lib.oracle_mbq_assign_residue.argtypes = [vp, u64, u32, vp, f32p]
+    lib.oracle_mbq_update_alpha.restype = None
+    lib.oracle_mbq_update_alpha.argtypes = [vp, vp, u64, u32, f32p, u32, f32p]
+    lib.oracle_mbq_bias.restype = ctypes.c_float
+    lib.oracle_mbq_bias.argtypes = [vp, vp, u64, u32, f32p]
+    lib.oracle_mbq_compress.restype = None
+    lib.oracle_mbq_compress.argtypes = [vp, u64, u32, u32, i32, f32p, vp, f32p]
+    lib.oracle_mbq_decompress.restype = i32
+    lib.oracle_mbq_decompress.argtypes = [vp, u64, u64, vp]
     _lib = lib
     return lib
 
@@ -168,3 +187,67 @@ def split_stream(stream, n: int, chunk: int):
 
 def bitwidth_schedule(is_backward: bool, n_lr_changes: int) -> int:
     return int(_load().oracle_bitwidth_schedule(int(is_backward), n_lr_changes))
+
+
+# ---------------------------------------------------------------- multi-bit quantization (forward path)
+
+def mbq_payload_offset(k: int) -> int:
+    return int(_load().oracle_mbq_payload_offset(k))
+
+
+def mbq_stream_bytes(n: int, k: int) -> int:
+    return int(_load().oracle_mbq_stream_bytes(n, k))
+
+
+def mbq_levels(alpha) -> np.ndarray:
+    alpha = _f32(alpha)
+    out = np.empty(1 << alpha.size, dtype=np.float32)
+    _load().oracle_mbq_levels(_ptr(alpha), alpha.size, _ptr(out))
+    return out
+
+
+def mbq_assign_nearest(x, alpha) -> np.ndarray:
+    x, alpha = _f32(x), _f32(alpha)
+    codes = np.empty(x.size, dtype=np.uint8)
+    _load().oracle_mbq_assign_nearest(_ptr(x), x.size, _ptr(alpha), alpha.size, _ptr(codes))
+    return codes
+
+
+def mbq_assign_residue(x, k: int):
+    x = _f32(x)
+    codes = np.empty(x.size, dtype=np.uint8)
+    alpha0 = np.empty(k, dtype=np.float32)
+    _load().oracle_mbq_assign_residue(_ptr(x), x.size, k, _ptr(codes), _ptr(alpha0))
+    return codes, alpha0
+
+
+def mbq_update_alpha(x, codes, alpha_prev, t: int) -> np.ndarray:
+    x, alpha_prev = _f32(x), _f32(alpha_prev)
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    out = np.empty(alpha_prev.size, dtype=np.float32)
+    _load().oracle_mbq_update_alpha(_ptr(x), _ptr(codes), x.size, alpha_prev.size, _ptr(alpha_prev), t, _ptr(out))
+    return out
+
+
+def mbq_bias(x, codes, alpha) -> float:
+    x, alpha = _f32(x), _f32(alpha)
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    return float(_load().oracle_mbq_bias(_ptr(x), _ptr(codes), x.size, alpha.size, _ptr(alpha)))
+
+
+def mbq_compress(x, k: int, t: int, init: bool, alpha_prev=None):
+    """-> (stream uint8[], alpha_next float32[k])."""
+    x = _f32(x)
+    alpha_prev = np.zeros(k, dtype=np.float32) if alpha_prev is None else _f32(alpha_prev)
+    stream = np.empty(mbq_stream_bytes(x.size, k), dtype=np.uint8)
+    alpha_next = np.empty(k, dtype=np.float32)
+    _load().oracle_mbq_compress(_ptr(x), x.size, k, t, int(init), _ptr(alpha_prev), _ptr(stream), _ptr(alpha_next))
+    return stream, alpha_next
+
+
+def mbq_decompress(stream, n: int) -> np.ndarray:
+    stream = np.ascontiguousarray(stream, dtype=np.uint8).reshape(-1)
+    xhat = np.empty(n, dtype=np.float32)
+    if _load().oracle_mbq_decompress(_ptr(stream), stream.size, n, _ptr(xhat)) != 0:
+        raise ValueError("oracle_mbq_decompress: invalid stream header")
+    return xhat

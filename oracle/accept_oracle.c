@@ -323,3 +323,194 @@ int oracle_bitwidth_schedule(int is_backward, int n_lr_changes) {
   if (is_backward) return n_lr_changes == 0 ? 8 : 4;
   return (2 + n_lr_changes > 4) ? 4 : 2 + n_lr_changes;
 }
+
+/* ============================================================================================
+ * Forward quantizer: multi-bit quantization (Sec. 3.3 "Forward Quantizer", Eq. 1-5), its encoder
+ * ("Forward Encoder") and the receiver side (Sec. 3.4 "Forward Decoder", "Forward Dequantizer").
+ *
+ * x_v ~ B_v alpha with B_v in {-1,+1}^(N x k): element i carries k signs b_i0..b_i,k-1, stored as
+ * the k-bit code c_i = sum_j [b_ij = +1] << j ("replace all the -1s with 0"), packed as bit planes
+ * (plane j = basis j).  The 2^k possible values (the set P of the paper) are
+ *     level(c) = (+-alpha_0) + (+-alpha_1) + ... summed in fp32 in the order j = 0..k-1.
+ *
+ * Readings:
+ *   - batch t >= 1: B^t = nearest element of P^(t-1) for every value (exact comparison of the
+ *     distances; a tie goes to the lower level; codes whose levels coincide: the smallest code);
+ *     then alpha_cur = (B^T B)^-1 B^T x (Eq. 3) and alpha^t = beta alpha^(t-1) + (1-beta) alpha_cur
+ *     with beta = min(0.9, (1+t)/(10+t)) (Eq. 4), all in double, rounded once to fp32.  If B^T B is
+ *     singular (a pivot below 1e-9 N) alpha_cur = alpha^(t-1).
+ *   - the stream carries alpha^t (the coefficients after the update) and m_q = E[B alpha^t - x]
+ *     (Eq. 5), so that the receiver computes B alpha^t - m_q ("Forward Dequantizer").
+ *   - batch 0 of an epoch: residue method: r = x; for j = 0..k-1: b_j = sign(r) (+1 for r >= 0),
+ *     alpha_j = mean |r|, r <- r - alpha_j b_j (fp32 residues, double means); no Eq. 3/4 update.
+ * ============================================================================================ */
+
+#define MBQ_MAGIC_KIND 1u /* header word 7 */
+
+uint64_t oracle_mbq_payload_offset(uint32_t k) {
+  uint64_t off = 32 + 4 * (uint64_t)(k + 1); /* alpha (k floats) and m_q: the 32(k+1) bits of Eq. 8 */
+  return (off + 15) / 16 * 16;
+}
+
+uint64_t oracle_mbq_stream_bytes(uint64_t n, uint32_t k) {
+  return oracle_mbq_payload_offset(k) + oracle_payload_bytes(n, k);
+}
+
+/* The set P: levels[c] for every code c. */
+void oracle_mbq_levels(const float* alpha, uint32_t k, float* levels) {
+  for (uint32_t c = 0; c < (1u << k); ++c) {
+    float v = 0.0f;
+    for (uint32_t j = 0; j < k; ++j) {
+      float term = ((c >> j) & 1u) ? alpha[j] : -alpha[j];
+      v = (j == 0) ? term : v + term;
+    }
+    levels[c] = v;
+  }
+}
+
+/* Closest value of P for every element. */
+void oracle_mbq_assign_nearest(const float* x, uint64_t n, const float* alpha, uint32_t k, uint8_t* codes) {
+  float levels[256];
+  oracle_mbq_levels(alpha, k, levels);
+  for (uint64_t i = 0; i < n; ++i) {
+    uint32_t best = 0;
+    double best_d = fabs((double)x[i] - (double)levels[0]);
+    for (uint32_t c = 1; c < (1u << k); ++c) {
+      double d = fabs((double)x[i] - (double)levels[c]);
+      if (d < best_d || (d == best_d && levels[c] < levels[best])) { best = c; best_d = d; }
+    }
+    codes[i] = (uint8_t)best;
+  }
+}
+
+/* Residue-based initialisation: signs of the successive residues and alpha_j = mean |residue|. */
+void oracle_mbq_assign_residue(const float* x, uint64_t n, uint32_t k, uint8_t* codes, float* alpha0) {
+  float* r = (float*)malloc(sizeof(float) * n);
+  memcpy(r, x, sizeof(float) * n);
+  memset(codes, 0, n);
+  for (uint32_t j = 0; j < k; ++j) {
+    double sum = 0.0;
+    for (uint64_t i = 0; i < n; ++i) sum += fabs((double)r[i]);
+    alpha0[j] = (float)(sum / (double)n);
+    for (uint64_t i = 0; i < n; ++i) {
+      if (r[i] >= 0.0f) { codes[i] |= (uint8_t)(1u << j); r[i] = r[i] - alpha0[j]; }
+      else r[i] = r[i] + alpha0[j];
+    }
+  }
+  free(r);
+}
+
+/* Eq. 3: least squares for alpha given the signs; returns 0 and leaves alpha_cur = alpha_prev if singular. */
+static int mbq_least_squares(const float* x, const uint8_t* codes, uint64_t n, uint32_t k, const float* alpha_prev,
+                             double* alpha_cur) {
+  double G[8][8], rhs[8];
+  for (uint32_t p = 0; p < k; ++p) {
+    rhs[p] = 0.0;
+    for (uint32_t q = 0; q < k; ++q) G[p][q] = 0.0;
+  }
+  for (uint64_t i = 0; i < n; ++i) {
+    double b[8];
+    for (uint32_t p = 0; p < k; ++p) b[p] = ((codes[i] >> p) & 1u) ? 1.0 : -1.0;
+    for (uint32_t p = 0; p < k; ++p) {
+      rhs[p] += b[p] * (double)x[i];
+      for (uint32_t q = 0; q < k; ++q) G[p][q] += b[p] * b[q];
+    }
+  }
+  /* Gaussian elimination with partial pivoting */
+  for (uint32_t c = 0; c < k; ++c) {
+    uint32_t piv = c;
+    for (uint32_t r = c + 1; r < k; ++r)
+      if (fabs(G[r][c]) > fabs(G[piv][c])) piv = r;
+    if (fabs(G[piv][c]) < 1e-9 * (double)n) {
+      for (uint32_t p = 0; p < k; ++p) alpha_cur[p] = (double)alpha_prev[p];
+      return 0;
+    }
+    if (piv != c) {
+      for (uint32_t q = 0; q < k; ++q) { double t = G[c][q]; G[c][q] = G[piv][q]; G[piv][q] = t; }
+      double t = rhs[c]; rhs[c] = rhs[piv]; rhs[piv] = t;
+    }
+    for (uint32_t r = c + 1; r < k; ++r) {
+      double f = G[r][c] / G[c][c];
+      for (uint32_t q = c; q < k; ++q) G[r][q] -= f * G[c][q];
+      rhs[r] -= f * rhs[c];
+    }
+  }
+  for (int c = (int)k - 1; c >= 0; --c) {
+    double s = rhs[c];
+    for (uint32_t q = (uint32_t)c + 1; q < k; ++q) s -= G[c][q] * alpha_cur[q];
+    alpha_cur[c] = s / G[c][c];
+  }
+  return 1;
+}
+
+/* Eq. 3 + Eq. 4: alpha^t from alpha^(t-1), the signs and the data. */
+void oracle_mbq_update_alpha(const float* x, const uint8_t* codes, uint64_t n, uint32_t k, const float* alpha_prev,
+                             uint32_t t, float* alpha_next) {
+  double cur[8];
+  mbq_least_squares(x, codes, n, k, alpha_prev, cur);
+  double beta = (1.0 + (double)t) / (10.0 + (double)t);
+  if (beta > 0.9) beta = 0.9;
+  for (uint32_t p = 0; p < k; ++p) alpha_next[p] = (float)(beta * (double)alpha_prev[p] + (1.0 - beta) * cur[p]);
+}
+
+/* Eq. 5: mean of the quantization error of B alpha. */
+float oracle_mbq_bias(const float* x, const uint8_t* codes, uint64_t n, uint32_t k, const float* alpha) {
+  double sum_x = 0.0, acc = 0.0;
+  for (uint64_t i = 0; i < n; ++i) sum_x += (double)x[i];
+  for (uint32_t p = 0; p < k; ++p) {
+    int64_t s = 0; /* sum of the signs of basis p */
+    for (uint64_t i = 0; i < n; ++i) s += ((codes[i] >> p) & 1u) ? 1 : -1;
+    acc += (double)alpha[p] * (double)s;
+  }
+  return (float)((acc - sum_x) / (double)n);
+}
+
+/* Whole forward compressor for batch t; init != 0 selects the residue method (alpha_prev unused).
+ * Writes the stream and alpha_next (= the alpha carried by the stream). */
+void oracle_mbq_compress(const float* x, uint64_t n, uint32_t k, uint32_t t, int init, const float* alpha_prev,
+                         void* stream, float* alpha_next) {
+  uint8_t* bytes = (uint8_t*)stream;
+  memset(bytes, 0, oracle_mbq_stream_bytes(n, k));
+  uint8_t* codes = (uint8_t*)malloc(n);
+  if (init) {
+    oracle_mbq_assign_residue(x, n, k, codes, alpha_next);
+  } else {
+    oracle_mbq_assign_nearest(x, n, alpha_prev, k, codes);
+    oracle_mbq_update_alpha(x, codes, n, k, alpha_prev, t, alpha_next);
+  }
+  float m_q = oracle_mbq_bias(x, codes, n, k, alpha_next);
+  uint32_t header[8] = {ORACLE_MAGIC, ORACLE_VERSION, (uint32_t)n, (uint32_t)(n >> 32), 0u, k, 0u, MBQ_MAGIC_KIND};
+  memcpy(bytes, header, 32);
+  memcpy(bytes + 32, alpha_next, 4 * k);
+  memcpy(bytes + 32 + 4 * k, &m_q, 4);
+  /* bit planes: plane j of group g = basis j of elements 32g..32g+31, -1 stored as 0 */
+  uint32_t* payload = (uint32_t*)(bytes + oracle_mbq_payload_offset(k));
+  for (uint64_t i = 0; i < n; ++i)
+    for (uint32_t j = 0; j < k; ++j)
+      payload[(i / 32) * k + j] |= (uint32_t)((codes[i] >> j) & 1u) << (i % 32);
+  free(codes);
+}
+
+/* Receiver: decode the planes, x_hat = B alpha - m_q.  Returns -1 on a bad header. */
+int oracle_mbq_decompress(const void* stream, uint64_t stream_bytes, uint64_t n_expected, float* xhat) {
+  const uint8_t* bytes = (const uint8_t*)stream;
+  uint32_t header[8];
+  if (stream_bytes < 32) return -1;
+  memcpy(header, bytes, 32);
+  uint64_t n = (uint64_t)header[2] | ((uint64_t)header[3] << 32);
+  uint32_t k = header[5];
+  if (header[0] != ORACLE_MAGIC || header[1] != ORACLE_VERSION || header[7] != MBQ_MAGIC_KIND) return -1;
+  if (n != n_expected || n == 0 || k < 1 || k > 4) return -1;
+  if (stream_bytes < oracle_mbq_stream_bytes(n, k)) return -1;
+  float alpha[8], m_q, levels[256];
+  memcpy(alpha, bytes + 32, 4 * k);
+  memcpy(&m_q, bytes + 32 + 4 * k, 4);
+  oracle_mbq_levels(alpha, k, levels);
+  const uint32_t* payload = (const uint32_t*)(bytes + oracle_mbq_payload_offset(k));
+  for (uint64_t i = 0; i < n; ++i) {
+    uint32_t c = 0;
+    for (uint32_t j = 0; j < k; ++j) c |= ((payload[(i / 32) * k + j] >> (i % 32)) & 1u) << j;
+    xhat[i] = levels[c] - m_q;
+  }
+  return 0;
+}

@@ -1,0 +1,161 @@
+"""Pins for the oracle's forward quantizer (multi-bit quantization, Eq. 1-5): the paper's level set,
+library least squares, brute-force nearest level, closed forms and exact-recovery cases."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def signs(codes, k):
+    """B in {-1,+1}^(n x k) from codes (bit j set <-> +1)."""
+    return ((codes[:, None] >> np.arange(k)) & 1).astype(np.float64) * 2 - 1
+
+
+def test_level_set_of_the_paper_k2():
+    rows = dict((l.split()[0], [float(v) for v in l.split()[1:]])
+                for l in open(os.path.join(GOLDEN, "mbq_level_set_k2.txt")) if l.strip() and not l.startswith("#"))
+    levels = oracle.mbq_levels(rows["alpha"])
+    a1, a2 = rows["alpha"]
+    assert sorted(levels.tolist()) == sorted([-a1 - a2, a1 - a2, -a1 + a2, a1 + a2]) == sorted(rows["levels"])
+    # code bit j set <-> +alpha_j
+    assert levels.tolist() == [-a1 - a2, a1 - a2, -a1 + a2, a1 + a2]
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 4])
+def test_levels_are_B_alpha(k):
+    alpha = np.array([1.7, 0.9, 0.41, 0.2][:k], dtype=np.float32)
+    codes = np.arange(1 << k, dtype=np.uint8)
+    want = signs(codes, k) @ alpha.astype(np.float64)
+    assert np.allclose(oracle.mbq_levels(alpha), want, rtol=0, atol=1e-6)
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 4])
+def test_nearest_level_against_brute_force(k):
+    rng = np.random.default_rng(k)
+    alpha = np.abs(rng.standard_normal(k)).astype(np.float32) + 0.05
+    x = workloads.random_tensor(5000, 40 + k, "normal") * np.float32(1.5)
+    codes = oracle.mbq_assign_nearest(x, alpha)
+    levels = oracle.mbq_levels(alpha).astype(np.float64)
+    dist = np.abs(x.astype(np.float64)[:, None] - levels[None, :])
+    assert np.array_equal(dist[np.arange(x.size), codes], dist.min(axis=1))
+    # a value equal to a level gets that level; a midpoint goes to the lower one
+    lv = np.sort(oracle.mbq_levels(np.array([2.0, 1.0][:min(k, 2)], dtype=np.float32)))
+    a = np.array([2.0, 1.0][:min(k, 2)], dtype=np.float32)
+    probe = np.concatenate([lv, (lv[:-1] + lv[1:]) / 2]).astype(np.float32)
+    got = oracle.mbq_levels(a)[oracle.mbq_assign_nearest(probe, a)]
+    assert np.array_equal(got[:lv.size], lv) and np.array_equal(got[lv.size:], lv[:-1])
+
+
+def test_duplicate_levels_pick_the_smallest_code():
+    alpha = np.array([1.0, 1.0], dtype=np.float32)  # codes 1 and 2 both give level 0
+    codes = oracle.mbq_assign_nearest(np.array([0.0, 0.1, -0.1, 0.9], dtype=np.float32), alpha)
+    assert codes.tolist() == [1, 1, 1, 1]
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 4])
+def test_alpha_update_is_least_squares_plus_moving_average(k):
+    """Eq. 3 against numpy's least squares, Eq. 4 with beta = min(0.9, (1+t)/(10+t))."""
+    x = workloads.random_tensor(20000, 7, "normal")
+    alpha_prev = np.array([0.8, 0.45, 0.25, 0.12][:k], dtype=np.float32)
+    codes = oracle.mbq_assign_nearest(x, alpha_prev)
+    B = signs(codes, k)
+    cur = np.linalg.lstsq(B, x.astype(np.float64), rcond=None)[0]
+    for t, beta in [(0, 0.1), (1, 2 / 11), (8, 0.5), (80, 0.9), (1000, 0.9)]:
+        want = beta * alpha_prev.astype(np.float64) + (1 - beta) * cur
+        got = oracle.mbq_update_alpha(x, codes, alpha_prev, t)
+        assert np.allclose(got, want, rtol=2e-7, atol=0)
+
+
+def test_singular_gram_matrix_keeps_alpha():
+    x = np.abs(workloads.random_tensor(512, 3, "normal")) + 10  # far above every level: all signs +1
+    alpha_prev = np.array([1.0, 0.5], dtype=np.float32)
+    codes = oracle.mbq_assign_nearest(x, alpha_prev)
+    assert np.all(codes == 3)
+    assert np.array_equal(oracle.mbq_update_alpha(x, codes, alpha_prev, 5), alpha_prev)
+
+
+@pytest.mark.parametrize("k", [2, 3, 4])
+def test_exact_recovery_when_the_data_lies_on_the_levels(k):
+    """x drawn from P: the signs are recovered, least squares returns alpha, no error, no bias."""
+    alpha = np.array([2.0, 1.0, 0.5, 0.25][:k], dtype=np.float32)  # sums are exact in fp32
+    rng = np.random.default_rng(5)
+    true_codes = rng.integers(0, 1 << k, 4096).astype(np.uint8)
+    x = oracle.mbq_levels(alpha)[true_codes]
+    codes = oracle.mbq_assign_nearest(x, alpha)
+    assert np.array_equal(codes, true_codes)
+    assert np.array_equal(oracle.mbq_update_alpha(x, codes, alpha, 3), alpha)
+    assert oracle.mbq_bias(x, codes, alpha) == 0.0
+    stream, nxt = oracle.mbq_compress(x, k, 3, False, alpha)
+    assert np.array_equal(nxt, alpha) and np.array_equal(oracle.mbq_decompress(stream, x.size), x)
+
+
+def test_bias_is_the_mean_quantization_error():
+    """Eq. 5: m_q = E[x_hat - x]; subtracting it makes the reconstruction's mean equal the data's."""
+    x = workloads.generate("cfg1_act", 0, 1 << 15)  # post-ReLU: strongly biased under symmetric levels
+    alpha = np.array([0.6, 0.3], dtype=np.float32)
+    codes = oracle.mbq_assign_nearest(x, alpha)
+    want = (signs(codes, 2) @ alpha.astype(np.float64) - x.astype(np.float64)).mean()
+    assert abs(oracle.mbq_bias(x, codes, alpha) - want) <= 1e-7 * max(1.0, abs(want))
+    stream, nxt = oracle.mbq_compress(x, 2, 4, False, alpha)
+    xhat = oracle.mbq_decompress(stream, x.size)
+    assert abs(xhat.astype(np.float64).mean() - x.astype(np.float64).mean()) < 1e-6
+    lv = oracle.mbq_levels(nxt).astype(np.float64)
+    m_q = float(stream[32 + 8:32 + 12].view(np.float32)[0])
+    assert set(np.unique(xhat)).issubset({np.float32(np.float32(v) - np.float32(m_q)) for v in oracle.mbq_levels(nxt)})
+    assert lv.size == 4
+
+
+def test_residue_initialisation():
+    """k = 1 is the closed form (sign, mean |x|); more bases never increase the residual energy."""
+    x = workloads.random_tensor(10000, 9, "normal")
+    codes, a = oracle.mbq_assign_residue(x, 1)
+    assert np.array_equal(codes, (x >= 0).astype(np.uint8))
+    assert abs(a[0] - np.abs(x.astype(np.float64)).mean()) < 1e-7
+    prev = None
+    for k in (1, 2, 3, 4):
+        codes, a = oracle.mbq_assign_residue(x, k)
+        err = np.linalg.norm(signs(codes, k) @ a.astype(np.float64) - x)
+        assert prev is None or err < prev
+        assert np.all(np.diff(a) < 0) and np.all(a > 0)
+        prev = err
+    # first basis and coefficient do not depend on k
+    assert np.array_equal(codes & 1, (x >= 0).astype(np.uint8))
+
+
+@pytest.mark.parametrize("k", [2, 3, 4])
+def test_stream_layout_and_size(k):
+    """Side words: alpha (k floats) and m_q, the 32(k+1) bits of Eq. 8; payload k bits per element as planes."""
+    n = 1000
+    x = workloads.random_tensor(n, k, "normal")
+    stream, alpha = oracle.mbq_compress(x, k, 0, True)
+    assert stream.size == oracle.mbq_stream_bytes(n, k) == -(-(32 + 4 * (k + 1)) // 16) * 16 + 4 * k * 32
+    hdr = stream[:32].view(np.uint32)
+    assert [int(v) for v in hdr] == [0x54504341, 1, n, 0, 0, k, 0, 1]
+    assert np.array_equal(stream[32:32 + 4 * k].view(np.float32), alpha)
+    codes, _ = oracle.mbq_assign_residue(x, k)
+    payload = stream[oracle.mbq_payload_offset(k):].view(np.uint32)
+    for i in (0, 1, 31, 32, 500, 999):
+        got = sum(((int(payload[(i // 32) * k + j]) >> (i % 32)) & 1) << j for j in range(k))
+        assert got == int(codes[i])
+    # the paper's table: largest MobileNetV2 output, 4096 KB -> 256/384/512 KB of planes (+ framing)
+    big = 4096 * 1024 // 4
+    assert oracle.mbq_stream_bytes(big, k) - oracle.mbq_payload_offset(k) == big * k // 8
+    assert abs(4 * big / oracle.mbq_stream_bytes(big, k) - 32 / k) < 1e-3 * 32 / k
+
+
+def test_alternating_updates_reduce_the_error():
+    """A few batches of the same data: nearest assignment + least squares never increases the error much
+    and ends below the residue initialisation (the alternating scheme the paper follows)."""
+    x = workloads.generate("cfg1_act", 0, 1 << 15)
+    k = 3
+    stream, alpha = oracle.mbq_compress(x, k, 0, True)
+    e0 = np.linalg.norm(oracle.mbq_decompress(stream, x.size) - x)
+    for t in range(1, 30):
+        stream, alpha = oracle.mbq_compress(x, k, t, False, alpha)
+    e1 = np.linalg.norm(oracle.mbq_decompress(stream, x.size) - x)
+    assert e1 < e0
