@@ -191,6 +191,51 @@ accept_status accept_decompress_host(const accept_params* p, const void* h_strea
                                      float* d_xhat, void* d_ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * ---------------------------------------------------------------------------------------------
+ * Forward quantizer of the paper: multi-bit quantization (Sec. 3.3 "Forward Quantizer", Eq. 1-5;
+ * "Forward Encoder"; Sec. 3.4 "Forward Decoder", "Forward Dequantizer").
+ *
+ * x ~ B alpha, B in {-1,+1}^(N x k), alpha in R^k (one alpha per tensor, as in the paper).  Element
+ * i carries the code c_i = sum_j [b_ij = +1] << j; level(c) = (+-alpha_0) + ... + (+-alpha_k-1)
+ * summed in fp32 in the order j = 0..k-1.
+ *   batch_index t >= 1 (init = 0): every value takes the nearest level of alpha_prev (exact
+ *     comparison; a tie goes to the lower level; coinciding levels: the smallest code), then
+ *     alpha_cur = (B^T B)^-1 B^T x (Eq. 3; kept at alpha_prev if B^T B is singular) and
+ *     alpha_next = beta alpha_prev + (1-beta) alpha_cur, beta = min(0.9, (1+t)/(10+t)) (Eq. 4).
+ *   init != 0 (batch 0 of an epoch): residue method: r = x; for j = 0..k-1: b_j = [r >= 0],
+ *     alpha_j = mean |r|, r <- r - alpha_j b_j; alpha_prev is not read; no Eq. 3/4 update.
+ *   The stream carries alpha_next and m_q = mean(B alpha_next - x) (Eq. 5); the receiver
+ *     computes xhat = level(c) - m_q.  Sums run in double in a fixed order (results repeat from
+ *     run to run; against another summation order alpha_next and m_q may differ in the last fp32
+ *     bit).  Non-finite input is not supported: ACCEPT_DEV_NONFINITE is set, codes are unspecified.
+ * Stream: [0,32) header (magic, version, n low, n high, 0, k, 0, 1), [32, 32+4k) alpha_next,
+ *   then m_q, zero pad to a multiple of 16, then bit planes: group g of 32 elements owns words
+ *   g*k .. g*k+k-1, bit t of word g*k+j = [b_(32g+t),j = +1] ("-1 replaced by 0").
+ * k in {2,3,4} (the paper's forward range); d_alpha_prev / d_alpha_next are DEVICE arrays of k
+ * floats (they may be the same array), so successive batches chain without a host round trip.
+ * The workspace (accept_mbq_workspace_size bytes, 16-byte aligned, zeroed once by the caller) holds
+ * the status word and per-block partial sums.  Launches: 2 (plus 2k when init).
+ */
+typedef struct {
+  uint64_t n_elems;
+  uint32_t k;
+  uint32_t batch_index; /* t of Eq. 4 */
+  uint32_t init;        /* 1: residue-based initialisation */
+  uint32_t reserved;    /* must be 0 */
+} accept_mbq_params;
+
+accept_status accept_mbq_check_params(const accept_mbq_params* p);
+size_t accept_mbq_compressed_size(const accept_mbq_params* p); /* 0 if p is invalid */
+size_t accept_mbq_payload_offset(const accept_mbq_params* p);
+size_t accept_mbq_workspace_size(const accept_mbq_params* p);
+accept_status accept_mbq_compress(const accept_mbq_params* p, const float* d_x, const float* d_alpha_prev,
+                                  float* d_alpha_next, void* d_stream, size_t stream_bytes, void* d_ws,
+                                  size_t ws_bytes, void* cuda_stream);
+/* Reads k and n from p; the kernel checks them against the header (ACCEPT_DEV_BAD_HEADER). */
+accept_status accept_mbq_decompress(const accept_mbq_params* p, const void* d_stream, size_t stream_bytes,
+                                    float* d_xhat, void* d_ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * Synchronises cuda_stream, copies the status word to the host and returns it in *status_bits
  * (ACCEPT_DEV_* bits).  Returns ACCEPT_ERR_CUDA if the stream reports an error.
  */

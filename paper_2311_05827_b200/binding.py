@@ -33,6 +33,8 @@ EXPORTS = [
     "accept_compress", "accept_decompress", "accept_compress_host", "accept_decompress_host",
     "accept_last_device_status", "accept_parse_header", "accept_bitwidth_schedule", "accept_launch_count",
     "accept_compress_static",
+    "accept_mbq_check_params", "accept_mbq_compressed_size", "accept_mbq_payload_offset", "accept_mbq_workspace_size",
+    "accept_mbq_compress", "accept_mbq_decompress",
 ]
 
 
@@ -62,6 +64,22 @@ class Params:
     def c(self) -> CParams:
         return CParams(self.n_elems, self.chunk_elems, self.k, self.range, self.round, self.layout, 0,
                        self.seed & (2**64 - 1), self.rng_offset & (2**64 - 1))
+
+
+class CMbqParams(ctypes.Structure):
+    _fields_ = [("n_elems", ctypes.c_uint64), ("k", ctypes.c_uint32), ("batch_index", ctypes.c_uint32),
+                ("init", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+
+
+@dataclass(frozen=True)
+class MbqParams:
+    n_elems: int
+    k: int
+    batch_index: int = 0
+    init: bool = False
+
+    def c(self) -> CMbqParams:
+        return CMbqParams(self.n_elems, self.k, self.batch_index, 1 if self.init else 0, 0)
 
 
 _lib = None
@@ -97,6 +115,16 @@ def lib() -> ctypes.CDLL:
     L.accept_bitwidth_schedule.argtypes = [ctypes.c_int, ctypes.c_int]
     L.accept_compress_static.restype = ctypes.c_int
     L.accept_compress_static.argtypes = [P, vp, vp, sz, vp, vp]
+    MP = ctypes.POINTER(CMbqParams)
+    L.accept_mbq_check_params.restype = ctypes.c_int
+    L.accept_mbq_check_params.argtypes = [MP]
+    for name in ("accept_mbq_compressed_size", "accept_mbq_payload_offset", "accept_mbq_workspace_size"):
+        getattr(L, name).restype = sz
+        getattr(L, name).argtypes = [MP]
+    L.accept_mbq_compress.restype = ctypes.c_int
+    L.accept_mbq_compress.argtypes = [MP, vp, vp, vp, vp, sz, vp, sz, vp]
+    L.accept_mbq_decompress.restype = ctypes.c_int
+    L.accept_mbq_decompress.argtypes = [MP, vp, sz, vp, vp, sz, vp]
     L.accept_launch_count.restype = u64
     L.accept_launch_count.argtypes = []
     _lib = L
@@ -195,13 +223,49 @@ def accept_last_device_status(d_ws, stream=None) -> int:
     return int(bits.value)
 
 
+# ---- multi-bit quantization (forward path) ----------------------------------------------------
+
+def accept_mbq_check_params(p: MbqParams) -> int:
+    return int(lib().accept_mbq_check_params(ctypes.byref(p.c())))
+
+
+def accept_mbq_compressed_size(p: MbqParams) -> int:
+    return int(lib().accept_mbq_compressed_size(ctypes.byref(p.c())))
+
+
+def accept_mbq_payload_offset(p: MbqParams) -> int:
+    return int(lib().accept_mbq_payload_offset(ctypes.byref(p.c())))
+
+
+def accept_mbq_workspace_size(p: MbqParams) -> int:
+    return int(lib().accept_mbq_workspace_size(ctypes.byref(p.c())))
+
+
+def accept_mbq_compress(p: MbqParams, d_x, d_alpha_prev, d_alpha_next, d_stream, d_ws, stream=None) -> None:
+    """d_alpha_prev (may be None when p.init) and d_alpha_next: float32 CUDA tensors of k elements."""
+    _check(lib().accept_mbq_compress(ctypes.byref(p.c()), d_x.data_ptr(),
+                                     None if d_alpha_prev is None else d_alpha_prev.data_ptr(),
+                                     d_alpha_next.data_ptr(), d_stream.data_ptr(),
+                                     d_stream.numel() * d_stream.element_size(), d_ws.data_ptr(),
+                                     d_ws.numel() * d_ws.element_size(), _stream_handle(stream)), "accept_mbq_compress")
+
+
+def accept_mbq_decompress(p: MbqParams, d_stream, d_xhat, d_ws, stream=None) -> None:
+    _check(lib().accept_mbq_decompress(ctypes.byref(p.c()), d_stream.data_ptr(),
+                                       d_stream.numel() * d_stream.element_size(), d_xhat.data_ptr(),
+                                       d_ws.data_ptr(), d_ws.numel() * d_ws.element_size(),
+                                       _stream_handle(stream)), "accept_mbq_decompress")
+
+
 # ---- small conveniences for callers (allocation only) -----------------------------------------
 
-def new_stream_buffer(p: Params, device="cuda"):
+def new_stream_buffer(p, device="cuda"):
     import torch
-    return torch.empty(accept_compressed_size(p), dtype=torch.uint8, device=device)
+    size = accept_mbq_compressed_size(p) if isinstance(p, MbqParams) else accept_compressed_size(p)
+    return torch.empty(size, dtype=torch.uint8, device=device)
 
 
-def new_workspace(p: Params, device="cuda"):
+def new_workspace(p, device="cuda"):
     import torch
-    return torch.zeros(accept_workspace_size(p) // 4, dtype=torch.int32, device=device)
+    size = accept_mbq_workspace_size(p) if isinstance(p, MbqParams) else accept_workspace_size(p)
+    return torch.zeros((size + 3) // 4, dtype=torch.int32, device=device)

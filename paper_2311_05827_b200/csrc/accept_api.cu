@@ -9,6 +9,7 @@
 
 #include "accept_kernels.cuh"
 #include "accept_wide.cuh"
+#include "accept_mbq.cuh"
 
 namespace {
 
@@ -168,6 +169,46 @@ accept_status launch_wide(const accept_params* p, const CodecArgs& a, uint8_t* r
   }
   g_launches.fetch_add(3, std::memory_order_relaxed);
   return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+}
+
+// ---- multi-bit quantization --------------------------------------------------------------------
+
+uint32_t mbq_blocks(const accept_mbq_params* p) {
+  return (uint32_t)((p->n_elems + accept::kMbqTile - 1) / accept::kMbqTile);
+}
+
+accept::MbqArgs mbq_args(const accept_mbq_params* p, void* d_stream, void* d_ws) {
+  accept::MbqArgs a{};
+  uint8_t* base = static_cast<uint8_t*>(d_stream);
+  uint8_t* ws = static_cast<uint8_t*>(d_ws);
+  a.header = reinterpret_cast<uint32_t*>(base);
+  a.side = reinterpret_cast<float*>(base + ACCEPT_HEADER_BYTES);
+  a.payload = reinterpret_cast<uint32_t*>(base + accept_mbq_payload_offset(p));
+  a.status = reinterpret_cast<uint32_t*>(ws);
+  a.alpha_init = reinterpret_cast<float*>(ws + 16);
+  a.n = p->n_elems;
+  a.n_blocks = mbq_blocks(p);
+  a.partial = reinterpret_cast<accept::MbqPartial*>(ws + 64);
+  a.residue_sum = reinterpret_cast<double*>(ws + 64 + (size_t)accept::kMbqPartialBytes * a.n_blocks);
+  a.k = p->k;
+  a.batch_index = p->batch_index;
+  a.init = p->init ? 1u : 0u;
+  return a;
+}
+
+template <int K>
+void launch_mbq_compress(const accept::MbqArgs& a, cudaStream_t s) {
+  if (a.init) {
+    for (int j = 0; j < K; ++j) {
+      accept::mbq_residue_sum_kernel<K><<<a.n_blocks, 256, 0, s>>>(a, j);
+      accept::mbq_residue_finalize_kernel<<<1, 256, 0, s>>>(a, j);
+    }
+    accept::mbq_encode_kernel<K, true><<<a.n_blocks, 256, 0, s>>>(a);
+  } else {
+    accept::mbq_encode_kernel<K, false><<<a.n_blocks, 256, 0, s>>>(a);
+  }
+  accept::mbq_finalize_kernel<K><<<1, 256, 0, s>>>(a);
+  g_launches.fetch_add(2 + (a.init ? 2 * K : 0), std::memory_order_relaxed);
 }
 
 // ---- built-in scratch for accept_compress_static ------------------------------------------------
@@ -354,6 +395,74 @@ int accept_bitwidth_schedule(int is_backward, int n_lr_changes) {
   if (n_lr_changes < 0) n_lr_changes = 0;
   if (is_backward) return n_lr_changes == 0 ? 8 : 4;
   return n_lr_changes >= 2 ? 4 : 2 + n_lr_changes;
+}
+
+accept_status accept_mbq_check_params(const accept_mbq_params* p) {
+  if (!p) return ACCEPT_ERR_NULL;
+  if (p->n_elems == 0 || p->n_elems / accept::kMbqTile > 0x7ffffff0ull) return ACCEPT_ERR_BAD_SIZE;
+  if (p->k < 2 || p->k > 4) return ACCEPT_ERR_BAD_K;
+  if (p->reserved != 0 || p->init > 1) return ACCEPT_ERR_BAD_ENUM;
+  return ACCEPT_OK;
+}
+
+size_t accept_mbq_payload_offset(const accept_mbq_params* p) {
+  if (accept_mbq_check_params(p) != ACCEPT_OK) return 0;
+  return (ACCEPT_HEADER_BYTES + 4 * (size_t)(p->k + 1) + 15) / 16 * 16;
+}
+
+size_t accept_mbq_compressed_size(const accept_mbq_params* p) {
+  if (accept_mbq_check_params(p) != ACCEPT_OK) return 0;
+  return accept_mbq_payload_offset(p) + (size_t)(4ull * p->k * ((p->n_elems + 31) / 32));
+}
+
+size_t accept_mbq_workspace_size(const accept_mbq_params* p) {
+  if (accept_mbq_check_params(p) != ACCEPT_OK) return 0;
+  // status + residue coefficients (64 bytes), one 128-byte record and one double per block
+  return 64 + (size_t)(accept::kMbqPartialBytes + 8) * mbq_blocks(p);
+}
+
+accept_status accept_mbq_compress(const accept_mbq_params* p, const float* d_x, const float* d_alpha_prev,
+                                  float* d_alpha_next, void* d_stream, size_t stream_bytes, void* d_ws,
+                                  size_t ws_bytes, void* cuda_stream) {
+  if (!p || !d_x || !d_alpha_next || !d_stream || !d_ws) return ACCEPT_ERR_NULL;
+  accept_status st = accept_mbq_check_params(p);
+  if (st != ACCEPT_OK) return st;
+  if (!p->init && !d_alpha_prev) return ACCEPT_ERR_NULL;
+  if (stream_bytes < accept_mbq_compressed_size(p) || ws_bytes < accept_mbq_workspace_size(p)) return ACCEPT_ERR_TOO_SMALL;
+  if (!is_aligned(d_x, 32) || !is_aligned(d_stream, 16) || !is_aligned(d_ws, 16) || !is_aligned(d_alpha_next, 4) ||
+      !is_aligned(d_alpha_prev, 4))
+    return ACCEPT_ERR_MISALIGNED;
+  accept::MbqArgs a = mbq_args(p, d_stream, d_ws);
+  a.x = d_x;
+  a.alpha_prev = d_alpha_prev;
+  a.alpha_next = d_alpha_next;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  switch (p->k) {
+    case 2: launch_mbq_compress<2>(a, s); break;
+    case 3: launch_mbq_compress<3>(a, s); break;
+    default: launch_mbq_compress<4>(a, s); break;
+  }
+  return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+}
+
+accept_status accept_mbq_decompress(const accept_mbq_params* p, const void* d_stream, size_t stream_bytes,
+                                    float* d_xhat, void* d_ws, size_t ws_bytes, void* cuda_stream) {
+  if (!p || !d_stream || !d_xhat || !d_ws) return ACCEPT_ERR_NULL;
+  accept_status st = accept_mbq_check_params(p);
+  if (st != ACCEPT_OK) return st;
+  if (stream_bytes < accept_mbq_compressed_size(p) || ws_bytes < 16) return ACCEPT_ERR_TOO_SMALL;
+  if (!is_aligned(d_xhat, 32) || !is_aligned(d_stream, 16) || !is_aligned(d_ws, 4)) return ACCEPT_ERR_MISALIGNED;
+  accept::MbqArgs a = mbq_args(p, const_cast<void*>(d_stream), d_ws);
+  a.xhat = d_xhat;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const unsigned grid = (unsigned)((p->n_elems + 4095) / 4096);
+  switch (p->k) {
+    case 2: accept::mbq_decode_kernel<2><<<grid, 256, 0, s>>>(a); break;
+    case 3: accept::mbq_decode_kernel<3><<<grid, 256, 0, s>>>(a); break;
+    default: accept::mbq_decode_kernel<4><<<grid, 256, 0, s>>>(a); break;
+  }
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
 }
 
 uint64_t accept_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -1,0 +1,453 @@
+// Forward quantizer of the paper: multi-bit quantization (Sec. 3.3 "Forward Quantizer", Eq. 1-5),
+// "Forward Encoder" (bit planes, -1 stored as 0) and the receiver (Sec. 3.4 "Forward Decoder",
+// "Forward Dequantizer").
+//
+// Element i carries k signs b_i0..b_i,k-1 as the code c_i = sum_j [b_ij = +1] << j; plane j of a
+// 32-element group is basis j.  level(c) = (+-alpha_0) + ... + (+-alpha_k-1), summed in fp32 in
+// the order j = 0..k-1.  One pass over the input assigns the signs, writes the planes and gathers
+// per block what Eq. 3-5 need: counts of +1 per basis, counts of differing signs per pair of bases
+// (integers: B^T B exactly), sum of x over the +1 elements of each basis and sum of x (double).
+// A single small block then adds the per-block partials in a fixed order, solves the k x k system,
+// applies the moving average and writes the side words.  Sums are order-fixed, so results repeat
+// from run to run.
+#pragma once
+#include "accept_kernels.cuh"
+
+namespace accept {
+
+constexpr int kMbqRounds = 4;                      // octets per thread
+constexpr int kMbqTile = kMbqRounds * 256 * 8;     // elements per block
+constexpr int kMbqPartialBytes = 128;              // per-block record in the workspace
+
+// Per-block partial sums (one 128-byte record per block of the encode pass).
+struct MbqPartial {
+  double plus[4];     // sum of x over the elements whose basis j is +1
+  double sum_x;       // sum of x
+  uint32_t count[4];  // number of +1 per basis
+  uint32_t differ[6]; // pairs (0,1) (0,2) (0,3) (1,2) (1,3) (2,3): elements whose two signs differ
+  uint32_t pad[12];
+};
+static_assert(sizeof(MbqPartial) == kMbqPartialBytes, "record size");
+
+struct MbqArgs {
+  const float* x;
+  float* xhat;
+  const float* alpha_prev;  // device, k floats (unused when init)
+  float* alpha_next;        // device, k floats
+  uint32_t* header;         // stream + 0
+  float* side;              // stream + 32: alpha (k floats), m_q
+  uint32_t* payload;
+  uint32_t* status;
+  MbqPartial* partial;      // workspace + 64
+  float* alpha_init;        // workspace + 16: coefficients found by the residue passes (init)
+  double* residue_sum;      // workspace + 32: scratch of the residue passes
+  uint64_t n;
+  uint32_t n_blocks;
+  uint32_t k, batch_index, init;
+};
+
+__device__ __forceinline__ uint32_t mbq_header_word(const MbqArgs& a, int i) {
+  switch (i) {
+    case 0: return 0x54504341u;
+    case 1: return 1u;
+    case 2: return (uint32_t)a.n;
+    case 3: return (uint32_t)(a.n >> 32);
+    case 5: return a.k;
+    case 7: return 1u;  // stream kind: multi-bit quantization
+    default: return 0u;
+  }
+}
+
+// level(c) for the coefficients in alpha[0..K)
+template <int K>
+__device__ __forceinline__ float mbq_level(const float* alpha, uint32_t c) {
+  float v = 0.0f;
+#pragma unroll
+  for (int j = 0; j < K; ++j) {
+    const float term = ((c >> j) & 1u) ? alpha[j] : -alpha[j];
+    v = (j == 0) ? term : __fadd_rn(v, term);
+  }
+  return v;
+}
+
+// Search table for the nearest level: thresholds between neighbouring sorted levels and the code
+// of each sorted position.  A threshold is the midpoint rounded DOWN to fp32: for an fp32 x,
+// "x > threshold" is then exactly "x is above the true midpoint" (a tie goes to the lower level).
+// Positions whose levels coincide all map to the smallest code among them.
+template <int K>
+struct MbqTable {
+  float thr[1 << K];     // thr[i], i >= 1: between sorted positions i-1 and i; thr[0] unused
+  uint32_t code[1 << K];
+};
+
+template <int K>
+__device__ void mbq_build_table(const float* alpha_global, MbqTable<K>* t, float* s_level, int tid) {
+  constexpr int L = 1 << K;
+  __shared__ float s_sorted[16];
+  float alpha[K];
+#pragma unroll
+  for (int j = 0; j < K; ++j) alpha[j] = __ldg(alpha_global + j);
+  if (tid < L) s_level[tid] = mbq_level<K>(alpha, tid);
+  __syncthreads();
+  if (tid < L) {
+    const float mine = s_level[tid];
+    int rank = 0;
+    uint32_t first = tid;
+    for (int d = 0; d < L; ++d) {
+      const float other = s_level[d];
+      rank += (other < mine || (other == mine && d < tid)) ? 1 : 0;
+      if (other == mine && (uint32_t)d < first) first = d;
+    }
+    s_sorted[rank] = mine;
+    t->code[rank] = first;
+  }
+  __syncthreads();
+  if (tid >= 1 && tid < L) t->thr[tid] = __fmul_rn(__fadd_rd(s_sorted[tid - 1], s_sorted[tid]), 0.5f);
+  if (tid == 0) t->thr[0] = 0.0f;
+  __syncthreads();
+}
+
+template <int K>
+__device__ __forceinline__ uint32_t mbq_nearest_code(const MbqTable<K>& t, float x) {
+  constexpr int L = 1 << K;
+  int idx = 0;
+#pragma unroll
+  for (int step = L / 2; step >= 1; step >>= 1)
+    if (x > t.thr[idx + step]) idx += step;
+  return t.code[idx];
+}
+
+// Signs of the successive residues with the given coefficients (residue method): bit j = [r_j >= 0].
+// Returns the residue after `upto` steps in *residue.
+template <int K>
+__device__ __forceinline__ uint32_t mbq_residue_code(const float (&alpha)[K], float x, int upto, float* residue) {
+  float r = x;
+  uint32_t c = 0;
+#pragma unroll
+  for (int j = 0; j < K; ++j) {
+    if (j < upto) {
+      if (r >= 0.0f) { c |= 1u << j; r = __fsub_rn(r, alpha[j]); }
+      else r = __fadd_rn(r, alpha[j]);
+    }
+  }
+  *residue = r;
+  return c;
+}
+
+__device__ __forceinline__ void mbq_ld_octet(const float* x, uint64_t n, uint64_t oct, float (&v)[8]) {
+  const uint64_t e = oct * 8;
+  if (e + 8 <= n) {
+    ld_octet(x + e, v);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = (e + i < n) ? __ldg(x + e + i) : 0.0f;
+  }
+}
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+  return v;
+}
+
+// Residue method, step j: per-block sum of |r_j| (r_0 = x) with the coefficients found so far.
+template <int K>
+__global__ void __launch_bounds__(256) mbq_residue_sum_kernel(const MbqArgs a, int j) {
+  __shared__ double s_part[8];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float alpha[K];
+#pragma unroll
+  for (int i = 0; i < K; ++i) alpha[i] = (i < j) ? a.alpha_init[i] : 0.0f;
+  const uint64_t n_oct = (a.n + 7) / 8;
+  double acc = 0.0;
+#pragma unroll
+  for (int r = 0; r < kMbqRounds; ++r) {
+    const uint64_t oct = (uint64_t)blockIdx.x * (kMbqRounds * 256) + r * 256 + tid;
+    if (oct < n_oct) {
+      float v[8];
+      mbq_ld_octet(a.x, a.n, oct, v);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        float res;
+        mbq_residue_code<K>(alpha, v[e], j, &res);
+        if (oct * 8 + e < a.n) acc += (double)fabsf(res);
+      }
+    }
+  }
+  acc = warp_sum(acc);
+  if (lane == 0) s_part[warp] = acc;
+  __syncthreads();
+  if (tid == 0) {
+    double s = 0.0;
+    for (int w = 0; w < 8; ++w) s += s_part[w];
+    a.residue_sum[blockIdx.x] = s;
+  }
+}
+
+// Residue method, step j: alpha_j = mean |r_j| (block partials added in index order).
+__global__ void __launch_bounds__(256) mbq_residue_finalize_kernel(const MbqArgs a, int j) {
+  __shared__ double s_part[256];
+  const int tid = threadIdx.x;
+  double s = 0.0;
+  for (uint32_t b = tid; b < a.n_blocks; b += 256) s += a.residue_sum[b];
+  s_part[tid] = s;
+  __syncthreads();
+  if (tid == 0) {
+    double total = 0.0;
+    for (int i = 0; i < 256; ++i) total += s_part[i];
+    a.alpha_init[j] = (float)(total / (double)a.n);
+  }
+}
+
+// Assign the signs, write the planes, gather the per-block sums.
+template <int K, bool INIT>
+__global__ void __launch_bounds__(256) mbq_encode_kernel(const MbqArgs a) {
+  __shared__ MbqTable<K> s_table;
+  __shared__ float s_level[16];
+  __shared__ double s_dbl[8][K + 1];
+  __shared__ uint32_t s_cnt[10];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float alpha[K];
+  if (INIT) {
+#pragma unroll
+    for (int j = 0; j < K; ++j) alpha[j] = a.alpha_init[j];
+  } else {
+#pragma unroll
+    for (int j = 0; j < K; ++j) alpha[j] = 0.0f;
+    mbq_build_table<K>(a.alpha_prev, &s_table, s_level, tid);
+  }
+  if (tid < 10) s_cnt[tid] = 0;
+  __syncthreads();
+
+  const uint64_t n_oct = (a.n + 7) / 8;
+  const uint64_t n_oct_stored = ((a.n + 31) / 32) * 4;
+  double plus[K], sum_x = 0.0;
+  uint32_t count[K], differ[6];
+#pragma unroll
+  for (int j = 0; j < K; ++j) { plus[j] = 0.0; count[j] = 0; }
+#pragma unroll
+  for (int p = 0; p < 6; ++p) differ[p] = 0;
+
+  float v[kMbqRounds][8];
+#pragma unroll
+  for (int r = 0; r < kMbqRounds; ++r) {
+    const uint64_t oct = (uint64_t)blockIdx.x * (kMbqRounds * 256) + r * 256 + tid;
+    if (oct < n_oct) {
+      mbq_ld_octet(a.x, a.n, oct, v[r]);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[r][e] = 0.0f;
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < kMbqRounds; ++r) {
+    const uint64_t oct = (uint64_t)blockIdx.x * (kMbqRounds * 256) + r * 256 + tid;
+    uint32_t xlo = 0, xhi = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      uint32_t c = 0;
+      if (oct * 8 + e < a.n) {
+        if (INIT) {
+          float res;
+          c = mbq_residue_code<K>(alpha, v[r][e], K, &res);
+        } else {
+          c = mbq_nearest_code<K>(s_table, v[r][e]);
+        }
+        const double xd = (double)v[r][e];
+        sum_x += xd;
+#pragma unroll
+        for (int j = 0; j < K; ++j)
+          if ((c >> j) & 1u) plus[j] += xd;
+      }
+      if (e < 4) xlo |= c << (8 * e);
+      else xhi |= c << (8 * (e - 4));
+    }
+    // plane form: byte j = the eight signs of basis j
+    const uint32_t planes = planes_nibbles(merge_nibbles(xlo, xhi));
+#pragma unroll
+    for (int j = 0; j < K; ++j) count[j] += __popc((planes >> (8 * j)) & 0xFFu);
+    {
+      int p = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = i + 1; j < 4; ++j, ++p)
+          if (j < K) differ[p] += __popc(((planes >> (8 * i)) ^ (planes >> (8 * j))) & 0xFFu);
+    }
+    const bool stored = oct < n_oct_stored;
+    const uint32_t any = __ballot_sync(0xffffffffu, stored);
+    if (any) store_bitplane_guarded<K>(a.payload, oct >> 2, xlo, xhi, lane, stored);
+  }
+
+  // block sums in a fixed order: lanes by butterfly, warps one after the other
+#pragma unroll
+  for (int j = 0; j < K; ++j) {
+    const double s = warp_sum(plus[j]);
+    if (lane == 0) s_dbl[warp][j] = s;
+    const uint32_t c = __reduce_add_sync(0xffffffffu, count[j]);
+    if (lane == 0) atomicAdd(&s_cnt[j], c);
+  }
+  {
+    const double s = warp_sum(sum_x);
+    if (lane == 0) s_dbl[warp][K] = s;
+  }
+#pragma unroll
+  for (int p = 0; p < 6; ++p) {
+    const uint32_t c = __reduce_add_sync(0xffffffffu, differ[p]);
+    if (lane == 0) atomicAdd(&s_cnt[4 + p], c);
+  }
+  __syncthreads();
+  if (tid == 0) {
+    MbqPartial out;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { out.plus[j] = 0.0; out.count[j] = 0; }
+    for (int j = 0; j < K; ++j) {
+      double s = 0.0;
+      for (int w = 0; w < 8; ++w) s += s_dbl[w][j];
+      out.plus[j] = s;
+      out.count[j] = s_cnt[j];
+    }
+    double s = 0.0;
+    for (int w = 0; w < 8; ++w) s += s_dbl[w][K];
+    out.sum_x = s;
+    for (int p = 0; p < 6; ++p) out.differ[p] = s_cnt[4 + p];
+    for (int p = 0; p < 12; ++p) out.pad[p] = 0;
+    a.partial[blockIdx.x] = out;
+  }
+}
+
+// Adds the per-block partials (fixed order), then Eq. 3 (least squares by Gaussian elimination with
+// partial pivoting, in double), Eq. 4 (moving average), Eq. 5 (bias), and writes header, side
+// words and alpha_next.  One block.
+template <int K>
+__global__ void __launch_bounds__(256) mbq_finalize_kernel(const MbqArgs a) {
+  __shared__ double s_dbl[256][K + 1];
+  __shared__ unsigned long long s_int[256][10];
+  const int tid = threadIdx.x;
+  double d[K + 1];
+  unsigned long long c[10];
+#pragma unroll
+  for (int j = 0; j <= K; ++j) d[j] = 0.0;
+#pragma unroll
+  for (int j = 0; j < 10; ++j) c[j] = 0;
+  for (uint32_t b = tid; b < a.n_blocks; b += 256) {
+    const MbqPartial& p = a.partial[b];
+#pragma unroll
+    for (int j = 0; j < K; ++j) { d[j] += p.plus[j]; c[j] += p.count[j]; }
+    d[K] += p.sum_x;
+#pragma unroll
+    for (int j = 0; j < 6; ++j) c[4 + j] += p.differ[j];
+  }
+#pragma unroll
+  for (int j = 0; j <= K; ++j) s_dbl[tid][j] = d[j];
+#pragma unroll
+  for (int j = 0; j < 10; ++j) s_int[tid][j] = c[j];
+  __syncthreads();
+  if (tid != 0) return;
+#pragma unroll
+  for (int j = 0; j <= K; ++j) d[j] = 0.0;
+#pragma unroll
+  for (int j = 0; j < 10; ++j) c[j] = 0;
+  for (int i = 0; i < 256; ++i) {
+#pragma unroll
+    for (int j = 0; j <= K; ++j) d[j] += s_dbl[i][j];
+#pragma unroll
+    for (int j = 0; j < 10; ++j) c[j] += s_int[i][j];
+  }
+  const double N = (double)a.n, sum_x = d[K];
+  float alpha_next[K];
+  if (a.init) {
+#pragma unroll
+    for (int j = 0; j < K; ++j) alpha_next[j] = a.alpha_init[j];
+  } else {
+    double G[K][K], rhs[K], cur[K], prev[K];
+    int pair = 0;
+    for (int i = 0; i < 4; ++i)
+      for (int j = i + 1; j < 4; ++j, ++pair)
+        if (j < K) G[i][j] = G[j][i] = N - 2.0 * (double)c[4 + pair];
+    for (int j = 0; j < K; ++j) {
+      G[j][j] = N;
+      rhs[j] = 2.0 * d[j] - sum_x;  // sum over +1 minus sum over -1
+      prev[j] = (double)__ldg(a.alpha_prev + j);
+    }
+    bool singular = false;
+    for (int col = 0; col < K && !singular; ++col) {
+      int piv = col;
+      for (int r = col + 1; r < K; ++r)
+        if (fabs(G[r][col]) > fabs(G[piv][col])) piv = r;
+      if (fabs(G[piv][col]) < 1e-9 * N) { singular = true; break; }
+      if (piv != col) {
+        for (int q = 0; q < K; ++q) { const double t = G[col][q]; G[col][q] = G[piv][q]; G[piv][q] = t; }
+        const double t = rhs[col]; rhs[col] = rhs[piv]; rhs[piv] = t;
+      }
+      for (int r = col + 1; r < K; ++r) {
+        const double f = G[r][col] / G[col][col];
+        for (int q = col; q < K; ++q) G[r][q] -= f * G[col][q];
+        rhs[r] -= f * rhs[col];
+      }
+    }
+    if (singular) {
+      for (int j = 0; j < K; ++j) cur[j] = prev[j];
+    } else {
+      for (int col = K - 1; col >= 0; --col) {
+        double s = rhs[col];
+        for (int q = col + 1; q < K; ++q) s -= G[col][q] * cur[q];
+        cur[col] = s / G[col][col];
+      }
+    }
+    double beta = (1.0 + (double)a.batch_index) / (10.0 + (double)a.batch_index);
+    if (beta > 0.9) beta = 0.9;
+    for (int j = 0; j < K; ++j) alpha_next[j] = (float)(beta * prev[j] + (1.0 - beta) * cur[j]);
+  }
+  double acc = 0.0;
+  for (int j = 0; j < K; ++j) acc += (double)alpha_next[j] * (2.0 * (double)c[j] - N);
+  const float m_q = (float)((acc - sum_x) / N);
+  for (int i = 0; i < 8; ++i) a.header[i] = mbq_header_word(a, i);
+  for (int j = 0; j < K; ++j) { a.side[j] = alpha_next[j]; a.alpha_next[j] = alpha_next[j]; }
+  a.side[K] = m_q;
+  // pad up to the payload
+  for (uint32_t* w = reinterpret_cast<uint32_t*>(a.side + K + 1); w < a.payload; ++w) *w = 0u;
+  if (!is_finite_bits((float)sum_x)) atomicOr(a.status, kDevNonFinite);
+}
+
+// Receiver: planes -> codes -> level(c) - m_q.
+template <int K>
+__global__ void __launch_bounds__(256, 8) mbq_decode_kernel(const MbqArgs a) {
+  __shared__ float s_value[1 << K];
+  const int tid = threadIdx.x, lane = tid & 31;
+  if (blockIdx.x == 0 && tid < 8 && a.header[tid] != mbq_header_word(a, tid)) atomicOr(a.status, kDevBadHeader);
+  if (tid < (1 << K)) {
+    float alpha[K];
+#pragma unroll
+    for (int j = 0; j < K; ++j) alpha[j] = __ldg(a.side + j);
+    s_value[tid] = __fsub_rn(mbq_level<K>(alpha, tid), __ldg(a.side + K));
+  }
+  __syncthreads();
+  const uint64_t n_oct = (a.n + 7) / 8, n_groups = (a.n + 31) / 32;
+  const int q = lane & 3;
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const uint64_t oct = (uint64_t)blockIdx.x * 512 + r * 256 + tid;
+    const uint64_t group = oct >> 2;
+    uint32_t w = 0;
+    if (group < n_groups && q < K) w = __ldg(a.payload + group * K + q);
+    const uint32_t nib = planes_nibbles(quad_transpose(w, lane));
+    if (oct < n_oct) {
+      float out[8];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        out[i] = s_value[(nib >> (8 * i)) & 0xFu];
+        out[4 + i] = s_value[(nib >> (8 * i + 4)) & 0xFu];
+      }
+      const uint64_t e = oct * 8;
+      if (e + 8 <= a.n) {
+        st_octet(a.xhat + e, out);
+      } else {
+        for (int i = 0; i < 8; ++i)
+          if (e + i < a.n) a.xhat[e + i] = out[i];
+      }
+    }
+  }
+}
+
+}  // namespace accept

@@ -1,0 +1,138 @@
+"""GPU parity of the forward quantizer (multi-bit quantization) against the oracle, through the C ABI.
+
+Bar: header and bit planes bit-exact (the sign decisions are taken in the same arithmetic on both
+sides); alpha_next and m_q, which come out of long sums whose order differs between the two sides,
+within one fp32 unit in the last place (they are equal in practice: the sums run in double);
+given the same stream, the receiver's output is bit-exact.
+"""
+import numpy as np
+import pytest
+
+import oracle
+import workloads
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+def _A():
+    import paper_2311_05827_b200 as A
+    return A
+
+
+def ulp_close(a, b):
+    a, b = np.asarray(a, dtype=np.float32), np.asarray(b, dtype=np.float32)
+    return np.all(np.abs(a.astype(np.float64) - b.astype(np.float64)) <= np.spacing(np.maximum(np.abs(a), np.abs(b))))
+
+
+def gpu_mbq_compress(x, k, t, init, alpha_prev):
+    A = _A()
+    p = A.MbqParams(x.size, k, t, init)
+    d_x = torch.from_numpy(x).cuda()
+    d_prev = None if alpha_prev is None else torch.from_numpy(np.asarray(alpha_prev, dtype=np.float32)).cuda()
+    d_next = torch.full((k,), float("nan"), dtype=torch.float32, device="cuda")
+    d_stream = A.new_stream_buffer(p)
+    d_stream.fill_(0x77)
+    d_ws = A.new_workspace(p)
+    A.accept_mbq_compress(p, d_x, d_prev, d_next, d_stream, d_ws)
+    status = A.accept_last_device_status(d_ws)
+    return p, d_stream, d_next.cpu().numpy(), status, d_ws
+
+
+def check_mbq(x, k, t, init, alpha_prev):
+    A = _A()
+    ref_stream, ref_alpha = oracle.mbq_compress(x, k, t, init, alpha_prev)
+    p, d_stream, alpha_next, status, d_ws = gpu_mbq_compress(x, k, t, init, alpha_prev)
+    got = d_stream.cpu().numpy()
+    assert status == 0 and got.size == ref_stream.size
+    off = A.accept_mbq_payload_offset(p)
+    assert off == oracle.mbq_payload_offset(k)
+    assert np.array_equal(got[:32], ref_stream[:32]), "header"
+    side_g, side_r = got[32:32 + 4 * (k + 1)].view(np.float32), ref_stream[32:32 + 4 * (k + 1)].view(np.float32)
+    assert ulp_close(side_g, side_r), f"side words {side_g} vs {side_r}"
+    assert np.array_equal(side_g[:k], alpha_next) and ulp_close(alpha_next, ref_alpha)
+    assert np.all(got[32 + 4 * (k + 1):off] == 0), "padding"
+    bad = np.nonzero(got[off:].view(np.uint32) != ref_stream[off:].view(np.uint32))[0]
+    assert bad.size == 0, f"{bad.size} plane words differ, first {bad[:5]}"
+    # receiver: the GPU decodes its own stream; the oracle decodes the same bytes
+    d_xhat = torch.full((x.size,), float("nan"), dtype=torch.float32, device="cuda")
+    A.accept_mbq_decompress(p, d_stream, d_xhat, d_ws)
+    assert A.accept_last_device_status(d_ws) == 0
+    want = oracle.mbq_decompress(got, x.size)
+    assert np.array_equal(d_xhat.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    return alpha_next, side_g
+
+
+@pytest.mark.parametrize("k", [2, 3, 4])
+@pytest.mark.parametrize("n", [1, 31, 32, 33, 1000, 8192, 8193, 8192 * 5 + 777, 1 << 20])
+def test_mbq_parity_shapes(k, n):
+    x = workloads.random_tensor(n, 100 + k, "normal")
+    alpha_prev = np.array([0.9, 0.5, 0.27, 0.14][:k], dtype=np.float32)
+    check_mbq(x, k, 3, False, alpha_prev)
+    check_mbq(x, k, 0, True, None)
+
+
+@pytest.mark.parametrize("k", [2, 3, 4])
+def test_mbq_chained_batches_follow_the_oracle(k):
+    """Residue initialisation, then batches whose alpha is chained on the device."""
+    A = _A()
+    n = 8192 * 7 + 100
+    alpha = None
+    for t in range(0, 6):
+        x = workloads.generate("cfg1_act", t * n, n)
+        alpha, side = check_mbq(x, k, t, t == 0, alpha)
+        assert np.all(np.isfinite(side))
+    assert np.all(alpha > 0)
+
+
+def test_mbq_ties_duplicates_and_unsorted_coefficients():
+    """Values exactly on levels and midpoints; equal and unordered coefficients; a zero coefficient."""
+    for alpha_prev in ([2.0, 1.0], [1.0, 1.0], [0.25, 2.0, 1.0], [1.0, 0.0, 0.5], [0.5, 0.5, 0.5, 0.5], [3.0, -1.0, 0.5]):
+        alpha_prev = np.array(alpha_prev, dtype=np.float32)
+        k = alpha_prev.size
+        lv = np.unique(oracle.mbq_levels(alpha_prev))
+        probe = np.concatenate([lv, (lv[:-1] + lv[1:]) / 2, lv + 1e-6, lv - 1e-6,
+                                workloads.random_tensor(5000, k, "normal") * 2]).astype(np.float32)
+        check_mbq(probe, k, 2, False, alpha_prev)
+
+
+def test_mbq_singular_system_keeps_alpha():
+    x = np.abs(workloads.random_tensor(5000, 3, "normal")) + 10
+    alpha_prev = np.array([1.0, 0.5], dtype=np.float32)
+    alpha_next, _ = check_mbq(x, 2, 5, False, alpha_prev)
+    assert np.array_equal(alpha_next, alpha_prev)
+
+
+@pytest.mark.parametrize("name,k", [("cfg3_act", 4), ("cfg1_act", 2), ("cfg1_act", 3)])
+def test_mbq_workloads(name, k):
+    """Post-ReLU activations of the workloads at full size (cfg3: 51M elements), every plane word compared."""
+    x = workloads.generate(name)
+    stream0, alpha0 = oracle.mbq_compress(x[:1 << 20], k, 0, True)
+    check_mbq(x, k, 1, False, alpha0)
+
+
+def test_mbq_header_mismatch_and_bad_arguments():
+    A = _A()
+    x = workloads.random_tensor(5000, 1, "normal")
+    p, d_stream, _, _, d_ws = gpu_mbq_compress(x, 3, 0, True, None)
+    d_xhat = torch.empty(5000, dtype=torch.float32, device="cuda")
+    A.accept_mbq_decompress(A.MbqParams(5000, 3), d_stream, d_xhat, d_ws)
+    assert A.accept_last_device_status(d_ws) == 0
+    big = torch.zeros(A.accept_mbq_compressed_size(A.MbqParams(5000, 4)), dtype=torch.uint8, device="cuda")
+    big[:d_stream.numel()] = d_stream
+    A.accept_mbq_decompress(A.MbqParams(5000, 4), big, d_xhat, d_ws)
+    assert A.accept_last_device_status(d_ws) == A.DEV_BAD_HEADER
+    assert A.accept_mbq_check_params(A.MbqParams(0, 3)) == 9
+    assert A.accept_mbq_check_params(A.MbqParams(10, 5)) == 2
+    assert A.accept_mbq_check_params(A.MbqParams(10, 1)) == 2
+    with pytest.raises(A.AcceptError):
+        A.accept_mbq_compress(A.MbqParams(5000, 3, 1, False), torch.from_numpy(x).cuda(), None,
+                              torch.empty(3, device="cuda"), d_stream, d_ws)
+
+
+def test_mbq_nonfinite_input_sets_the_status_bit():
+    x = workloads.random_tensor(20000, 1, "normal")
+    x[777] = np.inf
+    _, _, _, status, _ = gpu_mbq_compress(x, 2, 1, False, np.array([1.0, 0.5], dtype=np.float32))
+    assert status & 1

@@ -71,6 +71,16 @@ def test_workspace_grows_with_wide_chunks_and_static_scratch_refuses_them(A):
         assert lib.accept_compress_static(ctypes.byref(p.c()), x_ptr, good, size, None, None) == want
 
 
+def test_mbq_size_queries_match_oracle(A):
+    for n, k in [(1, 2), (1000, 3), (1 << 20, 4), (51380224, 4)]:
+        p = A.MbqParams(n, k)
+        assert A.accept_mbq_check_params(p) == 0
+        assert A.accept_mbq_compressed_size(p) == oracle.mbq_stream_bytes(n, k)
+        assert A.accept_mbq_payload_offset(p) == oracle.mbq_payload_offset(k)
+        assert A.accept_mbq_workspace_size(p) == 64 + 136 * -(-n // 8192)
+    assert A.accept_mbq_compressed_size(A.MbqParams(10, 7)) == 0
+
+
 def test_invalid_params_are_rejected(A):
     P = A.Params
     assert A.accept_check_params(P(0, 32, 4)) == 9
