@@ -207,7 +207,7 @@ void launch_mbq_compress(const accept::MbqArgs& a, cudaStream_t s) {
   } else {
     accept::mbq_encode_kernel<K, false><<<a.n_blocks, 256, 0, s>>>(a);
   }
-  accept::mbq_finalize_kernel<K><<<1, 256, 0, s>>>(a);
+  accept::mbq_finalize_kernel<K><<<1, accept::kMbqFinalizeThreads, 0, s>>>(a);
   g_launches.fetch_add(2 + (a.init ? 2 * K : 0), std::memory_order_relaxed);
 }
 

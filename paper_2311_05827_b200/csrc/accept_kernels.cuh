@@ -65,13 +65,15 @@ __device__ __forceinline__ void store_interleaved(uint32_t* payload, uint64_t oc
 
 // BITPLANE: lane q of a quad ends with the word of binary digit q (and q+4 for K = 8) of the
 // quad's group and stores it.  group = global index of the 32-element group.  All lanes call.
+// Returns the word of binary digit q = lane & 3 of the quad's group (K <= 4; 0 for K = 8).
 template <int K>
-__device__ __forceinline__ void store_bitplane_guarded(uint32_t* payload, uint64_t group, uint32_t xlo, uint32_t xhi,
-                                                       int lane, bool store) {
+__device__ __forceinline__ uint32_t store_bitplane_guarded(uint32_t* payload, uint64_t group, uint32_t xlo, uint32_t xhi,
+                                                           int lane, bool store) {
   const int q = lane & 3;
   if (K <= 4) {
     const uint32_t w = quad_transpose(planes_nibbles(merge_nibbles(xlo, xhi)), lane);
     if (store && q < K) payload[group * K + q] = w;
+    return w;
   } else {
     const uint32_t lo = merge_nibbles(xlo & 0x0F0F0F0Fu, xhi & 0x0F0F0F0Fu);
     const uint32_t hi = merge_nibbles((xlo >> 4) & 0x0F0F0F0Fu, (xhi >> 4) & 0x0F0F0F0Fu);
@@ -81,6 +83,7 @@ __device__ __forceinline__ void store_bitplane_guarded(uint32_t* payload, uint64
       payload[group * 8 + q] = w0;
       payload[group * 8 + 4 + q] = w1;
     }
+    return 0u;
   }
 }
 

@@ -18,6 +18,7 @@ namespace accept {
 constexpr int kMbqRounds = 4;                      // octets per thread
 constexpr int kMbqTile = kMbqRounds * 256 * 8;     // elements per block
 constexpr int kMbqPartialBytes = 128;              // per-block record in the workspace
+constexpr int kMbqFinalizeThreads = 256;           // threads of the single finalize block
 
 // Per-block partial sums (one 128-byte record per block of the encode pass).
 struct MbqPartial {
@@ -107,14 +108,17 @@ __device__ void mbq_build_table(const float* alpha_global, MbqTable<K>* t, float
   __syncthreads();
 }
 
+// Branch-free binary search over the sorted thresholds; the position is kept as a byte offset so
+// that every probe is a shared-memory load with an immediate displacement.
 template <int K>
 __device__ __forceinline__ uint32_t mbq_nearest_code(const MbqTable<K>& t, float x) {
   constexpr int L = 1 << K;
-  int idx = 0;
+  const char* thr = reinterpret_cast<const char*>(t.thr);
+  uint32_t off = 0;
 #pragma unroll
   for (int step = L / 2; step >= 1; step >>= 1)
-    if (x > t.thr[idx + step]) idx += step;
-  return t.code[idx];
+    if (x > *reinterpret_cast<const float*>(thr + off + 4 * step)) off += 4 * step;
+  return *reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(t.code) + off);
 }
 
 // Signs of the successive residues with the given coefficients (residue method): bit j = [r_j >= 0].
@@ -142,6 +146,11 @@ __device__ __forceinline__ void mbq_ld_octet(const float* x, uint64_t n, uint64_
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = (e + i < n) ? __ldg(x + e + i) : 0.0f;
   }
+}
+
+// acc += x when flag != 0, as one predicated add (no branch, no 64-bit select)
+__device__ __forceinline__ void add_if(double& acc, double x, uint32_t flag) {
+  asm("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p add.rn.f64 %0, %0, %1;\n\t}" : "+d"(acc) : "d"(x), "r"(flag));
 }
 
 __device__ __forceinline__ double warp_sum(double v) {
@@ -222,11 +231,9 @@ __global__ void __launch_bounds__(256) mbq_encode_kernel(const MbqArgs a) {
   const uint64_t n_oct = (a.n + 7) / 8;
   const uint64_t n_oct_stored = ((a.n + 31) / 32) * 4;
   double plus[K], sum_x = 0.0;
-  uint32_t count[K], differ[6];
+  uint32_t my_count = 0, my_differ[3] = {0, 0, 0};  // of basis q = lane & 3, and of the pairs (q, q ^ d)
 #pragma unroll
-  for (int j = 0; j < K; ++j) { plus[j] = 0.0; count[j] = 0; }
-#pragma unroll
-  for (int p = 0; p < 6; ++p) differ[p] = 0;
+  for (int j = 0; j < K; ++j) plus[j] = 0.0;
 
   float v[kMbqRounds][8];
 #pragma unroll
@@ -239,44 +246,46 @@ __global__ void __launch_bounds__(256) mbq_encode_kernel(const MbqArgs a) {
       for (int e = 0; e < 8; ++e) v[r][e] = 0.0f;
     }
   }
+  const int q = lane & 3;
 #pragma unroll
   for (int r = 0; r < kMbqRounds; ++r) {
     const uint64_t oct = (uint64_t)blockIdx.x * (kMbqRounds * 256) + r * 256 + tid;
-    uint32_t xlo = 0, xhi = 0;
+    // elements of this octet that exist (8 for all but the last octets of the tensor)
+    const int valid = (oct * 8 + 8 <= a.n) ? 8 : ((oct * 8 < a.n) ? (int)(a.n - oct * 8) : 0);
+    uint32_t c[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-      uint32_t c = 0;
-      if (oct * 8 + e < a.n) {
-        if (INIT) {
-          float res;
-          c = mbq_residue_code<K>(alpha, v[r][e], K, &res);
-        } else {
-          c = mbq_nearest_code<K>(s_table, v[r][e]);
-        }
-        const double xd = (double)v[r][e];
-        sum_x += xd;
-#pragma unroll
-        for (int j = 0; j < K; ++j)
-          if ((c >> j) & 1u) plus[j] += xd;
+      if (INIT) {
+        float res;
+        c[e] = mbq_residue_code<K>(alpha, v[r][e], K, &res);
+      } else {
+        c[e] = mbq_nearest_code<K>(s_table, v[r][e]);
       }
-      if (e < 4) xlo |= c << (8 * e);
-      else xhi |= c << (8 * (e - 4));
     }
-    // plane form: byte j = the eight signs of basis j
-    const uint32_t planes = planes_nibbles(merge_nibbles(xlo, xhi));
+    if (valid < 8) {  // codes of elements past the end are zero (their values were loaded as 0)
 #pragma unroll
-    for (int j = 0; j < K; ++j) count[j] += __popc((planes >> (8 * j)) & 0xFFu);
-    {
-      int p = 0;
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = i + 1; j < 4; ++j, ++p)
-          if (j < K) differ[p] += __popc(((planes >> (8 * i)) ^ (planes >> (8 * j))) & 0xFFu);
+      for (int e = 0; e < 8; ++e)
+        if (e >= valid) c[e] = 0;
     }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const double xd = (double)v[r][e];  // 0 past the end
+      sum_x += xd;
+#pragma unroll
+      for (int j = 0; j < K; ++j) add_if(plus[j], xd, c[e] & (1u << j));
+    }
+    const uint32_t xlo = pack_bytes<0>(c[0], c[1], c[2], c[3]);
+    const uint32_t xhi = pack_bytes<0>(c[4], c[5], c[6], c[7]);
     const bool stored = oct < n_oct_stored;
-    const uint32_t any = __ballot_sync(0xffffffffu, stored);
-    if (any) store_bitplane_guarded<K>(a.payload, oct >> 2, xlo, xhi, lane, stored);
+    // after the quad transpose lane q holds the 32 signs of basis q of its group: counts of +1 and,
+    // against the words of the other three lanes of the quad, counts of differing signs
+    const uint32_t w = store_bitplane_guarded<K>(a.payload, oct >> 2, xlo, xhi, lane, stored);
+    my_count += __popc(w);
+#pragma unroll
+    for (int d = 1; d < 4; ++d) {
+      const uint32_t other = __shfl_xor_sync(0xffffffffu, w, d);
+      my_differ[d - 1] += __popc(w ^ other);
+    }
   }
 
   // block sums in a fixed order: lanes by butterfly, warps one after the other
@@ -284,17 +293,28 @@ __global__ void __launch_bounds__(256) mbq_encode_kernel(const MbqArgs a) {
   for (int j = 0; j < K; ++j) {
     const double s = warp_sum(plus[j]);
     if (lane == 0) s_dbl[warp][j] = s;
-    const uint32_t c = __reduce_add_sync(0xffffffffu, count[j]);
-    if (lane == 0) atomicAdd(&s_cnt[j], c);
   }
   {
     const double s = warp_sum(sum_x);
     if (lane == 0) s_dbl[warp][K] = s;
   }
+  // lanes with the same q hold partial counts of the same basis / pairs: add over the eight quads
 #pragma unroll
-  for (int p = 0; p < 6; ++p) {
-    const uint32_t c = __reduce_add_sync(0xffffffffu, differ[p]);
-    if (lane == 0) atomicAdd(&s_cnt[4 + p], c);
+  for (int d = 4; d <= 16; d <<= 1) {
+    my_count += __shfl_xor_sync(0xffffffffu, my_count, d);
+#pragma unroll
+    for (int i = 0; i < 3; ++i) my_differ[i] += __shfl_xor_sync(0xffffffffu, my_differ[i], d);
+  }
+  if (lane < 4) {
+    atomicAdd(&s_cnt[q], my_count);
+#pragma unroll
+    for (int d = 1; d < 4; ++d) {
+      const int other = q ^ d;
+      if (q < other) {  // each pair once; pair index in the order (0,1) (0,2) (0,3) (1,2) (1,3) (2,3)
+        const int pair = (q == 0) ? other - 1 : (q == 1 ? other + 1 : 5);
+        atomicAdd(&s_cnt[4 + pair], my_differ[d - 1]);
+      }
+    }
   }
   __syncthreads();
   if (tid == 0) {
@@ -320,9 +340,9 @@ __global__ void __launch_bounds__(256) mbq_encode_kernel(const MbqArgs a) {
 // partial pivoting, in double), Eq. 4 (moving average), Eq. 5 (bias), and writes header, side
 // words and alpha_next.  One block.
 template <int K>
-__global__ void __launch_bounds__(256) mbq_finalize_kernel(const MbqArgs a) {
-  __shared__ double s_dbl[256][K + 1];
-  __shared__ unsigned long long s_int[256][10];
+__global__ void __launch_bounds__(kMbqFinalizeThreads) mbq_finalize_kernel(const MbqArgs a) {
+  __shared__ double s_dbl[kMbqFinalizeThreads][K + 1];
+  __shared__ unsigned long long s_int[kMbqFinalizeThreads][10];
   const int tid = threadIdx.x;
   double d[K + 1];
   unsigned long long c[10];
@@ -330,7 +350,9 @@ __global__ void __launch_bounds__(256) mbq_finalize_kernel(const MbqArgs a) {
   for (int j = 0; j <= K; ++j) d[j] = 0.0;
 #pragma unroll
   for (int j = 0; j < 10; ++j) c[j] = 0;
-  for (uint32_t b = tid; b < a.n_blocks; b += 256) {
+  // thread t adds records t, t + T, t + 2T, ... in that order
+#pragma unroll 4
+  for (uint32_t b = tid; b < a.n_blocks; b += kMbqFinalizeThreads) {
     const MbqPartial& p = a.partial[b];
 #pragma unroll
     for (int j = 0; j < K; ++j) { d[j] += p.plus[j]; c[j] += p.count[j]; }
@@ -348,7 +370,7 @@ __global__ void __launch_bounds__(256) mbq_finalize_kernel(const MbqArgs a) {
   for (int j = 0; j <= K; ++j) d[j] = 0.0;
 #pragma unroll
   for (int j = 0; j < 10; ++j) c[j] = 0;
-  for (int i = 0; i < 256; ++i) {
+  for (int i = 0; i < kMbqFinalizeThreads; ++i) {
 #pragma unroll
     for (int j = 0; j <= K; ++j) d[j] += s_dbl[i][j];
 #pragma unroll
