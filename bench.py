@@ -344,15 +344,13 @@ def run_gpu(args):
 
 
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch, filled from profiles/ once captured
-TRAFFIC = {("cfg4_hidden", "accept_compress"): 319.48e6, ("cfg4_hidden", "accept_decompress"): 277.41e6}
+TRAFFIC = {("cfg4_hidden", "accept_compress"): 318.74e6, ("cfg4_hidden", "accept_decompress"): 277.86e6}
 
 
 def sweep(A, torch, peak, args):
     """All five workloads, headline modes: per-kernel time and HBM fraction."""
     rows = []
     for name, spec in workloads.TENSORS.items():
-        if spec.n * 4 > (1 << 30) and args.sweep_max_bytes < (1 << 30) + 1:
-            pass
         if spec.n * 4 > args.sweep_max_bytes:
             continue
         x_host = workloads.generate(name)
@@ -372,6 +370,67 @@ def sweep(A, torch, peak, args):
                    100 * rows[-1]["decompress_frac_measured"]), file=sys.stderr)
             del codec
             torch.cuda.empty_cache()
+        if name in ("cfg3_grad", "cfg4_hidden"):
+            rows.append(sweep_per_tensor(A, torch, peak, name, spec, x_host))
+        if name == "cfg3_act":
+            rows.extend(sweep_mbq(A, torch, peak, name, spec, x_host))
+    return rows
+
+
+def sweep_per_tensor(A, torch, peak, name, spec, x_host):
+    """The paper's granularity: one range for the whole tensor (two passes over the input, 8 + k/8 B/element)."""
+    mode = spec.headline[0]
+    chunk = (spec.n + 31) // 32 * 32
+    codec = Codec(A, torch, x_host, chunk, mode, spec.seed)
+    ms_c, ms_d = codec.run_isolated(20)
+    assert codec.status() == 0
+    alg_c, alg_d = spec.n * (8.0 + mode.k / 8.0), spec.n * (4.0 + mode.k / 8.0)
+    row = {"workload": name, "mode": mode_name(mode) + "-one-range", "mbytes": spec.n * 4 / 2 ** 20, "copies": codec.copies,
+           "compress_ms": ms_c, "decompress_ms": ms_d, "compress_frac_measured": alg_c / ms_c / 1e6 / peak,
+           "decompress_frac_measured": alg_d / ms_d / 1e6 / peak, "compress_bytes_per_element": 8.0 + mode.k / 8.0}
+    print("# %-12s %-34s c %8.4f ms %6.1f%%  d %8.4f ms %6.1f%% (of measured copy bw)" %
+          (name, row["mode"][:34], ms_c, 100 * row["compress_frac_measured"], ms_d, 100 * row["decompress_frac_measured"]),
+          file=sys.stderr)
+    return row
+
+
+def sweep_mbq(A, torch, peak, name, spec, x_host):
+    """The forward quantizer (multi-bit quantization): residue initialisation, encode + coefficient update, decode."""
+    rows = []
+    n = spec.n
+    for k in (2, 3, 4):
+        p0, p1 = A.MbqParams(n, k, 0, True), A.MbqParams(n, k, 1, False)
+        copies = 2
+        x = [torch.from_numpy(x_host).cuda() for _ in range(copies)]
+        st = [A.new_stream_buffer(p0) for _ in range(copies)]
+        xh = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(copies)]
+        ws, alpha = A.new_workspace(p0), torch.zeros(k, dtype=torch.float32, device="cuda")
+
+        def timed(fn, steps=20, warm=3):
+            for i in range(warm):
+                fn(i % copies)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(steps):
+                fn(i % copies)
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / steps
+
+        ms_i = timed(lambda j: A.accept_mbq_compress(p0, x[j], None, alpha, st[j], ws), steps=5, warm=1)
+        ms_c = timed(lambda j: A.accept_mbq_compress(p1, x[j], alpha, alpha, st[j], ws))
+        ms_d = timed(lambda j: A.accept_mbq_decompress(p1, st[j], xh[j], ws))
+        assert A.accept_last_device_status(ws) == 0
+        alg = n * (4.0 + k / 8.0)
+        rows.append({"workload": name, "mode": "mbq-k%d" % k, "mbytes": n * 4 / 2 ** 20, "copies": copies,
+                     "init_ms": ms_i, "compress_ms": ms_c, "decompress_ms": ms_d,
+                     "compress_frac_measured": alg / ms_c / 1e6 / peak, "decompress_frac_measured": alg / ms_d / 1e6 / peak})
+        print("# %-12s %-34s c %8.4f ms %6.1f%%  d %8.4f ms %6.1f%% (of measured copy bw); residue init %.4f ms" %
+              (name, "mbq-k%d" % k, ms_c, 100 * rows[-1]["compress_frac_measured"], ms_d,
+               100 * rows[-1]["decompress_frac_measured"], ms_i), file=sys.stderr)
+        del x, st, xh
+        torch.cuda.empty_cache()
     return rows
 
 
