@@ -8,8 +8,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libaccept.so")
 SOURCES = [os.path.join(CSRC, "accept_api.cu")]
-DEPENDS = SOURCES + [os.path.join(CSRC, "accept_kernels.cuh"), os.path.join(CSRC, "accept_device.cuh"),
-                     os.path.join(os.path.dirname(HERE), "include", "accept.h")]
+DEPENDS = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh"))) + [
+    os.path.join(os.path.dirname(HERE), "include", "accept.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
