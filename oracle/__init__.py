@@ -84,6 +84,14 @@ def _load():
     lib.oracle_mbq_compress.argtypes = [vp, u64, u32, u32, i32, f32p, vp, f32p]
     lib.oracle_mbq_decompress.restype = i32
     lib.oracle_mbq_decompress.argtypes = [vp, u64, u64, vp]
+    lib.oracle_strided_payload_bytes.restype = u64
+    lib.oracle_strided_payload_bytes.argtypes = [u64, u32, u32]
+    lib.oracle_strided_stream_bytes.restype = u64
+    lib.oracle_strided_stream_bytes.argtypes = [u64, u32, u32, u32]
+    lib.oracle_compress_strided.restype = i32
+    lib.oracle_compress_strided.argtypes = [vp, u64, u32, u32, i32, i32, i32, u64, u64, u32, vp]
+    lib.oracle_decompress_strided.restype = i32
+    lib.oracle_decompress_strided.argtypes = [vp, u64, u64, vp]
     _lib = lib
     return lib
 
@@ -250,4 +258,29 @@ def mbq_decompress(stream, n: int) -> np.ndarray:
     xhat = np.empty(n, dtype=np.float32)
     if _load().oracle_mbq_decompress(_ptr(stream), stream.size, n, _ptr(xhat)) != 0:
         raise ValueError("oracle_mbq_decompress: invalid stream header")
+    return xhat
+
+
+# ---------------------------------------------------------------- grouping along the batch dimension
+
+def strided_stream_bytes(n: int, chunk: int, k: int, stride: int) -> int:
+    return int(_load().oracle_strided_stream_bytes(n, chunk, k, stride))
+
+
+def compress_strided(x, chunk: int, k: int, stride: int, range_: int = RANGE_ABSMAX, round_: int = ROUND_NEAREST,
+                     layout: int = LAYOUT_INTERLEAVED, seed: int = 0, rng_offset: int = 0):
+    """Pack groups = 32 batch neighbours of one feature; x is (n // stride) x stride.  -> (stream, flag)."""
+    x = _f32(x)
+    assert x.size % stride == 0
+    out = np.empty(strided_stream_bytes(x.size, chunk, k, stride), dtype=np.uint8)
+    flag = _load().oracle_compress_strided(_ptr(x), x.size, chunk, k, range_, round_, layout, seed, rng_offset,
+                                           stride, _ptr(out))
+    return out, int(flag)
+
+
+def decompress_strided(stream, n: int) -> np.ndarray:
+    stream = np.ascontiguousarray(stream, dtype=np.uint8).reshape(-1)
+    xhat = np.empty(n, dtype=np.float32)
+    if _load().oracle_decompress_strided(_ptr(stream), stream.size, n, _ptr(xhat)) != 0:
+        raise ValueError("oracle_decompress_strided: invalid stream header")
     return xhat

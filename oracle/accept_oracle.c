@@ -514,3 +514,80 @@ int oracle_mbq_decompress(const void* stream, uint64_t stream_bytes, uint64_t n_
   }
   return 0;
 }
+
+/* ============================================================================================
+ * Grouping along the batch dimension (Sec. 3.3: "the bit-wise encoder concatenates the quantized
+ * data along the batch size dimension"; "Forward Encoder": consecutive elements along the first
+ * dimension share an integer; "Backward Encoder": "combine two tensors along the first dimension").
+ *
+ * The tensor is n_b x F (F = w*h*c values per sample, group_stride).  A pack group is made of the
+ * 32 batch neighbours (rows 32g .. 32g+31) of one feature f instead of 32 consecutive values:
+ * group index G = g*F + f, words G*k .. G*k+k-1, element (row b, feature f) at position t = b % 32.
+ * Rows past n_b are zero bits ("ceil(n/8)" of Eq. 8).  Ranges stay per chunk of C consecutive
+ * values of the vectorised tensor.  Header word 7 holds F (0 = consecutive grouping).
+ * ============================================================================================ */
+
+uint64_t oracle_strided_payload_bytes(uint64_t n, uint32_t k, uint32_t F) {
+  uint64_t nb = n / F;
+  return 4ull * k * ((nb + 31) / 32) * F;
+}
+
+uint64_t oracle_strided_stream_bytes(uint64_t n, uint32_t C, uint32_t k, uint32_t F) {
+  return oracle_payload_offset(n, C) + oracle_strided_payload_bytes(n, k, F);
+}
+
+/* bit position of digit j of element i in the payload */
+static uint64_t strided_bit_position(uint64_t i, uint32_t j, uint32_t k, int layout, uint32_t F) {
+  uint64_t b = i / F, f = i % F;
+  uint64_t G = (b / 32) * F + f;
+  uint32_t t = (uint32_t)(b % 32);
+  if (layout == LAYOUT_INTERLEAVED) return 32ull * k * G + (uint64_t)k * t + j;
+  return 32ull * (k * G + j) + t;
+}
+
+int oracle_compress_strided(const float* x, uint64_t n, uint32_t C, uint32_t k, int range, int round_mode,
+                            int layout, uint64_t seed, uint64_t rng_offset, uint32_t F, void* stream) {
+  uint8_t* bytes = (uint8_t*)stream;
+  memset(bytes, 0, oracle_strided_stream_bytes(n, C, k, F));
+  uint32_t header[8] = {ORACLE_MAGIC, ORACLE_VERSION, (uint32_t)n, (uint32_t)(n >> 32), C, k,
+                        (uint32_t)range | ((uint32_t)round_mode << 8) | ((uint32_t)layout << 16), F};
+  memcpy(bytes, header, 32);
+  uint8_t* codes = (uint8_t*)malloc(n);
+  int flags = oracle_quantize(x, n, C, k, range, round_mode, seed, rng_offset, codes, (float*)(bytes + 32));
+  uint32_t* payload = (uint32_t*)(bytes + oracle_payload_offset(n, C));
+  for (uint64_t i = 0; i < n; ++i)
+    for (uint32_t j = 0; j < k; ++j) {
+      uint64_t pos = strided_bit_position(i, j, k, layout, F);
+      payload[pos / 32] |= (uint32_t)((codes[i] >> j) & 1u) << (pos % 32);
+    }
+  free(codes);
+  return flags;
+}
+
+int oracle_decompress_strided(const void* stream, uint64_t stream_bytes, uint64_t n_expected, float* xhat) {
+  const uint8_t* bytes = (const uint8_t*)stream;
+  uint32_t header[8];
+  if (stream_bytes < 32) return -1;
+  memcpy(header, bytes, 32);
+  uint64_t n = (uint64_t)header[2] | ((uint64_t)header[3] << 32);
+  uint32_t C = header[4], k = header[5], F = header[7];
+  int range = header[6] & 0xff, layout = (header[6] >> 16) & 0xff;
+  if (header[0] != ORACLE_MAGIC || header[1] != ORACLE_VERSION) return -1;
+  if (n != n_expected || n == 0 || C < 32 || C % 32 != 0 || F == 0 || n % F != 0) return -1;
+  if (!(k == 2 || k == 3 || k == 4 || k == 8) || range > 1 || layout > 1) return -1;
+  if (stream_bytes < oracle_strided_stream_bytes(n, C, k, F)) return -1;
+  const float* meta = (const float*)(bytes + 32);
+  const uint32_t* payload = (const uint32_t*)(bytes + oracle_payload_offset(n, C));
+  uint8_t* codes = (uint8_t*)malloc(n);
+  for (uint64_t i = 0; i < n; ++i) {
+    uint32_t c = 0;
+    for (uint32_t j = 0; j < k; ++j) {
+      uint64_t pos = strided_bit_position(i, j, k, layout, F);
+      c |= ((payload[pos / 32] >> (pos % 32)) & 1u) << j;
+    }
+    codes[i] = (uint8_t)c;
+  }
+  oracle_dequantize(codes, meta, n, C, k, range, xhat);
+  free(codes);
+  return 0;
+}
