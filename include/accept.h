@@ -31,7 +31,7 @@
  *
  * Stream layout (little-endian, byte offsets):
  *   [0,32)    header, eight u32: magic 0x54504341 ("ACPT"), version 1, n_elems low, n_elems high,
- *             chunk_elems, k, range | round<<8 | layout<<16, 0
+ *             chunk_elems, k, range | round<<8 | layout<<16, group_stride
  *   [32, 32+8M)   M = ceil(n_elems/chunk_elems) records {float s; float o}, one per chunk
  *   [P, ...)  payload, P = 32+8M rounded up to a multiple of 16.  Chunk m starts at word
  *             m*chunk_elems*k/32 of the payload.  A partial last chunk holds ceil(valid/32)*k
@@ -84,6 +84,15 @@ typedef enum { ACCEPT_LAYOUT_INTERLEAVED = 0, ACCEPT_LAYOUT_BITPLANE = 1 } accep
  *   n_elems      N >= 1, number of fp32 values.
  *   chunk_elems  C, multiple of 32, >= 32: elements sharing one range.
  *   k            bit width: 2, 3 (BITPLANE only), 4 or 8.
+ *   group_stride 0, or F = values per sample (w*h*c): the tensor is (n_elems/F) x F and a pack group is
+ *                made of the 32 BATCH neighbours (rows 32g..32g+31) of one feature f, as the paper's
+ *                encoders do (Sec. 3.3: "concatenates the quantized data along the batch size
+ *                dimension"): group index G = g*F + f, words G*k .. G*k+k-1 of the payload, element
+ *                (row b, feature f) at position t = b % 32 of its group; rows past the last are zero
+ *                bits; payload = 4*k*ceil(rows/32)*F bytes.  Ranges stay per chunk of consecutive
+ *                values.  Needs F % 8 == 0, n_elems % F == 0, 32-byte aligned tensors, and not
+ *                (k = 8 with BITPLANE); runs as range pass + constants + encode (workspace: 16
+ *                bytes per chunk more, as for chunk_elems > 32768).  Header word 7 carries F.
  *   seed, rng_offset  STOCHASTIC only.  Element i draws
  *                  U_i = (g >> 8) * 2^-24,
  *                  g   = h if ctr is even, h * 0x9E3779B1 (mod 2^32) if ctr is odd,
@@ -101,7 +110,7 @@ typedef struct {
   int32_t range;   /* accept_range  */
   int32_t round;   /* accept_round  */
   int32_t layout;  /* accept_layout */
-  uint32_t reserved; /* must be 0 */
+  uint32_t group_stride; /* 0: pack groups of 32 consecutive values; F > 0: see below */
   uint64_t seed;
   uint64_t rng_offset;
 } accept_params;
@@ -119,7 +128,7 @@ size_t accept_compressed_size(const accept_params* p);
 size_t accept_payload_offset(const accept_params* p);
 
 /*
- * Bytes of device workspace the kernels need: 16, plus 16 per chunk when chunk_elems > 32768
+ * Bytes of device workspace the kernels need: 16, plus 16 per chunk when chunk_elems > 32768 or group_stride != 0
  * (such chunks do not fit on chip: their ranges are gathered in the workspace first, and the input
  * is read twice).  Word 0 is the device status word; the caller zeroes the workspace once (and
  * whenever it wants to clear the status); the workspace must be 16-byte aligned.  0 if p is invalid.

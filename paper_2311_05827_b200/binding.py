@@ -47,7 +47,7 @@ class AcceptError(RuntimeError):
 class CParams(ctypes.Structure):
     _fields_ = [("n_elems", ctypes.c_uint64), ("chunk_elems", ctypes.c_uint32), ("k", ctypes.c_uint32),
                 ("range", ctypes.c_int32), ("round", ctypes.c_int32), ("layout", ctypes.c_int32),
-                ("reserved", ctypes.c_uint32), ("seed", ctypes.c_uint64), ("rng_offset", ctypes.c_uint64)]
+                ("group_stride", ctypes.c_uint32), ("seed", ctypes.c_uint64), ("rng_offset", ctypes.c_uint64)]
 
 
 @dataclass(frozen=True)
@@ -60,9 +60,10 @@ class Params:
     layout: int = LAYOUT_INTERLEAVED
     seed: int = 0
     rng_offset: int = 0
+    group_stride: int = 0
 
     def c(self) -> CParams:
-        return CParams(self.n_elems, self.chunk_elems, self.k, self.range, self.round, self.layout, 0,
+        return CParams(self.n_elems, self.chunk_elems, self.k, self.range, self.round, self.layout, self.group_stride,
                        self.seed & (2**64 - 1), self.rng_offset & (2**64 - 1))
 
 
@@ -172,7 +173,7 @@ def accept_parse_header(header_bytes: bytes) -> Params:
     buf = ctypes.create_string_buffer(bytes(header_bytes[:HEADER_BYTES]), HEADER_BYTES)
     out = CParams()
     _check(lib().accept_parse_header(ctypes.cast(buf, ctypes.c_void_p), ctypes.byref(out)), "accept_parse_header")
-    return Params(out.n_elems, out.chunk_elems, out.k, out.range, out.round, out.layout)
+    return Params(out.n_elems, out.chunk_elems, out.k, out.range, out.round, out.layout, group_stride=out.group_stride)
 
 
 # ---- device entry points -------------------------------------------------------------------

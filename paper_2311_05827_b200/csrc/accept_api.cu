@@ -10,6 +10,7 @@
 #include "accept_kernels.cuh"
 #include "accept_wide.cuh"
 #include "accept_mbq.cuh"
+#include "accept_strided.cuh"
 
 namespace {
 
@@ -25,6 +26,12 @@ uint64_t n_chunks_of(const accept_params* p) { return (p->n_elems + p->chunk_ele
 constexpr uint32_t kWideChunk = 32768;
 
 bool is_wide(const accept_params* p) { return p->chunk_elems > kWideChunk; }
+bool is_strided(const accept_params* p) { return p->group_stride != 0; }
+// pack groups stored in the payload
+uint64_t n_groups_of(const accept_params* p) {
+  if (!is_strided(p)) return (p->n_elems + 31) / 32;
+  return ((p->n_elems / p->group_stride + 31) / 32) * (uint64_t)p->group_stride;
+}
 
 // Geometry of the register-resident compress path for chunk size C: rounds R and threads per chunk.
 struct FastGeometry { int rounds; uint32_t tpc; };
@@ -55,6 +62,7 @@ CodecArgs make_args(const accept_params* p, void* d_stream, void* d_ws) {
     if (p->chunk_elems == (1u << s)) a.chunk_shift = s;
   a.header_word6 = (uint32_t)p->range | ((uint32_t)p->round << 8) | ((uint32_t)p->layout << 16);
   a.k = p->k;
+  a.group_stride = p->group_stride;
   return a;
 }
 
@@ -171,6 +179,66 @@ accept_status launch_wide(const accept_params* p, const CodecArgs& a, uint8_t* r
   return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
 }
 
+// ---- pack groups along the batch dimension ---------------------------------------------------------
+
+template <int K, int LAYOUT, int RANGE>
+void launch_strided_encode(int round, const CodecArgs& a, const accept::ChunkRecord* rec, dim3 grid, cudaStream_t s) {
+  if (round == accept::kNearest) accept::strided_encode_kernel<K, LAYOUT, RANGE, accept::kNearest><<<grid, 256, 0, s>>>(a, rec);
+  else accept::strided_encode_kernel<K, LAYOUT, RANGE, accept::kStochastic><<<grid, 256, 0, s>>>(a, rec);
+}
+
+template <int RANGE>
+void launch_strided_encode_for(const accept_params* p, const CodecArgs& a, const accept::ChunkRecord* rec, dim3 grid,
+                               cudaStream_t s) {
+  const bool bp = p->layout == ACCEPT_LAYOUT_BITPLANE;
+  switch (p->k) {
+    case 2: bp ? launch_strided_encode<2, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
+               : launch_strided_encode<2, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s); break;
+    case 3: launch_strided_encode<3, accept::kBitplane, RANGE>(p->round, a, rec, grid, s); break;
+    case 4: bp ? launch_strided_encode<4, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
+               : launch_strided_encode<4, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s); break;
+    default: launch_strided_encode<8, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s); break;
+  }
+}
+
+template <int RANGE>
+void launch_strided_decode_for(const accept_params* p, const CodecArgs& a, dim3 grid, cudaStream_t s) {
+  const bool bp = p->layout == ACCEPT_LAYOUT_BITPLANE;
+  switch (p->k) {
+    case 2: bp ? accept::strided_decode_kernel<2, accept::kBitplane, RANGE><<<grid, 256, 0, s>>>(a)
+               : accept::strided_decode_kernel<2, accept::kInterleaved, RANGE><<<grid, 256, 0, s>>>(a); break;
+    case 3: accept::strided_decode_kernel<3, accept::kBitplane, RANGE><<<grid, 256, 0, s>>>(a); break;
+    case 4: bp ? accept::strided_decode_kernel<4, accept::kBitplane, RANGE><<<grid, 256, 0, s>>>(a)
+               : accept::strided_decode_kernel<4, accept::kInterleaved, RANGE><<<grid, 256, 0, s>>>(a); break;
+    default: accept::strided_decode_kernel<8, accept::kInterleaved, RANGE><<<grid, 256, 0, s>>>(a); break;
+  }
+}
+
+dim3 strided_grid(const accept_params* p) {
+  const unsigned gx = (p->group_stride / 8 + accept::kStridedOctetsPerBlock - 1) / accept::kStridedOctetsPerBlock;
+  const unsigned gy = (unsigned)((p->n_elems / p->group_stride + 31) / 32);
+  return dim3(gx, gy, 1);
+}
+
+accept_status launch_strided(const accept_params* p, const CodecArgs& a, uint8_t* rec_bytes, cudaStream_t s) {
+  accept::ChunkRecord* rec = reinterpret_cast<accept::ChunkRecord*>(rec_bytes);
+  if (cudaMemsetAsync(rec, 0, sizeof(accept::ChunkRecord) * a.n_chunks, s) != cudaSuccess) return ACCEPT_ERR_CUDA;
+  const uint64_t n_oct = (p->n_elems + 7) / 8;
+  const unsigned range_grid = (unsigned)((n_oct + 4 * 256 - 1) / (4 * 256));
+  const unsigned fin_grid = (unsigned)((a.n_chunks + 255) / 256);
+  if (p->range == ACCEPT_RANGE_ABSMAX) {
+    accept::wide_range_kernel<accept::kAbsMax, 4><<<range_grid, 256, 0, s>>>(a, rec);
+    accept::wide_finalize_kernel<accept::kAbsMax><<<fin_grid, 256, 0, s>>>(a, rec);
+    launch_strided_encode_for<accept::kAbsMax>(p, a, rec, strided_grid(p), s);
+  } else {
+    accept::wide_range_kernel<accept::kMinMax, 4><<<range_grid, 256, 0, s>>>(a, rec);
+    accept::wide_finalize_kernel<accept::kMinMax><<<fin_grid, 256, 0, s>>>(a, rec);
+    launch_strided_encode_for<accept::kMinMax>(p, a, rec, strided_grid(p), s);
+  }
+  g_launches.fetch_add(3, std::memory_order_relaxed);
+  return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+}
+
 // ---- multi-bit quantization --------------------------------------------------------------------
 
 uint32_t mbq_blocks(const accept_mbq_params* p) {
@@ -258,7 +326,11 @@ accept_status accept_check_params(const accept_params* p) {
   if (p->layout != ACCEPT_LAYOUT_INTERLEAVED && p->layout != ACCEPT_LAYOUT_BITPLANE) return ACCEPT_ERR_BAD_ENUM;
   if (!(p->k == 2 || p->k == 3 || p->k == 4 || p->k == 8)) return ACCEPT_ERR_BAD_K;
   if (p->k == 3 && p->layout != ACCEPT_LAYOUT_BITPLANE) return ACCEPT_ERR_BAD_K;
-  if (p->reserved != 0) return ACCEPT_ERR_BAD_ENUM;
+  if (p->group_stride != 0) {
+    if (p->group_stride % 8 != 0 || p->n_elems % p->group_stride != 0) return ACCEPT_ERR_BAD_SIZE;
+    if (p->k == 8 && p->layout == ACCEPT_LAYOUT_BITPLANE) return ACCEPT_ERR_BAD_K;
+    if ((p->n_elems / p->group_stride + 31) / 32 > 65535) return ACCEPT_ERR_BAD_SIZE;  // batch groups ride on grid.y
+  }
   // one block per chunk / per 4096 elements must fit the grid's x dimension
   if (n_chunks_of(p) > 0x7fffffffull || p->n_elems / 4096 > 0x7ffffff0ull) return ACCEPT_ERR_BAD_SIZE;
   return ACCEPT_OK;
@@ -272,13 +344,13 @@ size_t accept_payload_offset(const accept_params* p) {
 
 size_t accept_compressed_size(const accept_params* p) {
   if (accept_check_params(p) != ACCEPT_OK) return 0;
-  return accept_payload_offset(p) + (size_t)(4ull * p->k * ((p->n_elems + 31) / 32));
+  return accept_payload_offset(p) + (size_t)(4ull * p->k * n_groups_of(p));
 }
 
 size_t accept_workspace_size(const accept_params* p) {
   if (accept_check_params(p) != ACCEPT_OK) return 0;
   // status word (+ pad); chunks wider than 32768 elements also need one 16-byte record each
-  return 16 + (is_wide(p) ? 16 * (size_t)n_chunks_of(p) : 0);
+  return 16 + ((is_wide(p) || is_strided(p)) ? 16 * (size_t)n_chunks_of(p) : 0);
 }
 
 accept_status accept_compress(const accept_params* p, const float* d_x, void* d_stream, size_t stream_bytes,
@@ -288,6 +360,10 @@ accept_status accept_compress(const accept_params* p, const float* d_x, void* d_
   CodecArgs a = make_args(p, d_stream, d_ws);
   a.x = d_x;
 
+  if (is_strided(p)) {
+    if (!is_aligned(d_x, 32) || !is_aligned(d_ws, 16)) return ACCEPT_ERR_MISALIGNED;
+    return launch_strided(p, a, static_cast<uint8_t*>(d_ws) + 16, static_cast<cudaStream_t>(cuda_stream));
+  }
   if (is_wide(p) && is_aligned(d_x, 32)) {
     if (!is_aligned(d_ws, 16)) return ACCEPT_ERR_MISALIGNED;
     return launch_wide(p, a, static_cast<uint8_t*>(d_ws) + 16, static_cast<cudaStream_t>(cuda_stream));
@@ -325,6 +401,14 @@ accept_status accept_decompress(const accept_params* p, const void* d_stream, si
   if (st != ACCEPT_OK) return st;
   CodecArgs a = make_args(p, const_cast<void*>(d_stream), d_ws);
   a.xhat = d_xhat;
+  if (is_strided(p)) {
+    if (!is_aligned(d_xhat, 32)) return ACCEPT_ERR_MISALIGNED;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (p->range == ACCEPT_RANGE_ABSMAX) launch_strided_decode_for<accept::kAbsMax>(p, a, strided_grid(p), s);
+    else launch_strided_decode_for<accept::kMinMax>(p, a, strided_grid(p), s);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+  }
   const bool aligned = is_aligned(d_xhat, 32);
   const int rounds = 2;  // octets per thread
   KernelFn fn = select_decompress(p, aligned, rounds);
@@ -378,7 +462,7 @@ accept_status accept_parse_header(const void* h_header, accept_params* out) {
   if (!h_header || !out) return ACCEPT_ERR_NULL;
   uint32_t h[8];
   std::memcpy(h, h_header, sizeof(h));
-  if (h[0] != ACCEPT_MAGIC || h[1] != ACCEPT_VERSION || h[7] != 0) return ACCEPT_ERR_BAD_STREAM_HEADER;
+  if (h[0] != ACCEPT_MAGIC || h[1] != ACCEPT_VERSION) return ACCEPT_ERR_BAD_STREAM_HEADER;
   accept_params p{};
   p.n_elems = (uint64_t)h[2] | ((uint64_t)h[3] << 32);
   p.chunk_elems = h[4];
@@ -386,6 +470,7 @@ accept_status accept_parse_header(const void* h_header, accept_params* out) {
   p.range = (int32_t)(h[6] & 0xFF);
   p.round = (int32_t)((h[6] >> 8) & 0xFF);
   p.layout = (int32_t)((h[6] >> 16) & 0xFF);
+  p.group_stride = h[7];
   if ((h[6] >> 24) != 0 || accept_check_params(&p) != ACCEPT_OK) return ACCEPT_ERR_BAD_STREAM_HEADER;
   *out = p;
   return ACCEPT_OK;

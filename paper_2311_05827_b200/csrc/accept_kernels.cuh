@@ -25,6 +25,7 @@ struct CodecArgs {
   uint32_t fast_blocks;   // blocks of the register-resident path; later blocks take the any-shape coder
   uint32_t header_word6;  // range | round<<8 | layout<<16
   uint32_t k;
+  uint32_t group_stride;  // 0, or values per sample when pack groups run along the batch dimension
 };
 
 // Word i of the 32-byte stream header.
@@ -37,7 +38,7 @@ __device__ __forceinline__ uint32_t header_word(const CodecArgs& a, int i) {
     case 4: return a.chunk;
     case 5: return a.k;
     case 6: return a.header_word6;
-    default: return 0u;
+    default: return a.group_stride;
   }
 }
 

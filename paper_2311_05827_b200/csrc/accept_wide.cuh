@@ -90,15 +90,26 @@ __global__ void __launch_bounds__(256) wide_range_kernel(const CodecArgs a, Chun
       merge_into_record<RANGE>(rec + m_first, rg.hi, rg.lo);
     }
   } else {
+    // the tile spans several chunks: a warp's 32 octets of one round (256 consecutive values) usually
+    // still lie in one chunk, then the warp reduces and issues one atomic per record word
 #pragma unroll
-    for (int r = 0; r < R; ++r)
+    for (int r = 0; r < R; ++r) {
+      const uint64_t m = chunk_of(a, (oct0 + r * 256 + tid) * 8);
+      Range<RANGE> rg;
+      rg.init();
       if (in[r]) {
-        Range<RANGE> rg;
-        rg.init();
 #pragma unroll
         for (int e = 0; e < 8; e += 2) rg.add2(v[r][e], v[r][e + 1]);
-        merge_into_record<RANGE>(rec + chunk_of(a, (oct0 + r * 256 + tid) * 8), rg.hi, rg.lo);
       }
+      const uint64_t m_lane0 = __shfl_sync(0xffffffffu, m, 0);
+      const bool uniform = __all_sync(0xffffffffu, in[r] && m == m_lane0);
+      if (uniform) {
+        rg.warp_reduce();
+        if (lane == 0) merge_into_record<RANGE>(rec + m, rg.hi, rg.lo);
+      } else if (in[r]) {
+        merge_into_record<RANGE>(rec + m, rg.hi, rg.lo);
+      }
+    }
   }
 }
 

@@ -1,0 +1,81 @@
+"""GPU parity of pack groups along the batch dimension (the paper's own grouping) against the oracle."""
+import numpy as np
+import pytest
+
+import oracle
+import workloads
+from oracle import (LAYOUT_BITPLANE, LAYOUT_INTERLEAVED, RANGE_ABSMAX, RANGE_MINMAX, ROUND_NEAREST,
+                    ROUND_STOCHASTIC)
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+def modes():
+    out = []
+    for layout in (LAYOUT_INTERLEAVED, LAYOUT_BITPLANE):
+        for k in ((2, 4, 8) if layout == LAYOUT_INTERLEAVED else (2, 3, 4)):
+            for range_ in (RANGE_ABSMAX, RANGE_MINMAX):
+                for round_ in (ROUND_NEAREST, ROUND_STOCHASTIC):
+                    out.append((k, range_, round_, layout))
+    return out
+
+
+def check(x, chunk, stride, k, range_, round_, layout, seed=0, rng_offset=0):
+    import paper_2311_05827_b200 as A
+    n = x.size
+    ref, flag = oracle.compress_strided(x, chunk, k, stride, range_, round_, layout, seed, rng_offset)
+    p = A.Params(n, chunk, k, range_, round_, layout, seed, rng_offset, group_stride=stride)
+    assert A.accept_compressed_size(p) == ref.size
+    d_stream = A.new_stream_buffer(p)
+    d_stream.fill_(0x3C)
+    d_ws = A.new_workspace(p)
+    A.accept_compress(p, torch.from_numpy(x.reshape(-1)).cuda(), d_stream, d_ws)
+    assert (A.accept_last_device_status(d_ws) & 1) == flag
+    got = d_stream.cpu().numpy()
+    if not np.array_equal(got, ref):
+        off = oracle.payload_offset(n, chunk)
+        assert np.array_equal(got[:32], ref[:32]), "header"
+        assert np.array_equal(got[32:off], ref[32:off]), "side words"
+        bad = np.nonzero(got[off:].view(np.uint32) != ref[off:].view(np.uint32))[0]
+        raise AssertionError(f"{bad.size} payload words differ, first {bad[:8]}")
+    d_xhat = torch.full((n,), float("nan"), dtype=torch.float32, device="cuda")
+    A.accept_decompress(p, d_stream, d_xhat, d_ws)
+    assert A.accept_last_device_status(d_ws) == flag
+    want = oracle.decompress_strided(ref, n)
+    assert np.array_equal(d_xhat.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    assert A.accept_parse_header(bytes(got[:32])).group_stride == stride
+
+
+@pytest.mark.parametrize("mode", modes())
+@pytest.mark.parametrize("rows,stride,chunk", [
+    (64, 24, 64 * 24),       # one range for the whole tensor, two full batch groups
+    (40, 16, 96),            # partly filled second batch group, small chunks
+    (33, 2056, 4096),        # chunk boundaries inside rows, more than one block of feature octets
+    (128, 4096, 4096),       # chunk = one sample
+])
+def test_strided_parity(mode, rows, stride, chunk):
+    k, range_, round_, layout = mode
+    x = workloads.random_tensor(rows * stride, rows + k, "normal")
+    check(x, chunk, stride, k, range_, round_, layout, seed=21, rng_offset=5)
+
+
+def test_strided_largest_latent_output_of_the_paper():
+    """Batch 128, 8192 values per sample (the 4096 KB output of Sec. 4.3.1), per-tensor range, both encoders."""
+    x = workloads.generate("cfg2_grad").reshape(32, -1)
+    x = np.concatenate([x, x * np.float32(0.5), -x, x * np.float32(0.25)]).reshape(-1)  # 128 x 32768
+    n = x.size
+    check(x, n, 32768, 4, RANGE_ABSMAX, ROUND_STOCHASTIC, LAYOUT_INTERLEAVED, seed=3)
+    check(x, n, 32768, 2, RANGE_ABSMAX, ROUND_NEAREST, LAYOUT_BITPLANE)
+
+
+def test_strided_nonfinite_and_bad_arguments():
+    import paper_2311_05827_b200 as A
+    x = workloads.random_tensor(64 * 64, 2, "normal")
+    x[70] = np.nan
+    check(x, 1024, 64, 4, RANGE_ABSMAX, ROUND_NEAREST, LAYOUT_BITPLANE)
+    assert A.accept_check_params(A.Params(64 * 64, 1024, 4, group_stride=12)) == 9     # not a multiple of 8
+    assert A.accept_check_params(A.Params(64 * 64 + 8, 1024, 4, group_stride=64)) == 9  # n not a multiple of F
+    assert A.accept_check_params(A.Params(64 * 64, 1024, 8, layout=LAYOUT_BITPLANE, group_stride=64)) == 2
+    assert A.accept_workspace_size(A.Params(64 * 64, 1024, 4, group_stride=64)) == 16 + 16 * 4
