@@ -241,8 +241,11 @@ accept_status launch_strided(const accept_params* p, const CodecArgs& a, uint8_t
 
 // ---- multi-bit quantization --------------------------------------------------------------------
 
+uint64_t mbq_tiles(const accept_mbq_params* p) { return (p->n_elems + accept::kMbqTile - 1) / accept::kMbqTile; }
+
 uint32_t mbq_blocks(const accept_mbq_params* p) {
-  return (uint32_t)((p->n_elems + accept::kMbqTile - 1) / accept::kMbqTile);
+  const uint64_t tiles = mbq_tiles(p);
+  return (uint32_t)(tiles < (uint64_t)accept::kMbqMaxBlocks ? tiles : (uint64_t)accept::kMbqMaxBlocks);
 }
 
 accept::MbqArgs mbq_args(const accept_mbq_params* p, void* d_stream, void* d_ws) {
@@ -256,6 +259,7 @@ accept::MbqArgs mbq_args(const accept_mbq_params* p, void* d_stream, void* d_ws)
   a.alpha_init = reinterpret_cast<float*>(ws + 16);
   a.n = p->n_elems;
   a.n_blocks = mbq_blocks(p);
+  a.n_tiles = mbq_tiles(p);
   a.partial = reinterpret_cast<accept::MbqPartial*>(ws + 64);
   a.residue_sum = reinterpret_cast<double*>(ws + 64 + (size_t)accept::kMbqPartialBytes * a.n_blocks);
   a.k = p->k;
@@ -484,7 +488,7 @@ int accept_bitwidth_schedule(int is_backward, int n_lr_changes) {
 
 accept_status accept_mbq_check_params(const accept_mbq_params* p) {
   if (!p) return ACCEPT_ERR_NULL;
-  if (p->n_elems == 0 || p->n_elems / accept::kMbqTile > 0x7ffffff0ull) return ACCEPT_ERR_BAD_SIZE;
+  if (p->n_elems == 0) return ACCEPT_ERR_BAD_SIZE;
   if (p->k < 2 || p->k > 4) return ACCEPT_ERR_BAD_K;
   if (p->reserved != 0 || p->init > 1) return ACCEPT_ERR_BAD_ENUM;
   return ACCEPT_OK;
@@ -502,7 +506,7 @@ size_t accept_mbq_compressed_size(const accept_mbq_params* p) {
 
 size_t accept_mbq_workspace_size(const accept_mbq_params* p) {
   if (accept_mbq_check_params(p) != ACCEPT_OK) return 0;
-  // status + residue coefficients (64 bytes), one 128-byte record and one double per block
+  // status + residue coefficients (64 bytes), one 128-byte record and one double per block (at most 1184 blocks)
   return 64 + (size_t)(accept::kMbqPartialBytes + 8) * mbq_blocks(p);
 }
 

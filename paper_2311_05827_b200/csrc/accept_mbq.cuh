@@ -19,6 +19,7 @@ constexpr int kMbqRounds = 4;                      // octets per thread
 constexpr int kMbqTile = kMbqRounds * 256 * 8;     // elements per block
 constexpr int kMbqPartialBytes = 128;              // per-block record in the workspace
 constexpr int kMbqFinalizeThreads = 256;           // threads of the single finalize block
+constexpr int kMbqMaxBlocks = 1184;                // 8 per SM on 148 SMs; fixed, so sums repeat on any device
 
 // Per-block partial sums (one 128-byte record per block of the encode pass).
 struct MbqPartial {
@@ -43,7 +44,8 @@ struct MbqArgs {
   float* alpha_init;        // workspace + 16: coefficients found by the residue passes (init)
   double* residue_sum;      // workspace + 32: scratch of the residue passes
   uint64_t n;
-  uint32_t n_blocks;
+  uint64_t n_tiles;         // tiles of kMbqTile elements
+  uint32_t n_blocks;        // blocks of the encode / residue passes = records in the workspace
   uint32_t k, batch_index, init;
 };
 
@@ -169,9 +171,10 @@ __global__ void __launch_bounds__(256) mbq_residue_sum_kernel(const MbqArgs a, i
   for (int i = 0; i < K; ++i) alpha[i] = (i < j) ? a.alpha_init[i] : 0.0f;
   const uint64_t n_oct = (a.n + 7) / 8;
   double acc = 0.0;
+  for (uint64_t tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x)
 #pragma unroll
   for (int r = 0; r < kMbqRounds; ++r) {
-    const uint64_t oct = (uint64_t)blockIdx.x * (kMbqRounds * 256) + r * 256 + tid;
+    const uint64_t oct = tile * (kMbqRounds * 256) + r * 256 + tid;
     if (oct < n_oct) {
       float v[8];
       mbq_ld_octet(a.x, a.n, oct, v);
@@ -235,10 +238,14 @@ __global__ void __launch_bounds__(256) mbq_encode_kernel(const MbqArgs a) {
 #pragma unroll
   for (int j = 0; j < K; ++j) plus[j] = 0.0;
 
+  const int q = lane & 3;
+  // a block walks over tiles with a stride of the grid and keeps its sums in registers: the block-level
+  // reduction and the record in the workspace are paid once per block, not once per tile
+  for (uint64_t tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x) {
   float v[kMbqRounds][8];
 #pragma unroll
   for (int r = 0; r < kMbqRounds; ++r) {
-    const uint64_t oct = (uint64_t)blockIdx.x * (kMbqRounds * 256) + r * 256 + tid;
+    const uint64_t oct = tile * (kMbqRounds * 256) + r * 256 + tid;
     if (oct < n_oct) {
       mbq_ld_octet(a.x, a.n, oct, v[r]);
     } else {
@@ -246,10 +253,9 @@ __global__ void __launch_bounds__(256) mbq_encode_kernel(const MbqArgs a) {
       for (int e = 0; e < 8; ++e) v[r][e] = 0.0f;
     }
   }
-  const int q = lane & 3;
 #pragma unroll
   for (int r = 0; r < kMbqRounds; ++r) {
-    const uint64_t oct = (uint64_t)blockIdx.x * (kMbqRounds * 256) + r * 256 + tid;
+    const uint64_t oct = tile * (kMbqRounds * 256) + r * 256 + tid;
     // elements of this octet that exist (8 for all but the last octets of the tensor)
     const int valid = (oct * 8 + 8 <= a.n) ? 8 : ((oct * 8 < a.n) ? (int)(a.n - oct * 8) : 0);
     uint32_t c[8];
@@ -287,6 +293,7 @@ __global__ void __launch_bounds__(256) mbq_encode_kernel(const MbqArgs a) {
       my_differ[d - 1] += __popc(w ^ other);
     }
   }
+  }  // tiles
 
   // block sums in a fixed order: lanes by butterfly, warps one after the other
 #pragma unroll
