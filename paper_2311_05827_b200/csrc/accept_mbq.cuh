@@ -348,8 +348,8 @@ __global__ void __launch_bounds__(256) mbq_encode_kernel(const MbqArgs a) {
 // words and alpha_next.  One block.
 template <int K>
 __global__ void __launch_bounds__(kMbqFinalizeThreads) mbq_finalize_kernel(const MbqArgs a) {
-  __shared__ double s_dbl[kMbqFinalizeThreads][K + 1];
-  __shared__ unsigned long long s_int[kMbqFinalizeThreads][10];
+  __shared__ double s_dbl[kMbqFinalizeThreads / 32][K + 1];
+  __shared__ unsigned long long s_int[kMbqFinalizeThreads / 32][10];
   const int tid = threadIdx.x;
   double d[K + 1];
   unsigned long long c[10];
@@ -367,17 +367,27 @@ __global__ void __launch_bounds__(kMbqFinalizeThreads) mbq_finalize_kernel(const
 #pragma unroll
     for (int j = 0; j < 6; ++j) c[4 + j] += p.differ[j];
   }
+  // fixed-order tree: butterfly over the lanes of each warp, then the warps one after the other
 #pragma unroll
-  for (int j = 0; j <= K; ++j) s_dbl[tid][j] = d[j];
+  for (int j = 0; j <= K; ++j) d[j] = warp_sum(d[j]);
 #pragma unroll
-  for (int j = 0; j < 10; ++j) s_int[tid][j] = c[j];
+  for (int j = 0; j < 10; ++j) {
+#pragma unroll
+    for (int sh = 16; sh >= 1; sh >>= 1) c[j] += __shfl_xor_sync(0xffffffffu, c[j], sh);
+  }
+  if ((tid & 31) == 0) {
+#pragma unroll
+    for (int j = 0; j <= K; ++j) s_dbl[tid >> 5][j] = d[j];
+#pragma unroll
+    for (int j = 0; j < 10; ++j) s_int[tid >> 5][j] = c[j];
+  }
   __syncthreads();
   if (tid != 0) return;
 #pragma unroll
   for (int j = 0; j <= K; ++j) d[j] = 0.0;
 #pragma unroll
   for (int j = 0; j < 10; ++j) c[j] = 0;
-  for (int i = 0; i < kMbqFinalizeThreads; ++i) {
+  for (int i = 0; i < kMbqFinalizeThreads / 32; ++i) {
 #pragma unroll
     for (int j = 0; j <= K; ++j) d[j] += s_dbl[i][j];
 #pragma unroll
