@@ -381,7 +381,7 @@ def sweep(A, torch, peak, args):
     """All five workloads, headline modes: per-kernel time and HBM fraction."""
     rows = []
     for name, spec in workloads.TENSORS.items():
-        if spec.n * 4 > args.sweep_max_bytes:
+        if spec.n * 4 > args.sweep_max_bytes or (args.sweep_only and name != args.sweep_only):
             continue
         x_host = workloads.generate(name)
         for mode in spec.headline:
@@ -412,7 +412,42 @@ def sweep(A, torch, peak, args):
             rows.append(sweep_per_tensor(A, torch, peak, name, spec, x_host))
         if name == "cfg3_act":
             rows.extend(sweep_mbq(A, torch, peak, name, spec, x_host))
+            rows.append(sweep_batch_groups(A, torch, peak, name, spec, x_host))
     return rows
+
+
+def sweep_batch_groups(A, torch, peak, name, spec, x_host):
+    """Pack groups along the batch dimension (the paper's grouping): the tensor as batch x (values per sample)."""
+    mode = spec.headline[0]
+    stride = spec.n // spec.shape[0]
+    p = A.Params(spec.n, spec.chunk, mode.k, mode.range, mode.round, mode.layout, spec.seed, 0, group_stride=stride)
+    copies = 2
+    x = [torch.from_numpy(x_host).cuda() for _ in range(copies)]
+    st = [A.new_stream_buffer(p) for _ in range(copies)]
+    xh = [torch.empty(spec.n, dtype=torch.float32, device="cuda") for _ in range(copies)]
+    ws = A.new_workspace(p)
+    times = []
+    for fn in (lambda j: A.accept_compress(p, x[j], st[j], ws), lambda j: A.accept_decompress(p, st[j], xh[j], ws)):
+        for i in range(3):
+            fn(i % copies)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(20):
+            fn(i % copies)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) / 20)
+    assert A.accept_last_device_status(ws) == 0
+    ms_c, ms_d = times
+    alg_c, alg_d = spec.n * (8.0 + mode.k / 8.0), spec.n * (4.0 + mode.k / 8.0)
+    row = {"workload": name, "mode": mode_name(mode) + "-batch-groups", "mbytes": spec.n * 4 / 2 ** 20, "copies": copies,
+           "group_stride": stride, "compress_ms": ms_c, "decompress_ms": ms_d, "compress_bytes_per_element": 8.0 + mode.k / 8.0,
+           "compress_frac_measured": alg_c / ms_c / 1e6 / peak, "decompress_frac_measured": alg_d / ms_d / 1e6 / peak}
+    print("# %-12s %-34s c %8.4f ms %6.1f%%  d %8.4f ms %6.1f%% (of measured copy bw)" %
+          (name, ("k%d-batch-groups-%dx%d" % (mode.k, spec.shape[0], stride))[:34], ms_c, 100 * row["compress_frac_measured"],
+           ms_d, 100 * row["decompress_frac_measured"]), file=sys.stderr)
+    return row
 
 
 def sweep_per_tensor(A, torch, peak, name, spec, x_host):
@@ -515,6 +550,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(workloads.TENSORS))
     ap.add_argument("--sweep", action="store_true", help="also time every workload's headline modes")
     ap.add_argument("--sweep-max-bytes", type=int, default=1 << 30)
+    ap.add_argument("--sweep-only", default=None, choices=sorted(workloads.TENSORS), help="restrict the sweep to one tensor")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernels-only", action="store_true",
                     help="profiling runs: skip the host-buffer and CPU-oracle legs (the line is then not a bench result)")

@@ -32,7 +32,7 @@ __device__ __forceinline__ void transpose4x4(uint32_t a0, uint32_t a1, uint32_t 
 constexpr int kStridedOctetsPerBlock = 64;
 
 template <int K, int LAYOUT, int RANGE, int ROUND>
-__global__ void __launch_bounds__(256) strided_encode_kernel(const CodecArgs a, const ChunkRecord* rec) {
+__global__ void __launch_bounds__(256, 4) strided_encode_kernel(const CodecArgs a, const ChunkRecord* rec) {
   const int tid = threadIdx.x, lane = tid & 31, sub = tid & 3;
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid < 8) {
     a.header[tid] = header_word(a, tid);
@@ -46,33 +46,43 @@ __global__ void __launch_bounds__(256) strided_encode_kernel(const CodecArgs a, 
   const uint64_t word0 = (g * F + (uint64_t)fo * 8) * K;  // first word of feature 8*fo of this batch group
   const Rng rng{(uint32_t)a.seed, (uint32_t)(a.seed >> 32)};
 
-  float v[8][8];
-  bool in[8];
-#pragma unroll
-  for (int r = 0; r < 8; ++r) {
-    const uint64_t row = g * 32 + sub * 8 + r;
-    in[r] = active && row < n_rows;
-    if (in[r]) ld_octet(a.x + row * F + (uint64_t)fo * 8, v[r]);
-  }
   uint32_t xlo[8], xhi[8];  // per row: codes of features 0..3 / 4..7
+  // four rows at a time: 128 bytes in flight per thread at half the registers, so that more blocks
+  // stay resident (the kernel waits on memory, not on arithmetic)
 #pragma unroll
-  for (int r = 0; r < 8; ++r) {
-    xlo[r] = 0; xhi[r] = 0;
-    if (in[r]) {
-      const uint64_t i0 = (g * 32 + sub * 8 + r) * F + (uint64_t)fo * 8;
-      const uint4 raw = __ldg(reinterpret_cast<const uint4*>(rec + chunk_of(a, i0)));
-      Scale sc;
-      sc.s = 0.0f; sc.o = 0.0f;
-      sc.inv = __uint_as_float(raw.z);
-      sc.base = __uint_as_float(raw.w);
-      sc.nonfinite = raw.x != 0u;
-      if (sc.nonfinite) {
+  for (int half = 0; half < 2; ++half) {
+    float v[4][8];
+    bool in[4];
+    uint4 raw[4];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) v[r][e] = 0.0f;
+    for (int r = 0; r < 4; ++r) {
+      const uint64_t row = g * 32 + sub * 8 + half * 4 + r;
+      in[r] = active && row < n_rows;
+      if (in[r]) {
+        const uint64_t i0 = row * F + (uint64_t)fo * 8;
+        ld_octet(a.x + i0, v[r]);
+        raw[r] = __ldg(reinterpret_cast<const uint4*>(rec + chunk_of(a, i0)));
       }
-      RngThread rt;
-      if (ROUND == kStochastic) rt.init(rng, a.rng_offset + i0, 8u);
-      quantize_octet<K, RANGE, ROUND>(v[r], sc, rng, rt, 0u, xlo[r], xhi[r]);
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int rr = half * 4 + r;
+      xlo[rr] = 0; xhi[rr] = 0;
+      if (in[r]) {
+        const uint64_t i0 = (g * 32 + sub * 8 + rr) * F + (uint64_t)fo * 8;
+        Scale sc;
+        sc.s = 0.0f; sc.o = 0.0f;
+        sc.inv = __uint_as_float(raw[r].z);
+        sc.base = __uint_as_float(raw[r].w);
+        sc.nonfinite = raw[r].x != 0u;
+        if (sc.nonfinite) {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) v[r][e] = 0.0f;
+        }
+        RngThread rt;
+        if (ROUND == kStochastic) rt.init(rng, a.rng_offset + i0, 8u);
+        quantize_octet<K, RANGE, ROUND>(v[r], sc, rng, rt, 0u, xlo[rr], xhi[rr]);
+      }
     }
   }
   // rows x features -> features x rows
