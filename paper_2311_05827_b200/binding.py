@@ -62,9 +62,14 @@ class Params:
     rng_offset: int = 0
     group_stride: int = 0
 
+    def __post_init__(self):
+        # the C struct is built once: calls only pass a reference to it
+        object.__setattr__(self, "_c", CParams(self.n_elems, self.chunk_elems, self.k, self.range, self.round,
+                                               self.layout, self.group_stride, self.seed & (2**64 - 1),
+                                               self.rng_offset & (2**64 - 1)))
+
     def c(self) -> CParams:
-        return CParams(self.n_elems, self.chunk_elems, self.k, self.range, self.round, self.layout, self.group_stride,
-                       self.seed & (2**64 - 1), self.rng_offset & (2**64 - 1))
+        return self._c
 
 
 class CMbqParams(ctypes.Structure):
