@@ -372,3 +372,47 @@ def test_workloads_sampled_parity_sweep(name):
         assert [int(v) for v in hdr[:6]] == [0x54504341, 1, n & 0xFFFFFFFF, n >> 32, chunk, m.k]
         assert bool(torch.isfinite(d_xhat).all())
         del d_stream, d_xhat
+
+
+def test_parity_beyond_32_bit_element_indices():
+    """A tensor of more than 2^32 elements (17 GB): element indices, byte offsets and random-number
+    counters all pass 2^32.  Values are drawn on the GPU; the oracle recomputes runs of chunks around
+    the interesting indices from slices copied back (chunks are independent, counters are indices)."""
+    A = _lib()
+    free, _ = torch.cuda.mem_get_info()
+    n, chunk = (1 << 32) + 4096 * 5 + 123, 4096
+    if free < 45 * (1 << 30):
+        pytest.skip("needs about 40 GB of free device memory")
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1234)
+    d_x = torch.empty(n, dtype=torch.float32, device="cuda")
+    step = 1 << 28
+    for s in range(0, n, step):
+        d_x[s:s + step].normal_(generator=gen)
+    for k, round_, layout in [(4, ROUND_STOCHASTIC, LAYOUT_INTERLEAVED), (2, ROUND_NEAREST, LAYOUT_BITPLANE)]:
+        p = A.Params(n, chunk, k, RANGE_ABSMAX, round_, layout, seed=99, rng_offset=0)
+        d_stream, d_ws = A.new_stream_buffer(p), A.new_workspace(p)
+        A.accept_compress(p, d_x, d_stream, d_ws)
+        d_xhat = torch.empty(n, dtype=torch.float32, device="cuda")
+        A.accept_decompress(p, d_stream, d_xhat, d_ws)
+        assert A.accept_last_device_status(d_ws) == 0
+        off = A.accept_payload_offset(p)
+        wpc = chunk * k // 32
+        n_chunks = -(-n // chunk)
+        for c0 in (0, (1 << 31) // chunk - 2, (1 << 32) // chunk - 3, n_chunks - 4):
+            c1 = min(c0 + 4, n_chunks)
+            e0, e1 = c0 * chunk, min(c1 * chunk, n)
+            xs = d_x[e0:e1].cpu().numpy()
+            ref, _ = oracle.compress(xs, chunk, k, RANGE_ABSMAX, round_, layout, 99, e0)
+            _, meta_r, pay_r = oracle.split_stream(ref, xs.size, chunk)
+            meta_g = d_stream[32 + 8 * c0:32 + 8 * c1].cpu().numpy().view(np.float32).reshape(-1, 2)
+            assert np.array_equal(meta_g.view(np.uint32), meta_r.view(np.uint32))
+            b0 = off + 4 * wpc * c0
+            pay_g = d_stream[b0:b0 + 4 * pay_r.size].cpu().numpy().view(np.uint32)
+            assert np.array_equal(pay_g, pay_r)
+            want = oracle.decompress(ref, xs.size)
+            assert np.array_equal(d_xhat[e0:e1].cpu().numpy().view(np.uint32), want.view(np.uint32))
+        hdr = d_stream[:32].cpu().numpy().view(np.uint32)
+        assert int(hdr[2]) == n & 0xFFFFFFFF and int(hdr[3]) == 1
+        del d_stream, d_xhat
+        torch.cuda.empty_cache()
