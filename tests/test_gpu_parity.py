@@ -47,7 +47,7 @@ def gpu_decompress(p, stream_np_or_dev, d_ws=None):
 
 
 def assert_float_parity(xhat_gpu, xhat_ref, x, chunk):
-    """spec tolerance, then the stricter bit-exact check."""
+    """Stated tolerance (1e-6 of the chunk's max - min), then the stricter bit-exact check."""
     n = x.size
     m = -(-n // chunk)
     pad = m * chunk - n
