@@ -95,9 +95,10 @@ typedef enum { ACCEPT_LAYOUT_INTERLEAVED = 0, ACCEPT_LAYOUT_BITPLANE = 1 } accep
  *                bytes per chunk more, as for chunk_elems > 32768).  Header word 7 carries F.
  *   seed, rng_offset  STOCHASTIC only.  Element i draws
  *                  U_i = (g >> 8) * 2^-24,
- *                  g   = h if ctr is even, h * 0x9E3779B1 (mod 2^32) if ctr is odd,
+ *                  g   = h * M[ctr & 3] (mod 2^32),  M = {1, 0x9E3779B1, 0x85EBCA77, 0xC2B2AE3D},
  *                  h   = fmix32( lo32(j) ^ fmix32( hi32(j) ^ lo32(seed) ^ 0x9E3779B9 ) ^ hi32(seed) ),
- *                  j   = ctr >> 1,  ctr = rng_offset + i (mod 2^64),
+ *                  j   = ctr >> 2,  ctr = rng_offset + i (mod 2^64)
+ *                (four neighbouring counters share one hash; each takes it times its own odd constant),
  *                fmix32 = the 32-bit finaliser of MurmurHash3:
  *                  h ^= h>>16; h *= 0x85EBCA6B; h ^= h>>13; h *= 0xC2B2AE35; h ^= h>>16.
  *                The same (seed, rng_offset) reproduces the same stream; advance rng_offset by

@@ -17,8 +17,7 @@
  *   - "dividing by the scaling factor" is computed as a product with inv = L/c (one division per
  *     chunk); pinned against true division in the tests;
  *   - nearest rounding is IEEE round-half-to-even;
- *   - the uniform generator of Eq. 7 is counter based (MurmurHash3's 32-bit finaliser, one hash per
- *     pair of counters, see oracle_rng_hash below); U has 24 bits; pr = t - floor(t) and the test
+ *   - the uniform generator of Eq. 7 is counter based (MurmurHash3's 32-bit finaliser, see oracle_rng_hash below: one hash per four counters); U has 24 bits; pr = t - floor(t) and the test
  *     U < pr are exact;
  *   - bit order in a packed word is LSB first (element t of a group <-> bit t).  The paper's only
  *     worked example, (00110110)_2 = 54, fixes the value of a word, not which element is the MSB:
@@ -69,14 +68,16 @@ static uint32_t fmix32(uint32_t h) {
   return h;
 }
 
-/* 32 random bits for counter ctr under seed.  Counters 2j and 2j+1 share the hash of their pair
- * index j; the odd one multiplies it by an odd constant (a bijection of the 32-bit word). */
+/* 32 random bits for counter ctr under seed.  Counters 4j .. 4j+3 share the hash of their quad
+ * index j; counter 4j+m multiplies it by the m-th of four odd constants (1 for m = 0), each a
+ * bijection of the 32-bit word. */
 uint32_t oracle_rng_hash(uint64_t seed, uint64_t ctr) {
-  uint64_t pair = ctr >> 1;
-  /* the constant keeps seed 0, pair 0 off the fixed point fmix32(0) = 0 */
-  uint32_t inner = fmix32((uint32_t)(pair >> 32) ^ (uint32_t)seed ^ 0x9E3779B9u);
-  uint32_t h = fmix32((uint32_t)pair ^ inner ^ (uint32_t)(seed >> 32));
-  return (ctr & 1) ? h * 0x9E3779B1u : h;
+  static const uint32_t lane_mul[4] = {1u, 0x9E3779B1u, 0x85EBCA77u, 0xC2B2AE3Du};
+  uint64_t quad = ctr >> 2;
+  /* the constant keeps seed 0, quad 0 off the fixed point fmix32(0) = 0 */
+  uint32_t inner = fmix32((uint32_t)(quad >> 32) ^ (uint32_t)seed ^ 0x9E3779B9u);
+  uint32_t h = fmix32((uint32_t)quad ^ inner ^ (uint32_t)(seed >> 32));
+  return h * lane_mul[ctr & 3];
 }
 
 /* U in [0,1) on a grid of 2^-24: the top 24 random bits. */

@@ -149,44 +149,49 @@ __device__ __forceinline__ uint32_t fmix32(uint32_t h) {
   return h;
 }
 
-// Two neighbouring counters share one hash: the element with the even counter takes the hashed
-// word as it is, the odd one takes it times kPairMul (an odd constant, so a bijection of the word).
-// This halves the per-element cost of the integer hash, which runs on the half-rate ALU pipe and
-// is what bounds stochastic rounding.
-constexpr uint32_t kPairMul = 0x9E3779B1u;
+// Four neighbouring counters (4j .. 4j+3) share one hash: counter 4j+m takes the hashed word times
+// kLaneMul[m] (odd constants, so each is a bijection of the word; m = 0 takes it as it is).  The
+// integer hash runs on the half-rate ALU pipe and is what bounds stochastic rounding; shared by
+// four elements it costs two ALU instructions per element, the extra products run on the FMA pipe.
+__device__ __forceinline__ uint32_t lane_word(uint32_t h, int m) {
+  return m == 0 ? h : h * (m == 1 ? 0x9E3779B1u : (m == 2 ? 0x85EBCA77u : 0xC2B2AE3Du));
+}
 
 struct Rng {
   uint32_t seed_lo, seed_hi;
-  // key for all pairs that share the upper 32 bits of their pair index; the constant keeps
-  // seed 0 / pair 0 off the fixed point fmix32(0) = 0
-  __device__ __forceinline__ uint32_t key(uint32_t pair_hi) const {
-    return fmix32(pair_hi ^ seed_lo ^ 0x9E3779B9u) ^ seed_hi;
+  // key for all quads that share the upper 32 bits of their quad index; the constant keeps
+  // seed 0 / quad 0 off the fixed point fmix32(0) = 0
+  __device__ __forceinline__ uint32_t key(uint32_t quad_hi) const {
+    return fmix32(quad_hi ^ seed_lo ^ 0x9E3779B9u) ^ seed_hi;
   }
-  // hashed word of a pair
-  __device__ __forceinline__ static uint32_t pair_hash(uint32_t pair_lo, uint32_t key) { return fmix32(pair_lo ^ key); }
-  // 32 random bits of any counter (the octet path below shares the pair hashes instead)
+  // hashed word of a quad
+  __device__ __forceinline__ static uint32_t quad_hash(uint32_t quad_lo, uint32_t key) { return fmix32(quad_lo ^ key); }
+  // 32 random bits of any counter (the octet path below shares the quad hashes instead)
   __device__ __forceinline__ uint32_t word(uint64_t ctr) const {
-    const uint64_t pair = ctr >> 1;
-    const uint32_t h = pair_hash((uint32_t)pair, key((uint32_t)(pair >> 32)));
-    return (ctr & 1) ? h * kPairMul : h;
+    const uint64_t quad = ctr >> 2;
+    const uint32_t h = quad_hash((uint32_t)quad, key((uint32_t)(quad >> 32)));
+    const int m = (int)(ctr & 3);
+    return m == 0 ? h : h * (m == 1 ? 0x9E3779B1u : (m == 2 ? 0x85EBCA77u : 0xC2B2AE3Du));
   }
 };
 
-// What a thread works out once for all the octets it quantizes stochastically: the pair index and
-// key of its first counter, the counter's parity (the same for every octet, octets start 8 apart)
-// and whether the low word of the pair index stays clear of a wrap over the thread's whole span.
+// What a thread works out once for all the octets it quantizes stochastically: the quad index and
+// key of its first counter, the counter's position in its quad (the same for every octet, octets
+// start 8 apart) and whether the low word of the quad index stays clear of a wrap over the thread's
+// whole span.
 struct RngThread {
   uint64_t ctr_first;
-  uint32_t pair_lo, key;
-  bool odd, fast;
+  uint32_t quad_lo, key;
+  int off;    // ctr_first & 3
+  bool fast;
   // span = distance, in counters, from the thread's first counter to one past its last
   __device__ __forceinline__ void init(const Rng& rng, uint64_t ctr, uint32_t span) {
     ctr_first = ctr;
-    const uint64_t pair = ctr >> 1;
-    pair_lo = (uint32_t)pair;
-    key = rng.key((uint32_t)(pair >> 32));
-    odd = ctr & 1;
-    fast = pair_lo <= 0xFFFFFFFFu - (span / 2 + 1);
+    const uint64_t quad = ctr >> 2;
+    quad_lo = (uint32_t)quad;
+    key = rng.key((uint32_t)(quad >> 32));
+    off = (int)(ctr & 3);
+    fast = quad_lo <= 0xFFFFFFFFu - (span / 4 + 2);
   }
 };
 
@@ -236,18 +241,18 @@ __device__ __forceinline__ uint32_t pack_bytes(uint32_t b0, uint32_t b1, uint32_
   return __byte_perm(p01, p23, 0x5410);
 }
 
-// Stochastic codes of an octet whose first counter has parity ODD; pair_lo/key address its first pair.
-template <int K, int RANGE, int ODD>
-__device__ __forceinline__ void quantize_octet_stochastic(const float (&v)[8], const Scale& sc, uint32_t pair_lo,
+// Stochastic codes of an octet whose first counter sits at position OFF of its quad; quad_lo/key
+// address that quad.
+template <int K, int RANGE, int OFF>
+__device__ __forceinline__ void quantize_octet_stochastic(const float (&v)[8], const Scale& sc, uint32_t quad_lo,
                                                           uint32_t key, uint32_t (&b)[8]) {
-  uint32_t h[4 + ODD];
+  constexpr int NQ = (OFF == 0) ? 2 : 3;
+  uint32_t h[NQ];
 #pragma unroll
-  for (int p = 0; p < 4 + ODD; ++p) h[p] = Rng::pair_hash(pair_lo + p, key);
+  for (int p = 0; p < NQ; ++p) h[p] = Rng::quad_hash(quad_lo + p, key);
 #pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    const uint32_t w = h[(e + ODD) >> 1];
-    b[e] = quantize_stochastic_word<K, RANGE>(v[e], sc, ((e + ODD) & 1) ? w * kPairMul : w);
-  }
+  for (int e = 0; e < 8; ++e)
+    b[e] = quantize_stochastic_word<K, RANGE>(v[e], sc, lane_word(h[(e + OFF) >> 2], (e + OFF) & 3));
 }
 
 // Quantizes an octet.  xlo holds the codes of elements 0..3 one per byte, xhi those of 4..7.
@@ -258,9 +263,12 @@ __device__ __forceinline__ void quantize_octet(const float (&v)[8], const Scale&
   uint32_t b[8];
   if (ROUND == kStochastic) {
     if (rt.fast) {
-      if (rt.odd) quantize_octet_stochastic<K, RANGE, 1>(v, sc, rt.pair_lo + delta / 2, rt.key, b);
-      else quantize_octet_stochastic<K, RANGE, 0>(v, sc, rt.pair_lo + delta / 2, rt.key, b);
-    } else {  // the pair index's low word (or the counter itself) wraps somewhere in this thread's span
+      const uint32_t q0 = rt.quad_lo + delta / 4;  // delta is a multiple of 8
+      if (rt.off == 0) quantize_octet_stochastic<K, RANGE, 0>(v, sc, q0, rt.key, b);
+      else if (rt.off == 1) quantize_octet_stochastic<K, RANGE, 1>(v, sc, q0, rt.key, b);
+      else if (rt.off == 2) quantize_octet_stochastic<K, RANGE, 2>(v, sc, q0, rt.key, b);
+      else quantize_octet_stochastic<K, RANGE, 3>(v, sc, q0, rt.key, b);
+    } else {  // the quad index's low word (or the counter itself) wraps somewhere in this thread's span
 #pragma unroll
       for (int e = 0; e < 8; ++e) b[e] = quantize_stochastic_word<K, RANGE>(v[e], sc, rng.word(rt.ctr_first + delta + e));
     }

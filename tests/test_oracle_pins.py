@@ -341,27 +341,34 @@ def fmix32_py(h):
     return h
 
 
-def test_rng_pair_structure_and_finaliser():
-    """Counters 2j, 2j+1 share one finaliser output; the odd one is that word times an odd constant
-    (a bijection, so each stays uniform); seed 0 / counter 0 does not sit on fmix32(0) = 0."""
+LANE_MUL = (1, 0x9E3779B1, 0x85EBCA77, 0xC2B2AE3D)
+
+
+def test_rng_quad_structure_and_finaliser():
+    """Counters 4j .. 4j+3 share one finaliser output; counter 4j+m is that word times the m-th odd
+    constant (a bijection, so each stays uniform); seed 0 / counter 0 does not sit on fmix32(0) = 0."""
     assert fmix32_py(0) == 0 and fmix32_py(1) == 0x514E28B7  # published finaliser: fixed point and one value
     for seed, j in [(0, 0), (5, 77), (2 ** 63 + 9, 2 ** 40 + 3)]:
-        even, odd = oracle.rng_hash(seed, 2 * j), oracle.rng_hash(seed, 2 * j + 1)
-        assert odd == (even * 0x9E3779B1) & 0xFFFFFFFF
         inner = fmix32_py(((j >> 32) ^ (seed & 0xFFFFFFFF) ^ 0x9E3779B9) & 0xFFFFFFFF)
-        assert even == fmix32_py(((j & 0xFFFFFFFF) ^ inner ^ (seed >> 32)) & 0xFFFFFFFF)
-    assert oracle.rng_hash(0, 0) != 0 and oracle.rng_hash(0, 1) != 0
+        h = fmix32_py(((j & 0xFFFFFFFF) ^ inner ^ (seed >> 32)) & 0xFFFFFFFF)
+        for m in range(4):
+            assert oracle.rng_hash(seed, 4 * j + m) == (h * LANE_MUL[m]) & 0xFFFFFFFF
+    assert all(oracle.rng_hash(0, m) != 0 for m in range(4)) and all(v % 2 == 1 for v in LANE_MUL)
 
 
-def test_rng_pairs_are_jointly_uniform():
-    """The two numbers of a pair: no correlation, and a 16 x 16 chi-square of (U_even, U_odd)."""
+def test_rng_quads_are_jointly_uniform():
+    """The four numbers of a quad, pair by pair: no correlation, and a 16 x 16 chi-square."""
     n = 1 << 16
-    u = np.array([oracle.rng_uniform(3, i) for i in range(2 * n)]).reshape(n, 2)
-    assert abs(np.corrcoef(u[:, 0], u[:, 1])[0, 1]) < 0.02
-    cells = (u[:, 0] * 16).astype(int) * 16 + (u[:, 1] * 16).astype(int)
-    hist = np.bincount(cells, minlength=256)
-    chi2 = ((hist - n / 256) ** 2 / (n / 256)).sum()
-    assert chi2 < 360  # 255 dof: mean 255, sd 22.6
+    u = np.array([oracle.rng_uniform(3, i) for i in range(4 * n)]).reshape(n, 4)
+    for a in range(4):
+        for b in range(a + 1, 4):
+            assert abs(np.corrcoef(u[:, a], u[:, b])[0, 1]) < 0.02
+            cells = (u[:, a] * 16).astype(int) * 16 + (u[:, b] * 16).astype(int)
+            hist = np.bincount(cells, minlength=256)
+            chi2 = ((hist - n / 256) ** 2 / (n / 256)).sum()
+            assert chi2 < 360, (a, b, chi2)  # 255 dof: mean 255, sd 22.6
+    # sums of the four numbers of a quad behave like sums of independent uniforms (variance 4/12)
+    assert abs(u.sum(axis=1).var() - 4 / 12) < 0.01
     # the low bits of the 24 used are as balanced as the high ones
     r = (u * 2 ** 24).astype(np.int64)
     for b in range(24):
