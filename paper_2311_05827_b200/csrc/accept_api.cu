@@ -6,6 +6,7 @@
 #include <atomic>
 #include <cstring>
 #include <mutex>
+#include <utility>
 
 #include "accept_kernels.cuh"
 #include "accept_wide.cuh"
@@ -64,6 +65,23 @@ CodecArgs make_args(const accept_params* p, void* d_stream, void* d_ws) {
   a.k = p->k;
   a.group_stride = p->group_stride;
   return a;
+}
+
+// Launch with programmatic stream serialization: every kernel of this library starts with
+// grid_dependency_handshake(), so it may be scheduled while its predecessor in the stream drains.
+template <typename... Params, typename... Args>
+cudaError_t launch_overlapped(void (*fn)(Params...), dim3 grid, unsigned block, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(block, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, fn, std::forward<Args>(args)...);
 }
 
 // ---- kernel tables -------------------------------------------------------------------------
@@ -139,8 +157,8 @@ KernelFn select_decompress(const accept_params* p, bool aligned, int rounds) {
 
 template <int K, int LAYOUT, int RANGE>
 void launch_wide_encode(int round, const CodecArgs& a, const accept::ChunkRecord* rec, unsigned grid, cudaStream_t s) {
-  if (round == accept::kNearest) accept::wide_encode_kernel<K, LAYOUT, RANGE, accept::kNearest, 2><<<grid, 256, 0, s>>>(a, rec);
-  else accept::wide_encode_kernel<K, LAYOUT, RANGE, accept::kStochastic, 2><<<grid, 256, 0, s>>>(a, rec);
+  if (round == accept::kNearest) launch_overlapped(accept::wide_encode_kernel<K, LAYOUT, RANGE, accept::kNearest, 2>, dim3(grid), 256, s, a, rec);
+  else launch_overlapped(accept::wide_encode_kernel<K, LAYOUT, RANGE, accept::kStochastic, 2>, dim3(grid), 256, s, a, rec);
 }
 
 template <int RANGE>
@@ -167,12 +185,12 @@ accept_status launch_wide(const accept_params* p, const CodecArgs& a, uint8_t* r
   const unsigned fin_grid = (unsigned)((a.n_chunks + 255) / 256);
   const unsigned enc_grid = (unsigned)((((p->n_elems + 31) / 32) * 4 + 2 * 256 - 1) / (2 * 256));
   if (p->range == ACCEPT_RANGE_ABSMAX) {
-    accept::wide_range_kernel<accept::kAbsMax, 4><<<range_grid, 256, 0, s>>>(a, rec);
-    accept::wide_finalize_kernel<accept::kAbsMax><<<fin_grid, 256, 0, s>>>(a, rec);
+    launch_overlapped(accept::wide_range_kernel<accept::kAbsMax, 4>, dim3(range_grid), 256, s, a, rec);
+    launch_overlapped(accept::wide_finalize_kernel<accept::kAbsMax>, dim3(fin_grid), 256, s, a, rec);
     launch_wide_encode_for<accept::kAbsMax>(p, a, rec, enc_grid, s);
   } else {
-    accept::wide_range_kernel<accept::kMinMax, 4><<<range_grid, 256, 0, s>>>(a, rec);
-    accept::wide_finalize_kernel<accept::kMinMax><<<fin_grid, 256, 0, s>>>(a, rec);
+    launch_overlapped(accept::wide_range_kernel<accept::kMinMax, 4>, dim3(range_grid), 256, s, a, rec);
+    launch_overlapped(accept::wide_finalize_kernel<accept::kMinMax>, dim3(fin_grid), 256, s, a, rec);
     launch_wide_encode_for<accept::kMinMax>(p, a, rec, enc_grid, s);
   }
   g_launches.fetch_add(3, std::memory_order_relaxed);
@@ -183,8 +201,8 @@ accept_status launch_wide(const accept_params* p, const CodecArgs& a, uint8_t* r
 
 template <int K, int LAYOUT, int RANGE>
 void launch_strided_encode(int round, const CodecArgs& a, const accept::ChunkRecord* rec, dim3 grid, cudaStream_t s) {
-  if (round == accept::kNearest) accept::strided_encode_kernel<K, LAYOUT, RANGE, accept::kNearest><<<grid, 256, 0, s>>>(a, rec);
-  else accept::strided_encode_kernel<K, LAYOUT, RANGE, accept::kStochastic><<<grid, 256, 0, s>>>(a, rec);
+  if (round == accept::kNearest) launch_overlapped(accept::strided_encode_kernel<K, LAYOUT, RANGE, accept::kNearest>, dim3(grid), 256, s, a, rec);
+  else launch_overlapped(accept::strided_encode_kernel<K, LAYOUT, RANGE, accept::kStochastic>, dim3(grid), 256, s, a, rec);
 }
 
 template <int RANGE>
@@ -205,12 +223,12 @@ template <int RANGE>
 void launch_strided_decode_for(const accept_params* p, const CodecArgs& a, dim3 grid, cudaStream_t s) {
   const bool bp = p->layout == ACCEPT_LAYOUT_BITPLANE;
   switch (p->k) {
-    case 2: bp ? accept::strided_decode_kernel<2, accept::kBitplane, RANGE><<<grid, 256, 0, s>>>(a)
-               : accept::strided_decode_kernel<2, accept::kInterleaved, RANGE><<<grid, 256, 0, s>>>(a); break;
-    case 3: accept::strided_decode_kernel<3, accept::kBitplane, RANGE><<<grid, 256, 0, s>>>(a); break;
-    case 4: bp ? accept::strided_decode_kernel<4, accept::kBitplane, RANGE><<<grid, 256, 0, s>>>(a)
-               : accept::strided_decode_kernel<4, accept::kInterleaved, RANGE><<<grid, 256, 0, s>>>(a); break;
-    default: accept::strided_decode_kernel<8, accept::kInterleaved, RANGE><<<grid, 256, 0, s>>>(a); break;
+    case 2: bp ? launch_overlapped(accept::strided_decode_kernel<2, accept::kBitplane, RANGE>, dim3(grid), 256, s, a)
+               : launch_overlapped(accept::strided_decode_kernel<2, accept::kInterleaved, RANGE>, dim3(grid), 256, s, a); break;
+    case 3: launch_overlapped(accept::strided_decode_kernel<3, accept::kBitplane, RANGE>, dim3(grid), 256, s, a); break;
+    case 4: bp ? launch_overlapped(accept::strided_decode_kernel<4, accept::kBitplane, RANGE>, dim3(grid), 256, s, a)
+               : launch_overlapped(accept::strided_decode_kernel<4, accept::kInterleaved, RANGE>, dim3(grid), 256, s, a); break;
+    default: launch_overlapped(accept::strided_decode_kernel<8, accept::kInterleaved, RANGE>, dim3(grid), 256, s, a); break;
   }
 }
 
@@ -227,12 +245,12 @@ accept_status launch_strided(const accept_params* p, const CodecArgs& a, uint8_t
   const unsigned range_grid = (unsigned)((n_oct + 4 * 256 - 1) / (4 * 256));
   const unsigned fin_grid = (unsigned)((a.n_chunks + 255) / 256);
   if (p->range == ACCEPT_RANGE_ABSMAX) {
-    accept::wide_range_kernel<accept::kAbsMax, 4><<<range_grid, 256, 0, s>>>(a, rec);
-    accept::wide_finalize_kernel<accept::kAbsMax><<<fin_grid, 256, 0, s>>>(a, rec);
+    launch_overlapped(accept::wide_range_kernel<accept::kAbsMax, 4>, dim3(range_grid), 256, s, a, rec);
+    launch_overlapped(accept::wide_finalize_kernel<accept::kAbsMax>, dim3(fin_grid), 256, s, a, rec);
     launch_strided_encode_for<accept::kAbsMax>(p, a, rec, strided_grid(p), s);
   } else {
-    accept::wide_range_kernel<accept::kMinMax, 4><<<range_grid, 256, 0, s>>>(a, rec);
-    accept::wide_finalize_kernel<accept::kMinMax><<<fin_grid, 256, 0, s>>>(a, rec);
+    launch_overlapped(accept::wide_range_kernel<accept::kMinMax, 4>, dim3(range_grid), 256, s, a, rec);
+    launch_overlapped(accept::wide_finalize_kernel<accept::kMinMax>, dim3(fin_grid), 256, s, a, rec);
     launch_strided_encode_for<accept::kMinMax>(p, a, rec, strided_grid(p), s);
   }
   g_launches.fetch_add(3, std::memory_order_relaxed);
@@ -272,14 +290,14 @@ template <int K>
 void launch_mbq_compress(const accept::MbqArgs& a, cudaStream_t s) {
   if (a.init) {
     for (int j = 0; j < K; ++j) {
-      accept::mbq_residue_sum_kernel<K><<<a.n_blocks, 256, 0, s>>>(a, j);
-      accept::mbq_residue_finalize_kernel<<<1, 256, 0, s>>>(a, j);
+      launch_overlapped(accept::mbq_residue_sum_kernel<K>, dim3(a.n_blocks), 256, s, a, j);
+      launch_overlapped(accept::mbq_residue_finalize_kernel, dim3(1), 256, s, a, j);
     }
-    accept::mbq_encode_kernel<K, true><<<a.n_blocks, 256, 0, s>>>(a);
+    launch_overlapped(accept::mbq_encode_kernel<K, true>, dim3(a.n_blocks), 256, s, a);
   } else {
-    accept::mbq_encode_kernel<K, false><<<a.n_blocks, 256, 0, s>>>(a);
+    launch_overlapped(accept::mbq_encode_kernel<K, false>, dim3(a.n_blocks), 256, s, a);
   }
-  accept::mbq_finalize_kernel<K><<<1, accept::kMbqFinalizeThreads, 0, s>>>(a);
+  launch_overlapped(accept::mbq_finalize_kernel<K>, dim3(1), accept::kMbqFinalizeThreads, s, a);
   g_launches.fetch_add(2 + (a.init ? 2 * K : 0), std::memory_order_relaxed);
 }
 
@@ -394,9 +412,9 @@ accept_status accept_compress(const accept_params* p, const float* d_x, void* d_
   a.fast_blocks = (uint32_t)fast_blocks;
   const uint64_t grid = fast_blocks + (a.n_chunks - a.n_fast_chunks);
   KernelFn fn = select_compress(p, fast ? g.rounds : 2, block <= 256);
-  fn<<<(unsigned)grid, block, 0, static_cast<cudaStream_t>(cuda_stream)>>>(a);
+  const cudaError_t err = launch_overlapped(fn, (unsigned)grid, block, static_cast<cudaStream_t>(cuda_stream), a);
   g_launches.fetch_add(1, std::memory_order_relaxed);
-  return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+  return err == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
 }
 
 accept_status accept_decompress(const accept_params* p, const void* d_stream, size_t stream_bytes, float* d_xhat,
@@ -418,9 +436,9 @@ accept_status accept_decompress(const accept_params* p, const void* d_stream, si
   KernelFn fn = select_decompress(p, aligned, rounds);
   const uint64_t per_block = aligned ? 2048ull * rounds : 256;  // elements per block
   const uint64_t grid = (p->n_elems + per_block - 1) / per_block;
-  fn<<<(unsigned)grid, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(a);
+  const cudaError_t err = launch_overlapped(fn, (unsigned)grid, 256, static_cast<cudaStream_t>(cuda_stream), a);
   g_launches.fetch_add(1, std::memory_order_relaxed);
-  return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+  return err == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
 }
 
 accept_status accept_compress_host(const accept_params* p, const float* h_x, void* h_stream, size_t stream_bytes,
@@ -546,9 +564,9 @@ accept_status accept_mbq_decompress(const accept_mbq_params* p, const void* d_st
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   const unsigned grid = (unsigned)((p->n_elems + 4095) / 4096);
   switch (p->k) {
-    case 2: accept::mbq_decode_kernel<2><<<grid, 256, 0, s>>>(a); break;
-    case 3: accept::mbq_decode_kernel<3><<<grid, 256, 0, s>>>(a); break;
-    default: accept::mbq_decode_kernel<4><<<grid, 256, 0, s>>>(a); break;
+    case 2: launch_overlapped(accept::mbq_decode_kernel<2>, dim3(grid), 256, s, a); break;
+    case 3: launch_overlapped(accept::mbq_decode_kernel<3>, dim3(grid), 256, s, a); break;
+    default: launch_overlapped(accept::mbq_decode_kernel<4>, dim3(grid), 256, s, a); break;
   }
   g_launches.fetch_add(1, std::memory_order_relaxed);
   return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;

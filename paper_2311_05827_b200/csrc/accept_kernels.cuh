@@ -42,6 +42,15 @@ __device__ __forceinline__ uint32_t header_word(const CodecArgs& a, int i) {
   }
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may be
+// scheduled while the kernel before it in the stream is still draining.  Every kernel here waits
+// for that predecessor (and the visibility of its writes) before it touches memory, and lets its
+// own successor be scheduled right away: what overlaps is launch latency and the tail of the grid.
+__device__ __forceinline__ void grid_dependency_handshake() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 constexpr int kFastBlock = 128;     // threads per block when a chunk needs at most 128 threads (finer tail than 256: measured)
 constexpr int kGenericBlock = 256;  // threads per block of the any-shape path
 
@@ -165,6 +174,7 @@ template <int K, int LAYOUT, int RANGE, int ROUND, int R, int BLOCK_MAX>
 __global__ void __launch_bounds__(BLOCK_MAX, BLOCK_MAX == 256 ? (R <= 2 ? 6 : 4) : 1) compress_kernel(const CodecArgs a) {
   __shared__ float s_hi[32], s_lo[32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  grid_dependency_handshake();
 
   if (blockIdx.x == 0 && tid < 8) {
     // stream header and the pad between the side words and the payload
@@ -349,6 +359,7 @@ __device__ __forceinline__ void decode_tile(const CodecArgs& a, const RawOctet (
 template <int K, int LAYOUT, int RANGE, int R>
 __global__ void __launch_bounds__(256, R <= 2 ? 8 : 6) decompress_kernel(const CodecArgs a) {
   const int tid = threadIdx.x, lane = tid & 31;
+  grid_dependency_handshake();
   if (blockIdx.x == 0 && tid < 8) {
     // the rounding mode (bits 8..15 of word 6) does not change how a stream is read
     const uint32_t mask = (tid == 6) ? 0xFFFF00FFu : 0xFFFFFFFFu;
@@ -366,6 +377,7 @@ __global__ void __launch_bounds__(256, R <= 2 ? 8 : 6) decompress_kernel(const C
 // Scalar any-alignment decoder for output pointers that are not 32-byte aligned.
 template <int K, int LAYOUT, int RANGE>
 __global__ void __launch_bounds__(256) decompress_unaligned_kernel(const CodecArgs a) {
+  grid_dependency_handshake();
   const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= a.n) return;
   uint32_t u = 0;

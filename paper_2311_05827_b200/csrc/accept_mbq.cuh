@@ -164,6 +164,7 @@ __device__ __forceinline__ double warp_sum(double v) {
 // Residue method, step j: per-block sum of |r_j| (r_0 = x) with the coefficients found so far.
 template <int K>
 __global__ void __launch_bounds__(256) mbq_residue_sum_kernel(const MbqArgs a, int j) {
+  grid_dependency_handshake();
   __shared__ double s_part[8];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   float alpha[K];
@@ -198,6 +199,7 @@ __global__ void __launch_bounds__(256) mbq_residue_sum_kernel(const MbqArgs a, i
 
 // Residue method, step j: alpha_j = mean |r_j| (block partials added in index order).
 __global__ void __launch_bounds__(256) mbq_residue_finalize_kernel(const MbqArgs a, int j) {
+  grid_dependency_handshake();
   __shared__ double s_part[256];
   const int tid = threadIdx.x;
   double s = 0.0;
@@ -214,6 +216,7 @@ __global__ void __launch_bounds__(256) mbq_residue_finalize_kernel(const MbqArgs
 // Assign the signs, write the planes, gather the per-block sums.
 template <int K, bool INIT>
 __global__ void __launch_bounds__(256) mbq_encode_kernel(const MbqArgs a) {
+  grid_dependency_handshake();
   __shared__ MbqTable<K> s_table;
   __shared__ float s_level[16];
   __shared__ double s_dbl[8][K + 1];
@@ -348,6 +351,7 @@ __global__ void __launch_bounds__(256) mbq_encode_kernel(const MbqArgs a) {
 // words and alpha_next.  One block.
 template <int K>
 __global__ void __launch_bounds__(kMbqFinalizeThreads) mbq_finalize_kernel(const MbqArgs a) {
+  grid_dependency_handshake();
   __shared__ double s_dbl[kMbqFinalizeThreads / 32][K + 1];
   __shared__ unsigned long long s_int[kMbqFinalizeThreads / 32][10];
   const int tid = threadIdx.x;
@@ -452,6 +456,7 @@ __global__ void __launch_bounds__(kMbqFinalizeThreads) mbq_finalize_kernel(const
 // Receiver: planes -> codes -> level(c) - m_q.
 template <int K>
 __global__ void __launch_bounds__(256, 8) mbq_decode_kernel(const MbqArgs a) {
+  grid_dependency_handshake();
   __shared__ float s_value[1 << K];
   const int tid = threadIdx.x, lane = tid & 31;
   if (blockIdx.x == 0 && tid < 8 && a.header[tid] != mbq_header_word(a, tid)) atomicOr(a.status, kDevBadHeader);

@@ -33,6 +33,7 @@ constexpr int kStridedOctetsPerBlock = 64;
 
 template <int K, int LAYOUT, int RANGE, int ROUND>
 __global__ void __launch_bounds__(256, 4) strided_encode_kernel(const CodecArgs a, const ChunkRecord* rec) {
+  grid_dependency_handshake();
   const int tid = threadIdx.x, lane = tid & 31, sub = tid & 3;
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid < 8) {
     a.header[tid] = header_word(a, tid);
@@ -125,6 +126,7 @@ __global__ void __launch_bounds__(256, 4) strided_encode_kernel(const CodecArgs 
 
 template <int K, int LAYOUT, int RANGE>
 __global__ void __launch_bounds__(256) strided_decode_kernel(const CodecArgs a) {
+  grid_dependency_handshake();
   const int tid = threadIdx.x, lane = tid & 31, sub = tid & 3;
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid < 8) {
     const uint32_t mask = (tid == 6) ? 0xFFFF00FFu : 0xFFFFFFFFu;

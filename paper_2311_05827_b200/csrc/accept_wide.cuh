@@ -58,6 +58,7 @@ __device__ __forceinline__ uint64_t chunk_of(const CodecArgs& a, uint64_t e) {
 // octet merges on its own.
 template <int RANGE, int R>
 __global__ void __launch_bounds__(256) wide_range_kernel(const CodecArgs a, ChunkRecord* rec) {
+  grid_dependency_handshake();
   __shared__ float s_hi[8], s_lo[8];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint64_t n_oct = (a.n + 7) / 8;
@@ -117,6 +118,7 @@ __global__ void __launch_bounds__(256) wide_range_kernel(const CodecArgs a, Chun
 // stream) and the encoder's constants (written over the record: a = 1 if the chunk is non-finite).
 template <int RANGE>
 __global__ void __launch_bounds__(256) wide_finalize_kernel(const CodecArgs a, ChunkRecord* rec) {
+  grid_dependency_handshake();
   const uint64_t m = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (m >= a.n_chunks) return;
   float hi, lo = 0.0f;
@@ -144,6 +146,7 @@ __global__ void __launch_bounds__(256) wide_finalize_kernel(const CodecArgs a, C
 // Pass 3: quantize + pack with the constants of each octet's chunk.
 template <int K, int LAYOUT, int RANGE, int ROUND, int R>
 __global__ void __launch_bounds__(256, 5) wide_encode_kernel(const CodecArgs a, const ChunkRecord* rec) {
+  grid_dependency_handshake();
   const int tid = threadIdx.x, lane = tid & 31;
   if (blockIdx.x == 0 && tid < 8) {
     a.header[tid] = header_word(a, tid);
