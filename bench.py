@@ -289,6 +289,30 @@ def time_oracle(x_host, chunk, mode, seed, budget_s=10.0, max_reps=50):
     return tc / reps, td / reps, reps
 
 
+def time_oracle_all_cores(x_host, chunk, mode, seed, reps=3):
+    """The same oracle over disjoint chunk ranges, one thread per host core (ctypes calls drop the GIL):
+    (seconds per round trip, threads).  Each slice becomes a stream of its own; counters continue across slices."""
+    import oracle
+    from concurrent.futures import ThreadPoolExecutor
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    n_chunks = -(-x_host.size // chunk)
+    per = -(-n_chunks // cores) * chunk
+    slices = [(lo, min(lo + per, x_host.size)) for lo in range(0, x_host.size, per)]
+
+    def one(bounds):
+        lo, hi = bounds
+        stream, _ = oracle.compress(x_host[lo:hi], chunk, mode.k, mode.range, mode.round, mode.layout, seed, lo)
+        oracle.decompress(stream, hi - lo)
+
+    with ThreadPoolExecutor(max_workers=len(slices)) as pool:
+        list(pool.map(one, slices))          # untimed: loads the library, touches the pages
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            list(pool.map(one, slices))
+        dt = (time.perf_counter() - t0) / reps
+    return dt, len(slices)
+
+
 def max_over_ranks(values, dist, device):
     """Element-wise maximum of per-rank timings (the slowest rank defines the job's time)."""
     import torch
@@ -392,6 +416,10 @@ def run_gpu(args):
                                "sample": "whole %s tensor (%d elements), %d round trips; compress %.3f s, decompress %.3f s each"
                                          % (args.workload, n, reps, tc, td),
                                "host_cores_available": os.cpu_count()}
+        t_all, threads = time_oracle_all_cores(x_host, spec.chunk, mode, spec.seed)
+        out["cpu_baseline"]["all_cores"] = {"value": 4 * n / t_all / 1e9, "unit": UNIT, "cores": threads,
+                                            "sample": "the same tensor split into %d contiguous chunk ranges, one thread each, "
+                                                      "3 round trips" % threads}
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
