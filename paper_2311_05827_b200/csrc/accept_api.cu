@@ -155,14 +155,23 @@ KernelFn select_decompress(const accept_params* p, bool aligned, int rounds) {
 
 // ---- wide chunks: ranges, constants, encode ------------------------------------------------------
 
+// Octets per thread of the encode pass: the stochastic quantizer is instruction bound and amortises its
+// per-thread generator set-up over four octets; the nearest one is memory bound and keeps two.
+constexpr int kWideOctetsNearest = 2, kWideOctetsStochastic = 4;
+
 template <int K, int LAYOUT, int RANGE>
-void launch_wide_encode(int round, const CodecArgs& a, const accept::ChunkRecord* rec, unsigned grid, cudaStream_t s) {
-  if (round == accept::kNearest) launch_overlapped(accept::wide_encode_kernel<K, LAYOUT, RANGE, accept::kNearest, 2>, dim3(grid), 256, s, a, rec);
-  else launch_overlapped(accept::wide_encode_kernel<K, LAYOUT, RANGE, accept::kStochastic, 2>, dim3(grid), 256, s, a, rec);
+void launch_wide_encode(int round, const CodecArgs& a, const accept::ChunkRecord* rec, uint64_t n_oct_stored, cudaStream_t s) {
+  if (round == accept::kNearest) {
+    const unsigned grid = (unsigned)((n_oct_stored + kWideOctetsNearest * 256 - 1) / (kWideOctetsNearest * 256));
+    launch_overlapped(accept::wide_encode_kernel<K, LAYOUT, RANGE, accept::kNearest, kWideOctetsNearest>, dim3(grid), 256, s, a, rec);
+  } else {
+    const unsigned grid = (unsigned)((n_oct_stored + kWideOctetsStochastic * 256 - 1) / (kWideOctetsStochastic * 256));
+    launch_overlapped(accept::wide_encode_kernel<K, LAYOUT, RANGE, accept::kStochastic, kWideOctetsStochastic>, dim3(grid), 256, s, a, rec);
+  }
 }
 
 template <int RANGE>
-void launch_wide_encode_for(const accept_params* p, const CodecArgs& a, const accept::ChunkRecord* rec, unsigned grid,
+void launch_wide_encode_for(const accept_params* p, const CodecArgs& a, const accept::ChunkRecord* rec, uint64_t grid,
                             cudaStream_t s) {
   const bool bp = p->layout == ACCEPT_LAYOUT_BITPLANE;
   switch (p->k) {
@@ -183,7 +192,7 @@ accept_status launch_wide(const accept_params* p, const CodecArgs& a, uint8_t* r
   const uint64_t n_oct = (p->n_elems + 7) / 8;
   const unsigned range_grid = (unsigned)((n_oct + 4 * 256 - 1) / (4 * 256));
   const unsigned fin_grid = (unsigned)((a.n_chunks + 255) / 256);
-  const unsigned enc_grid = (unsigned)((((p->n_elems + 31) / 32) * 4 + 2 * 256 - 1) / (2 * 256));
+  const uint64_t enc_grid = ((p->n_elems + 31) / 32) * 4;  // octets the encode pass stores
   if (p->range == ACCEPT_RANGE_ABSMAX) {
     launch_overlapped(accept::wide_range_kernel<accept::kAbsMax, 4>, dim3(range_grid), 256, s, a, rec);
     launch_overlapped(accept::wide_finalize_kernel<accept::kAbsMax>, dim3(fin_grid), 256, s, a, rec);

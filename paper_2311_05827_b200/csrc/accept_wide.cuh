@@ -143,9 +143,21 @@ __global__ void __launch_bounds__(256) wide_finalize_kernel(const CodecArgs a, C
   rec[m].base = sc.base;
 }
 
-// Pass 3: quantize + pack with the constants of each octet's chunk.
+// Pass 3: quantize + pack with the constants of each octet's chunk.  A tile that lies inside the
+// tensor and inside one chunk (all but the tiles on a chunk boundary and the last one) reads its
+// record once and skips the per-octet guards.
+__device__ __forceinline__ Scale scale_from_record(const ChunkRecord* rec) {
+  const uint4 raw = __ldg(reinterpret_cast<const uint4*>(rec));
+  Scale sc;
+  sc.s = 0.0f; sc.o = 0.0f;
+  sc.inv = __uint_as_float(raw.z);
+  sc.base = __uint_as_float(raw.w);
+  sc.nonfinite = raw.x != 0u;
+  return sc;
+}
+
 template <int K, int LAYOUT, int RANGE, int ROUND, int R>
-__global__ void __launch_bounds__(256, 5) wide_encode_kernel(const CodecArgs a, const ChunkRecord* rec) {
+__global__ void __launch_bounds__(256, R <= 2 ? 5 : 4) wide_encode_kernel(const CodecArgs a, const ChunkRecord* rec) {
   grid_dependency_handshake();
   const int tid = threadIdx.x, lane = tid & 31;
   if (blockIdx.x == 0 && tid < 8) {
@@ -153,7 +165,34 @@ __global__ void __launch_bounds__(256, 5) wide_encode_kernel(const CodecArgs a, 
     if ((a.n_chunks & 1) && tid < 2) reinterpret_cast<uint32_t*>(a.meta + a.n_chunks)[tid] = 0u;
   }
   const uint64_t n_oct_stored = ((a.n + 31) / 32) * 4;  // whole pack groups are stored
-  const uint64_t oct0 = (uint64_t)blockIdx.x * (R * 256) + tid;
+  const uint64_t tile_oct = (uint64_t)blockIdx.x * (R * 256);
+  const uint64_t oct0 = tile_oct + tid;
+  const Rng rng{(uint32_t)a.seed, (uint32_t)(a.seed >> 32)};
+  RngThread rt;
+  if (ROUND == kStochastic) rt.init(rng, a.rng_offset + oct0 * 8, 8u * (R - 1) * 256u + 8u);
+
+  const uint64_t tile_first = tile_oct * 8, tile_last = tile_first + (uint64_t)R * 256 * 8 - 1;
+  const uint64_t tile_chunk = chunk_of(a, tile_first);
+  if (tile_last < a.n && chunk_of(a, tile_last) == tile_chunk) {
+    float v[R][8];
+#pragma unroll
+    for (int r = 0; r < R; ++r) ld_octet(a.x + (oct0 + r * 256) * 8, v[r]);
+    const Scale sc = scale_from_record(rec + tile_chunk);
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const uint64_t oct = oct0 + r * 256;
+      if (sc.nonfinite) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[r][i] = 0.0f;
+      }
+      uint32_t xlo, xhi;
+      quantize_octet<K, RANGE, ROUND>(v[r], sc, rng, rt, 8u * r * 256u, xlo, xhi);
+      if (LAYOUT == kInterleaved) store_interleaved<K>(a.payload, oct, xlo, xhi);
+      else store_bitplane<K>(a.payload, oct >> 2, xlo, xhi, lane);
+    }
+    return;
+  }
+
   float v[R][8];
 #pragma unroll
   for (int r = 0; r < R; ++r) {
@@ -165,21 +204,13 @@ __global__ void __launch_bounds__(256, 5) wide_encode_kernel(const CodecArgs a, 
       for (int e = 0; e < 8; ++e) v[r][e] = 0.0f;
     }
   }
-  const Rng rng{(uint32_t)a.seed, (uint32_t)(a.seed >> 32)};
-  RngThread rt;
-  if (ROUND == kStochastic) rt.init(rng, a.rng_offset + oct0 * 8, 8u * (R - 1) * 256u + 8u);
 #pragma unroll
   for (int r = 0; r < R; ++r) {
     const uint64_t oct = oct0 + r * 256, e = oct * 8;
     const bool stored = oct < n_oct_stored;
     uint32_t xlo = 0, xhi = 0;
     if (e < a.n) {
-      const uint4 raw = __ldg(reinterpret_cast<const uint4*>(rec + chunk_of(a, e)));
-      Scale sc;
-      sc.s = 0.0f; sc.o = 0.0f;
-      sc.inv = __uint_as_float(raw.z);
-      sc.base = __uint_as_float(raw.w);
-      sc.nonfinite = raw.x != 0u;
+      const Scale sc = scale_from_record(rec + chunk_of(a, e));
       if (sc.nonfinite) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) v[r][i] = 0.0f;
