@@ -74,6 +74,7 @@ typedef enum {
 /* Bits of the device status word (word 0 of the workspace); sticky until the caller clears it. */
 #define ACCEPT_DEV_NONFINITE 1u   /* some chunk held NaN/Inf (or an overflowing MINMAX range) */
 #define ACCEPT_DEV_BAD_HEADER 2u  /* accept_decompress: stream header differs from the parameters */
+#define ACCEPT_DEV_COPY_TIMEOUT 4u /* an asynchronous copy inside a kernel did not complete within a second; output invalid */
 
 typedef enum { ACCEPT_RANGE_ABSMAX = 0, ACCEPT_RANGE_MINMAX = 1 } accept_range;
 typedef enum { ACCEPT_ROUND_NEAREST = 0, ACCEPT_ROUND_STOCHASTIC = 1 } accept_round;

@@ -19,7 +19,7 @@ LAYOUT_INTERLEAVED, LAYOUT_BITPLANE = 0, 1
 HEADER_BYTES = 32
 
 OK = 0
-DEV_NONFINITE, DEV_BAD_HEADER = 1, 2
+DEV_NONFINITE, DEV_BAD_HEADER, DEV_COPY_TIMEOUT = 1, 2, 4
 
 STATUS_NAMES = {
     0: "ACCEPT_OK", 1: "ACCEPT_ERR_NULL", 2: "ACCEPT_ERR_BAD_K", 3: "ACCEPT_ERR_BAD_CHUNK",

@@ -70,11 +70,12 @@ CodecArgs make_args(const accept_params* p, void* d_stream, void* d_ws) {
 // Launch with programmatic stream serialization: every kernel of this library starts with
 // grid_dependency_handshake(), so it may be scheduled while its predecessor in the stream drains.
 template <typename... Params, typename... Args>
-cudaError_t launch_overlapped(void (*fn)(Params...), dim3 grid, unsigned block, cudaStream_t s, Args&&... args) {
+cudaError_t launch_overlapped_shared(void (*fn)(Params...), dim3 grid, unsigned block, size_t shared_bytes, cudaStream_t s,
+                                     Args&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = dim3(block, 1, 1);
-  cfg.dynamicSmemBytes = 0;
+  cfg.dynamicSmemBytes = shared_bytes;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -82,6 +83,11 @@ cudaError_t launch_overlapped(void (*fn)(Params...), dim3 grid, unsigned block, 
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, fn, std::forward<Args>(args)...);
+}
+
+template <typename... Params, typename... Args>
+cudaError_t launch_overlapped(void (*fn)(Params...), dim3 grid, unsigned block, cudaStream_t s, Args&&... args) {
+  return launch_overlapped_shared(fn, grid, block, 0, s, std::forward<Args>(args)...);
 }
 
 // ---- kernel tables -------------------------------------------------------------------------
@@ -208,10 +214,28 @@ accept_status launch_wide(const accept_params* p, const CodecArgs& a, uint8_t* r
 
 // ---- pack groups along the batch dimension ---------------------------------------------------------
 
+// The encoder is persistent: at most three blocks (64 KB of staged tile each) per SM of a B200.
+constexpr unsigned kStridedEncodeBlocks = 3 * 148;
+
 template <int K, int LAYOUT, int RANGE>
-void launch_strided_encode(int round, const CodecArgs& a, const accept::ChunkRecord* rec, dim3 grid, cudaStream_t s) {
-  if (round == accept::kNearest) launch_overlapped(accept::strided_encode_kernel<K, LAYOUT, RANGE, accept::kNearest>, dim3(grid), 256, s, a, rec);
-  else launch_overlapped(accept::strided_encode_kernel<K, LAYOUT, RANGE, accept::kStochastic>, dim3(grid), 256, s, a, rec);
+void launch_strided_encode(int round, const CodecArgs& a, const accept::ChunkRecord* rec, dim3 tiles, cudaStream_t s) {
+  if (round != accept::kNearest) {  // instruction bound: one tile per block, rows in registers
+    launch_overlapped(accept::strided_encode_direct_kernel<K, LAYOUT, RANGE, accept::kStochastic>, tiles, 256, s, a, rec);
+    return;
+  }
+  // memory bound: persistent blocks with a staged tile, which needs more dynamic shared memory than a
+  // kernel gets without opting in (the attribute is per device: set every time)
+  auto fn = accept::strided_encode_kernel<K, LAYOUT, RANGE, accept::kNearest>;
+  if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, accept::kStridedSmemBytes) != cudaSuccess) return;
+  const uint64_t n_tiles = (uint64_t)tiles.x * tiles.y;
+  const unsigned grid = (unsigned)(n_tiles < kStridedEncodeBlocks ? n_tiles : kStridedEncodeBlocks);
+  accept::StridedTiling t;
+  t.tiles_x = tiles.x;
+  t.tiles_y = tiles.y;
+  t.n_rows = (uint32_t)(a.n / a.group_stride);
+  t.step_x = grid % tiles.x;
+  t.step_y = grid / tiles.x;
+  launch_overlapped_shared(fn, dim3(grid), 256, accept::kStridedSmemBytes, s, a, rec, t);
 }
 
 template <int RANGE>

@@ -14,7 +14,7 @@ constexpr int kAbsMax = 0, kMinMax = 1;
 constexpr int kNearest = 0, kStochastic = 1;
 constexpr int kInterleaved = 0, kBitplane = 1;
 
-constexpr uint32_t kDevNonFinite = 1u, kDevBadHeader = 2u;
+constexpr uint32_t kDevNonFinite = 1u, kDevBadHeader = 2u, kDevCopyTimeout = 4u;
 
 // 1.5 * 2^23: adding it to |t| < 2^22 rounds t to an integer (ties to even, the fp32 adder's
 // rounding) and leaves that integer in the low mantissa bits.

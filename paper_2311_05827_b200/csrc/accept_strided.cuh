@@ -31,8 +31,264 @@ __device__ __forceinline__ void transpose4x4(uint32_t a0, uint32_t a1, uint32_t 
 // quad byte transpose.  Block = 64 feature octets x 4 row blocks.
 constexpr int kStridedOctetsPerBlock = 64;
 
+// The encoder is persistent: a block walks over tiles of 32 rows x 2 KB and stages them in shared
+// memory with asynchronous bulk copies (one per row, issued by the lanes of warp 0, completion counted
+// in bytes on an mbarrier), so that the bytes in flight per SM are set by shared memory (three resident
+// blocks x 64 KB), not by registers, and the next tile streams in while this one is coded.
+// A tile is two stages: rows 4h..4h+3 of every block of eight rows form stage h.  Once every thread has
+// moved its rows of a stage to registers, the same stage of the next tile is requested.
+// The rows of a block of eight are 2 KB apart; each block of eight rows starts 32 bytes further than a
+// multiple of 16 KB, which spreads the four lanes of a quad over different banks.
+constexpr int kStridedRowBytes = kStridedOctetsPerBlock * 32;
+constexpr int kStridedRowBlockPitch = 8 * kStridedRowBytes + 32;
+constexpr int kStridedTileBytes = 4 * kStridedRowBlockPitch;
+constexpr int kStridedSmemBytes = kStridedTileBytes + 16;  // + two mbarriers
+
+__device__ __forceinline__ uint32_t smem_address(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbarrier_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbarrier_expect_bytes(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_copy_to_shared(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// Waits for the phase of the given parity; gives up after about a second.
+__device__ __forceinline__ bool mbarrier_wait(uint32_t bar, uint32_t parity) {
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
+    if ((it & 63u) == 63u) {
+      unsigned long long now;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > 1000000000ull) return false;
+    }
+  }
+}
+
+// Transposes a thread's 8 rows x 8 features of codes and stores the words of its eight features.
+template <int K, int LAYOUT>
+__device__ __forceinline__ void strided_store_tile(const CodecArgs& a, const uint32_t (&xlo)[8], const uint32_t (&xhi)[8],
+                                                   uint64_t word0, bool active, int sub, int lane) {
+  // rows x features -> features x rows
+  uint32_t ylo[8], yhi[8];  // per feature: codes of rows 0..3 / 4..7 of this block of eight rows
+  {
+    uint32_t o[4];
+    transpose4x4(xlo[0], xlo[1], xlo[2], xlo[3], o);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) ylo[e] = o[e];
+    transpose4x4(xlo[4], xlo[5], xlo[6], xlo[7], o);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) yhi[e] = o[e];
+    transpose4x4(xhi[0], xhi[1], xhi[2], xhi[3], o);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) ylo[4 + e] = o[e];
+    transpose4x4(xhi[4], xhi[5], xhi[6], xhi[7], o);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) yhi[4 + e] = o[e];
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    uint32_t* group_words = a.payload + word0 + (uint64_t)e * K;
+    if (LAYOUT == kBitplane) {
+      // byte j = digit j of my eight rows; after the quad transpose lane q holds digit q of all 32 rows
+      const uint32_t w = quad_transpose(planes_nibbles(merge_nibbles(ylo[e], yhi[e])), lane);
+      if (active && sub < K) group_words[sub] = w;
+    } else if (K == 8) {
+      if (active) reinterpret_cast<uint2*>(group_words)[sub] = make_uint2(ylo[e], yhi[e]);
+    } else if (K == 4) {
+      const uint32_t zlo = ylo[e] | (ylo[e] >> 4), zhi = yhi[e] | (yhi[e] >> 4);
+      if (active) group_words[sub] = __byte_perm(zlo, zhi, 0x6420);
+    } else {  // K == 2: sixteen bits per eight rows
+      uint32_t zlo = ylo[e] | (ylo[e] >> 6), zhi = yhi[e] | (yhi[e] >> 6);
+      zlo |= zlo >> 12;
+      zhi |= zhi >> 12;
+      if (active) reinterpret_cast<uint16_t*>(group_words)[sub] = (uint16_t)__byte_perm(zlo, zhi, 0x0040);
+    }
+  }
+}
+
+// How the persistent encoder walks the tensor: tiles_x x tiles_y tiles, taken in row-major order with a
+// stride of one grid; the stride is given split into whole tile rows and a remainder so that a block
+// advances its tile coordinates with an add and a compare.
+struct StridedTiling {
+  uint32_t tiles_x, tiles_y;
+  uint32_t n_rows;           // batch rows of the tensor
+  uint32_t step_x, step_y;   // gridDim.x = step_y * tiles_x + step_x
+};
+
+// Warp 0 requests stage `half` of tile (bx, g): lane = row of the tile, rows with ((row / 4) & 1) == half.
+__device__ __forceinline__ void strided_request_stage(const CodecArgs& a, const StridedTiling& t, uint32_t bx, uint32_t g,
+                                                      int half, int lane, uint32_t tile0, uint32_t bar) {
+  const uint32_t F = a.group_stride;
+  const uint32_t fo0 = bx * kStridedOctetsPerBlock;
+  const uint32_t row_bytes = min((uint32_t)kStridedOctetsPerBlock, F / 8 - fo0) * 32;
+  const uint32_t rows_left = t.n_rows - g * 32;
+  const uint32_t valid = (rows_left >= 32 ? 0xFFFFFFFFu : ((1u << rows_left) - 1u)) & (half ? 0xF0F0F0F0u : 0x0F0F0F0Fu);
+  if (lane == 0) mbarrier_expect_bytes(bar, __popc(valid) * row_bytes);
+  __syncwarp();
+  if ((valid >> lane) & 1u) {
+    const float* src = a.x + (uint64_t)(g * 32 + lane) * F + (uint64_t)fo0 * 8;
+    const uint32_t dst = tile0 + (lane >> 3) * kStridedRowBlockPitch + (lane & 7) * kStridedRowBytes;
+    bulk_copy_to_shared(dst, src, row_bytes, bar);
+  }
+}
+
+// The encoder's constants of the four rows a thread codes in stage `half` of tile (bx, g): inv (sign
+// bit = chunk is non-finite) and, for MINMAX, base.  Rows outside the tensor get in = false.
+template <int RANGE>
+struct StridedRowConstants {
+  float inv[4], base[4];
+  bool in[4];
+  __device__ __forceinline__ void fetch(const CodecArgs& a, const ChunkRecord* rec, const StridedTiling& t, uint32_t bx,
+                                        uint32_t g, int half, int tid) {
+    const uint32_t F = a.group_stride;
+    const uint32_t fo = bx * kStridedOctetsPerBlock + (tid >> 2);
+    const bool active = fo < F / 8;
+    const uint32_t row0 = g * 32 + (tid & 3) * 8 + half * 4;
+    uint64_t i0 = (uint64_t)row0 * F + (uint64_t)fo * 8;
+#pragma unroll
+    for (int r = 0; r < 4; ++r, i0 += F) {
+      in[r] = active && row0 + r < t.n_rows;
+      inv[r] = 0.0f;
+      base[r] = 0.0f;
+      if (in[r]) {
+        const ChunkRecord* c = rec + chunk_of(a, i0);
+        if (RANGE == kAbsMax) {
+          inv[r] = __ldg(&c->inv);
+        } else {
+          const float2 ib = __ldg(reinterpret_cast<const float2*>(&c->inv));
+          inv[r] = ib.x;
+          base[r] = ib.y;
+        }
+      }
+    }
+  }
+};
+
 template <int K, int LAYOUT, int RANGE, int ROUND>
-__global__ void __launch_bounds__(256, 4) strided_encode_kernel(const CodecArgs a, const ChunkRecord* rec) {
+__global__ void __launch_bounds__(256, 3) strided_encode_kernel(const CodecArgs a, const ChunkRecord* rec,
+                                                                const StridedTiling t) {
+  extern __shared__ __align__(128) uint8_t s_tile[];
+  grid_dependency_handshake();
+  const int tid = threadIdx.x, lane = tid & 31, sub = tid & 3;
+  if (blockIdx.x == 0 && tid < 8) {
+    a.header[tid] = header_word(a, tid);
+    if ((a.n_chunks & 1) && tid < 2) reinterpret_cast<uint32_t*>(a.meta + a.n_chunks)[tid] = 0u;
+  }
+  const uint32_t F = a.group_stride;
+  const Rng rng{(uint32_t)a.seed, (uint32_t)(a.seed >> 32)};
+
+  const uint32_t tile0 = smem_address(s_tile);
+  const uint32_t bar[2] = {smem_address(s_tile + kStridedTileBytes), smem_address(s_tile + kStridedTileBytes) + 8u};
+  if (tid == 0) {
+    mbarrier_init(bar[0], 1);
+    mbarrier_init(bar[1], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  uint32_t bx = blockIdx.x % t.tiles_x, g = blockIdx.x / t.tiles_x;  // this block's tile; g >= tiles_y: none left
+  bool pending[2] = {false, false};  // a request of the stage's current phase is in flight
+  uint32_t parity[2] = {0u, 0u};     // parity of the stage's current phase
+  if (g < t.tiles_y) {
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      if (tid < 32) strided_request_stage(a, t, bx, g, half, lane, tile0, bar[half]);
+      pending[half] = true;
+    }
+  }
+  bool failed = false;
+  StridedRowConstants<RANGE> cur, nxt;  // constants are fetched one stage ahead of their use
+  if (g < t.tiles_y) cur.fetch(a, rec, t, bx, g, 0, tid);
+  while (g < t.tiles_y) {
+    uint32_t next_bx = bx + t.step_x, next_g = g + t.step_y;
+    if (next_bx >= t.tiles_x) { next_bx -= t.tiles_x; ++next_g; }
+    const bool has_next = next_g < t.tiles_y;
+    const uint32_t fo = bx * kStridedOctetsPerBlock + (tid >> 2);  // feature octet of this thread
+    const bool active = fo < F / 8;                                // inactive lanes still shuffle
+    const uint64_t word0 = ((uint64_t)g * F + (uint64_t)fo * 8) * K;  // first word of feature 8*fo of this batch group
+
+    uint32_t xlo[8], xhi[8];  // per row: codes of features 0..3 / 4..7
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      float v[4][8];
+      const bool ok = !failed && mbarrier_wait(bar[half], parity[half]);
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const float4* src = reinterpret_cast<const float4*>(s_tile + sub * kStridedRowBlockPitch +
+                                                            (half * 4 + r) * kStridedRowBytes + (tid >> 2) * 32);
+        float4 p0 = make_float4(0.f, 0.f, 0.f, 0.f), p1 = p0;
+        if (cur.in[r] && ok) { p0 = src[0]; p1 = src[1]; }
+        v[r][0] = p0.x; v[r][1] = p0.y; v[r][2] = p0.z; v[r][3] = p0.w;
+        v[r][4] = p1.x; v[r][5] = p1.y; v[r][6] = p1.z; v[r][7] = p1.w;
+      }
+      // every thread holds its rows of this stage, or some thread gave up (the verdict is the block's)
+      if (!failed) {
+        if (__syncthreads_and(ok)) {
+          pending[half] = false;
+          parity[half] ^= 1u;
+          if (has_next) {
+            if (tid < 32) strided_request_stage(a, t, next_bx, next_g, half, lane, tile0, bar[half]);
+            pending[half] = true;
+          }
+        } else {
+          failed = true;
+        }
+      }
+      if (half == 0) nxt.fetch(a, rec, t, bx, g, 1, tid);
+      else if (has_next) nxt.fetch(a, rec, t, next_bx, next_g, 0, tid);
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int rr = half * 4 + r;
+        xlo[rr] = 0; xhi[rr] = 0;
+        if (cur.in[r] && !failed) {
+          const uint64_t i0 = (uint64_t)(g * 32 + sub * 8 + rr) * F + (uint64_t)fo * 8;
+          Scale sc;
+          sc.s = 0.0f; sc.o = 0.0f;
+          sc.inv = fabsf(cur.inv[r]);
+          sc.base = cur.base[r];
+          sc.nonfinite = (__float_as_uint(cur.inv[r]) >> 31) != 0u;
+          if (sc.nonfinite) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[r][e] = 0.0f;
+          }
+          RngThread rt;
+          if (ROUND == kStochastic) rt.init(rng, a.rng_offset + i0, 8u);
+          quantize_octet<K, RANGE, ROUND>(v[r], sc, rng, rt, 0u, xlo[rr], xhi[rr]);
+        }
+      }
+      cur = nxt;
+    }
+    if (failed) break;
+    strided_store_tile<K, LAYOUT>(a, xlo, xhi, word0, active, sub, lane);
+    bx = next_bx;
+    g = next_g;
+  }
+  if (failed) {
+    // a copy did not arrive: report it, give what is still in flight a bounded time to land, and leave
+    if (tid == 0) atomicOr(a.status, kDevCopyTimeout);
+#pragma unroll
+    for (int half = 0; half < 2; ++half)
+      if (pending[half]) mbarrier_wait(bar[half], parity[half]);
+  }
+}
+
+// The same encoder with its rows loaded straight into registers, one tile per block: under STOCHASTIC
+// rounding the kernel is bound by instruction issue, not by bytes in flight, and the 32 resident warps
+// this form allows (against 24 with a staged tile) are worth more than the staging.
+template <int K, int LAYOUT, int RANGE, int ROUND>
+__global__ void __launch_bounds__(256, 4) strided_encode_direct_kernel(const CodecArgs a, const ChunkRecord* rec) {
   grid_dependency_handshake();
   const int tid = threadIdx.x, lane = tid & 31, sub = tid & 3;
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid < 8) {
@@ -73,7 +329,7 @@ __global__ void __launch_bounds__(256, 4) strided_encode_kernel(const CodecArgs 
         const uint64_t i0 = (g * 32 + sub * 8 + rr) * F + (uint64_t)fo * 8;
         Scale sc;
         sc.s = 0.0f; sc.o = 0.0f;
-        sc.inv = __uint_as_float(raw[r].z);
+        sc.inv = fabsf(__uint_as_float(raw[r].z));
         sc.base = __uint_as_float(raw[r].w);
         sc.nonfinite = raw[r].x != 0u;
         if (sc.nonfinite) {
@@ -86,42 +342,7 @@ __global__ void __launch_bounds__(256, 4) strided_encode_kernel(const CodecArgs 
       }
     }
   }
-  // rows x features -> features x rows
-  uint32_t ylo[8], yhi[8];  // per feature: codes of rows 0..3 / 4..7 of this block of eight rows
-  {
-    uint32_t o[4];
-    transpose4x4(xlo[0], xlo[1], xlo[2], xlo[3], o);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) ylo[e] = o[e];
-    transpose4x4(xlo[4], xlo[5], xlo[6], xlo[7], o);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) yhi[e] = o[e];
-    transpose4x4(xhi[0], xhi[1], xhi[2], xhi[3], o);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) ylo[4 + e] = o[e];
-    transpose4x4(xhi[4], xhi[5], xhi[6], xhi[7], o);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) yhi[4 + e] = o[e];
-  }
-#pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    uint32_t* group_words = a.payload + word0 + (uint64_t)e * K;
-    if (LAYOUT == kBitplane) {
-      // byte j = digit j of my eight rows; after the quad transpose lane q holds digit q of all 32 rows
-      const uint32_t w = quad_transpose(planes_nibbles(merge_nibbles(ylo[e], yhi[e])), lane);
-      if (active && sub < K) group_words[sub] = w;
-    } else if (K == 8) {
-      if (active) reinterpret_cast<uint2*>(group_words)[sub] = make_uint2(ylo[e], yhi[e]);
-    } else if (K == 4) {
-      const uint32_t zlo = ylo[e] | (ylo[e] >> 4), zhi = yhi[e] | (yhi[e] >> 4);
-      if (active) group_words[sub] = __byte_perm(zlo, zhi, 0x6420);
-    } else {  // K == 2: sixteen bits per eight rows
-      uint32_t zlo = ylo[e] | (ylo[e] >> 6), zhi = yhi[e] | (yhi[e] >> 6);
-      zlo |= zlo >> 12;
-      zhi |= zhi >> 12;
-      if (active) reinterpret_cast<uint16_t*>(group_words)[sub] = (uint16_t)__byte_perm(zlo, zhi, 0x0040);
-    }
-  }
+  strided_store_tile<K, LAYOUT>(a, xlo, xhi, word0, active, sub, lane);
 }
 
 template <int K, int LAYOUT, int RANGE>

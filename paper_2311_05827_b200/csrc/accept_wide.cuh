@@ -115,7 +115,9 @@ __global__ void __launch_bounds__(256) wide_range_kernel(const CodecArgs a, Chun
 }
 
 // Pass 2: one thread per chunk turns the gathered range into the side words (written to the
-// stream) and the encoder's constants (written over the record: a = 1 if the chunk is non-finite).
+// stream) and the encoder's constants (written over the record: a = 1 if the chunk is non-finite;
+// the same flag is the sign bit of inv, which is never negative otherwise, for readers that fetch
+// only inv and base).
 template <int RANGE>
 __global__ void __launch_bounds__(256) wide_finalize_kernel(const CodecArgs a, ChunkRecord* rec) {
   grid_dependency_handshake();
@@ -139,7 +141,7 @@ __global__ void __launch_bounds__(256) wide_finalize_kernel(const CodecArgs a, C
   if (sc.nonfinite) atomicOr(a.status, kDevNonFinite);
   rec[m].a = sc.nonfinite ? 1u : 0u;
   rec[m].b = 0u;
-  rec[m].inv = sc.inv;
+  rec[m].inv = sc.nonfinite ? -0.0f : sc.inv;
   rec[m].base = sc.base;
 }
 
@@ -150,7 +152,7 @@ __device__ __forceinline__ Scale scale_from_record(const ChunkRecord* rec) {
   const uint4 raw = __ldg(reinterpret_cast<const uint4*>(rec));
   Scale sc;
   sc.s = 0.0f; sc.o = 0.0f;
-  sc.inv = __uint_as_float(raw.z);
+  sc.inv = fabsf(__uint_as_float(raw.z));
   sc.base = __uint_as_float(raw.w);
   sc.nonfinite = raw.x != 0u;
   return sc;
