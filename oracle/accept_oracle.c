@@ -335,8 +335,9 @@ int oracle_bitwidth_schedule(int is_backward, int n_lr_changes) {
  *     level(c) = (+-alpha_0) + (+-alpha_1) + ... summed in fp32 in the order j = 0..k-1.
  *
  * Readings:
- *   - batch t >= 1: B^t = nearest element of P^(t-1) for every value (exact comparison of the
- *     distances; a tie goes to the lower level; codes whose levels coincide: the smallest code);
+ *   - batch t >= 1: B^t = nearest element of P^(t-1) for every value (the distances are compared
+ *     exactly, whatever the magnitudes of x and the levels; a tie goes to the lower level; codes
+ *     whose levels coincide: the smallest code);
  *     then alpha_cur = (B^T B)^-1 B^T x (Eq. 3) and alpha^t = beta alpha^(t-1) + (1-beta) alpha_cur
  *     with beta = min(0.9, (1+t)/(10+t)) (Eq. 4), all in double, rounded once to fp32.  If B^T B is
  *     singular (a pivot below 1e-9 N) alpha_cur = alpha^(t-1).
@@ -369,16 +370,52 @@ void oracle_mbq_levels(const float* alpha, uint32_t k, float* levels) {
   }
 }
 
-/* Closest value of P for every element. */
+/* s + e = a + b exactly (Knuth's two-sum; no overflow for fp32-sized inputs). */
+static void two_sum(double a, double b, double* s, double* e) {
+  double sum = a + b;
+  double bv = sum - a;
+  *e = (a - (sum - bv)) + (b - bv);
+  *s = sum;
+}
+
+/* Sign of 2x - (a + b), exactly.  -(a + b) is held as a two-term non-overlapping expansion and 2x is
+ * added to it term by term (smallest first), each step an exact two-sum; the largest non-zero term of
+ * the resulting non-overlapping expansion carries the sign of the whole sum. */
+static int sign_2x_minus_sum(float x, float a, float b) {
+  double s, e, q, h1, h2;
+  two_sum(-(double)a, -(double)b, &s, &e);
+  two_sum(2.0 * (double)x, e, &q, &h1);
+  two_sum(q, s, &q, &h2);
+  if (q != 0.0) return q > 0.0 ? 1 : -1;
+  if (h2 != 0.0) return h2 > 0.0 ? 1 : -1;
+  if (h1 != 0.0) return h1 > 0.0 ? 1 : -1;
+  return 0;
+}
+
+/* Is level a strictly closer to x than level b?  |x - a| < |x - b| decided without rounding: the
+ * differences themselves need up to 277 bits when x and the levels are far apart, so for x strictly
+ * between the two levels the test is 2x against a + b; outside, the nearer end wins. */
+static int strictly_closer(float x, float a, float b) {
+  if (a == b) return 0;
+  float lo = a < b ? a : b, hi = a < b ? b : a;
+  int lower_wins; /* 1: lo is strictly closer, 0: tie, -1: hi is strictly closer */
+  if (x <= lo) lower_wins = 1;
+  else if (x >= hi) lower_wins = -1;
+  else lower_wins = -sign_2x_minus_sum(x, lo, hi);
+  return a < b ? lower_wins > 0 : lower_wins < 0;
+}
+
+/* Closest value of P for every element (Sec. 3.3 "Forward Quantizer": each value takes the closest
+ * element of P); a tie goes to the lower level, coinciding levels to the smallest code. */
 void oracle_mbq_assign_nearest(const float* x, uint64_t n, const float* alpha, uint32_t k, uint8_t* codes) {
   float levels[256];
   oracle_mbq_levels(alpha, k, levels);
   for (uint64_t i = 0; i < n; ++i) {
     uint32_t best = 0;
-    double best_d = fabs((double)x[i] - (double)levels[0]);
     for (uint32_t c = 1; c < (1u << k); ++c) {
-      double d = fabs((double)x[i] - (double)levels[c]);
-      if (d < best_d || (d == best_d && levels[c] < levels[best])) { best = c; best_d = d; }
+      int closer = strictly_closer(x[i], levels[c], levels[best]);
+      int tie = !closer && !strictly_closer(x[i], levels[best], levels[c]);
+      if (closer || (tie && levels[c] < levels[best])) best = c;
     }
     codes[i] = (uint8_t)best;
   }

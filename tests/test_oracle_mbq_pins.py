@@ -51,6 +51,36 @@ def test_nearest_level_against_brute_force(k):
     assert np.array_equal(got[:lv.size], lv) and np.array_equal(got[lv.size:], lv[:-1])
 
 
+@pytest.mark.parametrize("alpha", [[0.9, 0.5, 0.27, 0.14], [3e-30, 1.4e-30, 0.6e-30], [2e37, 1e37], [1.0, 0.5, 0.2500001]])
+def test_nearest_level_is_exact_against_rational_arithmetic(alpha):
+    """The closest level, decided in exact rational arithmetic, for values whose distances to two
+    levels differ by less than any rounding of the differences could show: next to every midpoint,
+    next to zero (between the two innermost levels), and at the far ends of the fp32 range."""
+    from fractions import Fraction
+    alpha = np.array(alpha, dtype=np.float32)
+    levels = oracle.mbq_levels(alpha)
+    lv = np.unique(levels).astype(np.float64)
+    mid = ((lv[:-1] + lv[1:]) / 2).astype(np.float32)
+    probe = [mid]
+    up, down = mid.copy(), mid.copy()
+    for _ in range(2):
+        up, down = np.nextafter(up, np.float32(np.inf)), np.nextafter(down, np.float32(-np.inf))
+        probe += [up.copy(), down.copy()]
+    tiny = np.float32(1e-45)
+    probe.append(np.array([0.0, tiny, -tiny, 1e-38, -1e-38, 1e-20, -1e-20, 3e38, -3e38, 1e10, -1e10, 7.0, -7.0],
+                          dtype=np.float32))
+    probe = np.concatenate(probe).astype(np.float32)
+    codes = oracle.mbq_assign_nearest(probe, alpha)
+    exact = [Fraction(float(v)) for v in levels]
+    for x, c in zip(probe, codes):
+        fx = Fraction(float(x))
+        dist = [abs(fx - l) for l in exact]
+        best = min(dist)
+        # among the levels at the smallest distance: the lowest level, then the smallest code
+        want = min((i for i, d in enumerate(dist) if d == best), key=lambda i: (exact[i], i))
+        assert c == want, (x, c, want)
+
+
 def test_duplicate_levels_pick_the_smallest_code():
     alpha = np.array([1.0, 1.0], dtype=np.float32)  # codes 1 and 2 both give level 0
     codes = oracle.mbq_assign_nearest(np.array([0.0, 0.1, -0.1, 0.9], dtype=np.float32), alpha)
