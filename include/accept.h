@@ -225,7 +225,8 @@ accept_status accept_decompress_host(const accept_params* p, const void* h_strea
  * k in {2,3,4} (the paper's forward range); d_alpha_prev / d_alpha_next are DEVICE arrays of k
  * floats (they may be the same array), so successive batches chain without a host round trip.
  * The workspace (accept_mbq_workspace_size bytes, 16-byte aligned, zeroed once by the caller) holds
- * the status word and per-block partial sums (at most 161 KB).  Launches: 2 (plus 2k when init).
+ * the status word and per-block partial sums (at most 47 KB).  Launches: 2 (plus 2k when init).  The encode
+ * kernel of a batch >= 1 asks for 128 KB of dynamic shared memory per block (its search table).
  */
 typedef struct {
   uint64_t n_elems;

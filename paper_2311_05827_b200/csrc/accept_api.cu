@@ -299,6 +299,11 @@ uint32_t mbq_blocks(const accept_mbq_params* p) {
   return (uint32_t)(tiles < (uint64_t)accept::kMbqMaxBlocks ? tiles : (uint64_t)accept::kMbqMaxBlocks);
 }
 
+uint32_t mbq_residue_blocks(const accept_mbq_params* p) {
+  const uint64_t tiles = mbq_tiles(p);
+  return (uint32_t)(tiles < (uint64_t)accept::kMbqResidueBlocks ? tiles : (uint64_t)accept::kMbqResidueBlocks);
+}
+
 accept::MbqArgs mbq_args(const accept_mbq_params* p, void* d_stream, void* d_ws) {
   accept::MbqArgs a{};
   uint8_t* base = static_cast<uint8_t*>(d_stream);
@@ -310,6 +315,7 @@ accept::MbqArgs mbq_args(const accept_mbq_params* p, void* d_stream, void* d_ws)
   a.alpha_init = reinterpret_cast<float*>(ws + 16);
   a.n = p->n_elems;
   a.n_blocks = mbq_blocks(p);
+  a.n_residue_blocks = mbq_residue_blocks(p);
   a.n_tiles = mbq_tiles(p);
   a.partial = reinterpret_cast<accept::MbqPartial*>(ws + 64);
   a.residue_sum = reinterpret_cast<double*>(ws + 64 + (size_t)accept::kMbqPartialBytes * a.n_blocks);
@@ -321,14 +327,19 @@ accept::MbqArgs mbq_args(const accept_mbq_params* p, void* d_stream, void* d_ws)
 
 template <int K>
 void launch_mbq_compress(const accept::MbqArgs& a, cudaStream_t s) {
+  const dim3 grid((a.n_blocks + accept::kMbqGroups - 1) / accept::kMbqGroups);
   if (a.init) {
     for (int j = 0; j < K; ++j) {
-      launch_overlapped(accept::mbq_residue_sum_kernel<K>, dim3(a.n_blocks), 256, s, a, j);
+      launch_overlapped(accept::mbq_residue_sum_kernel<K>, dim3(a.n_residue_blocks), 256, s, a, j);
       launch_overlapped(accept::mbq_residue_finalize_kernel, dim3(1), 256, s, a, j);
     }
-    launch_overlapped(accept::mbq_encode_kernel<K, true>, dim3(a.n_blocks), 256, s, a);
+    launch_overlapped(accept::mbq_encode_kernel<K, true>, grid, accept::kMbqEncodeThreads, s, a);
   } else {
-    launch_overlapped(accept::mbq_encode_kernel<K, false>, dim3(a.n_blocks), 256, s, a);
+    // the search grid needs more dynamic shared memory than a kernel gets without opting in (the
+    // attribute is per device: set every time)
+    auto fn = accept::mbq_encode_kernel<K, false>;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, accept::kMbqGridBytes) != cudaSuccess) return;
+    launch_overlapped_shared(fn, grid, accept::kMbqEncodeThreads, accept::kMbqGridBytes, s, a);
   }
   launch_overlapped(accept::mbq_finalize_kernel<K>, dim3(1), accept::kMbqFinalizeThreads, s, a);
   g_launches.fetch_add(2 + (a.init ? 2 * K : 0), std::memory_order_relaxed);
@@ -557,8 +568,9 @@ size_t accept_mbq_compressed_size(const accept_mbq_params* p) {
 
 size_t accept_mbq_workspace_size(const accept_mbq_params* p) {
   if (accept_mbq_check_params(p) != ACCEPT_OK) return 0;
-  // status + residue coefficients (64 bytes), one 128-byte record and one double per block (at most 1184 blocks)
-  return 64 + (size_t)(accept::kMbqPartialBytes + 8) * mbq_blocks(p);
+  // status + residue coefficients (64 bytes), one 128-byte record per group of the encode pass (at most 296) and one
+  // double per block of a residue pass (at most 1184)
+  return 64 + (size_t)accept::kMbqPartialBytes * mbq_blocks(p) + 8 * (size_t)mbq_residue_blocks(p);
 }
 
 accept_status accept_mbq_compress(const accept_mbq_params* p, const float* d_x, const float* d_alpha_prev,

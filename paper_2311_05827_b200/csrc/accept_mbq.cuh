@@ -4,22 +4,30 @@
 //
 // Element i carries k signs b_i0..b_i,k-1 as the code c_i = sum_j [b_ij = +1] << j; plane j of a
 // 32-element group is basis j.  level(c) = (+-alpha_0) + ... + (+-alpha_k-1), summed in fp32 in
-// the order j = 0..k-1.  One pass over the input assigns the signs, writes the planes and gathers
-// per block what Eq. 3-5 need: counts of +1 per basis, counts of differing signs per pair of bases
-// (integers: B^T B exactly), sum of x over the +1 elements of each basis and sum of x (double).
-// A single small block then adds the per-block partials in a fixed order, solves the k x k system,
-// applies the moving average and writes the side words.  Sums are order-fixed, so results repeat
-// from run to run.
+// the order j = 0..k-1.  One pass over the input assigns the signs (nearest level through a
+// uniform grid over the span of the levels, one shared-memory lookup and one comparison per
+// element), writes the planes and gathers per group of 256 threads what Eq. 3-5 need: counts of +1
+// per basis, counts of differing signs per pair of bases (integers: B^T B exactly), sum of x over
+// the +1 elements of each basis and sum of x (double).  A single small block then adds the
+// partials in a fixed order, solves the k x k system, applies the moving average and writes the
+// side words.  Sums are order-fixed, so results repeat from run to run.
 #pragma once
 #include "accept_kernels.cuh"
 
 namespace accept {
 
-constexpr int kMbqRounds = 4;                      // octets per thread
+constexpr int kMbqRounds = 2;                      // octets per thread and tile
 constexpr int kMbqTile = kMbqRounds * 256 * 8;     // elements per block
 constexpr int kMbqPartialBytes = 128;              // per-block record in the workspace
 constexpr int kMbqFinalizeThreads = 256;           // threads of the single finalize block
-constexpr int kMbqMaxBlocks = 1184;                // 8 per SM on 148 SMs; fixed, so sums repeat on any device
+constexpr int kMbqGroups = 2;                      // 256-thread groups per block of the encode pass (one block per SM);
+                                                   // 3 groups at 80 registers were slower than 2 at 113 (measured)
+constexpr int kMbqEncodeThreads = 256 * kMbqGroups;
+constexpr int kMbqMaxBlocks = 148 * kMbqGroups;    // groups of the encode pass = records in the workspace; fixed, so sums
+                                                   // repeat on any device
+constexpr int kMbqResidueBlocks = 1184;            // blocks of a residue pass (fixed for the same reason)
+constexpr int kMbqCells = 256;                     // cells of the uniform search grid
+constexpr int kMbqGridBytes = kMbqCells * 32 * 16; // one 16-byte entry per cell and lane
 
 // Per-block partial sums (one 128-byte record per block of the encode pass).
 struct MbqPartial {
@@ -45,7 +53,8 @@ struct MbqArgs {
   double* residue_sum;      // workspace + 32: scratch of the residue passes
   uint64_t n;
   uint64_t n_tiles;         // tiles of kMbqTile elements
-  uint32_t n_blocks;        // blocks of the encode / residue passes = records in the workspace
+  uint32_t n_blocks;        // 256-thread groups of the encode pass = records in the workspace
+  uint32_t n_residue_blocks;  // blocks of a residue pass = doubles in the workspace
   uint32_t k, batch_index, init;
 };
 
@@ -74,8 +83,9 @@ __device__ __forceinline__ float mbq_level(const float* alpha, uint32_t c) {
 }
 
 // Search table for the nearest level: thresholds between neighbouring sorted levels and the code
-// of each sorted position.  A threshold is the midpoint rounded DOWN to fp32: for an fp32 x,
-// "x > threshold" is then exactly "x is above the true midpoint" (a tie goes to the lower level).
+// of each sorted position.  A threshold is the midpoint rounded DOWN to fp32 (the sum and, for
+// subnormal levels, the halving too): for an fp32 x, "x > threshold" is then exactly "x is above
+// the true midpoint" (a tie goes to the lower level).  Level sums must stay below the fp32 maximum.
 // Positions whose levels coincide all map to the smallest code among them.
 template <int K>
 struct MbqTable {
@@ -105,7 +115,7 @@ __device__ void mbq_build_table(const float* alpha_global, MbqTable<K>* t, float
     t->code[rank] = first;
   }
   __syncthreads();
-  if (tid >= 1 && tid < L) t->thr[tid] = __fmul_rn(__fadd_rd(s_sorted[tid - 1], s_sorted[tid]), 0.5f);
+  if (tid >= 1 && tid < L) t->thr[tid] = __fmul_rd(__fadd_rd(s_sorted[tid - 1], s_sorted[tid]), 0.5f);
   if (tid == 0) t->thr[0] = 0.0f;
   __syncthreads();
 }
@@ -121,6 +131,111 @@ __device__ __forceinline__ uint32_t mbq_nearest_code(const MbqTable<K>& t, float
   for (int step = L / 2; step >= 1; step >>= 1)
     if (x > *reinterpret_cast<const float*>(thr + off + 4 * step)) off += 4 * step;
   return *reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(t.code) + off);
+}
+
+// ---- signs as flag bytes ------------------------------------------------------------------------
+//
+// Inside the encode pass the k signs of an element travel as a word with one FLAG BYTE per basis:
+// byte j = 0x10 when b_j = +1, else 0.  Two things come cheaply from that form:
+//  * moved to byte 3 of the high word of a double (low word 0), a flag byte is the number
+//    2^-767 (exponent field 0x100) or +0: "add x to the sum of basis j when b_j = +1" becomes one
+//    byte permute and one fused multiply-add, acc += x * flag.  Scaling by a power of two is exact
+//    (|x| from 2^-149 to 2^128 stays far inside the range of a double), so the sums are the plain
+//    ones times 2^-767 and are scaled back exactly at the end;
+//  * the plane form of an octet (byte j = the signs of basis j of its 8 elements) is a sum of the
+//    eight words times 1, 2, 4, 8: integer multiply-adds instead of byte permutes and bit swaps.
+constexpr uint32_t kMbqFlag = 0x10u;
+
+// code (bit j = [b_j = +1]) -> flag bytes
+__device__ __forceinline__ uint32_t mbq_flags_of_code(uint32_t c) {
+  return ((c * 0x00204081u) & 0x01010101u) << 4;
+}
+
+// acc += x * (flag byte J of `flags` as a double: 2^-767 or +0)
+template <int J>
+__device__ __forceinline__ void mbq_add_flagged(double& acc, double x, uint32_t flags) {
+  acc = __fma_rn(x, __hiloint2double((int)__byte_perm(flags, 0u, 0x0444u | ((uint32_t)J << 12)), 0), acc);
+}
+
+// flag words of the 8 elements of an octet -> plane form (bit 8*j + e = [b_j of element e = +1])
+__device__ __forceinline__ uint32_t mbq_planes_of_flags(const uint32_t (&f)[8]) {
+  const uint32_t lo = f[0] + 2u * f[1] + 4u * f[2] + 8u * f[3];  // bits 4..7 of every byte: elements 0..3
+  const uint32_t hi = f[4] + 2u * f[5] + 4u * f[6] + 8u * f[7];  // bits 4..7 of every byte: elements 4..7
+  return (lo >> 4) | hi;
+}
+
+// Nearest level through a uniform grid.  The span of the levels (with a margin) is cut into 256
+// cells; cell_offset() is a non-decreasing function of x, so every x of a cell below the cell of a
+// threshold lies below that threshold and every x of a cell above it lies above.  When no cell
+// holds more than one threshold, one comparison with "the threshold inside my cell" finishes the
+// search: entry = {that threshold (+inf if the cell has none), flag bytes of the code below it,
+// flag bytes of the code above it, 0}.  The decisions are the ones of the threshold search, exactly;
+// when two thresholds share a cell (coinciding or very close levels), or a level is not finite,
+// the grid is marked unusable and the kernel searches the sorted thresholds instead.
+//
+// The table is stored once per lane, entry (cell, lane) at byte 512 * cell + 16 * lane: whatever
+// cells the 32 lanes of a warp ask for, lane l only ever touches its own 16-byte column of the
+// banks, so a lookup is one 128-bit shared load without bank conflicts (a single shared copy
+// cost 8.6 wavefronts per load on post-ReLU data and bound the pass).  128 KB per block.
+struct MbqGridInfo {
+  float scale;  // 1 / (2 * span)
+  int usable;
+};
+
+// Byte offset of entry (cell of x, lane); lane_bytes = 16 * lane.  Two fused multiply-adds on the
+// FMA pipe and one logic operation: the first maps the span onto [0, 1] and saturates, the second
+// leaves round(255 * 512 * t) in the low mantissa bits; keeping bits 9..16 of it gives
+// 512 * floor(that / 512).  NaN goes to cell 0.
+__device__ __forceinline__ uint32_t mbq_cell_offset(float x, float scale, uint32_t lane_bytes) {
+  float t;
+  asm("fma.rn.sat.f32 %0, %1, %2, 0f3F000000;" : "=f"(t) : "f"(x), "f"(scale));
+  return (__float_as_uint(__fmaf_rn(t, 130560.0f, kMagic)) & 0x1FE00u) | lane_bytes;
+}
+
+// Called by all threads of the block.
+template <int K>
+__device__ void mbq_build_grid(const MbqTable<K>& t, const float* s_level, MbqGridInfo* info, uint4* cells, int tid,
+                               int n_threads) {
+  constexpr int L = 1 << K;
+  __shared__ uint32_t s_cell_of[L];
+  __shared__ uint4 s_entry[kMbqCells];
+  if (tid == 0) {
+    float amax = 0.0f;
+    bool finite = true;
+    for (int c = 0; c < L; ++c) {
+      finite = finite && is_finite_bits(s_level[c]);
+      amax = fmaxf(amax, fabsf(s_level[c]));
+    }
+    const float scale = __fdiv_rn(0.5f, __fmul_rn(amax, 1.03125f));
+    info->scale = scale;
+    info->usable = (finite && amax > 0.0f && is_finite_bits(scale)) ? 1 : 0;
+  }
+  __syncthreads();
+  if (tid >= 1 && tid < L) s_cell_of[tid] = mbq_cell_offset(t.thr[tid], info->scale, 0u) >> 9;
+  __syncthreads();
+  if (tid < kMbqCells) {
+    int below = 0, inside = 0;
+    float thr = __int_as_float(0x7f800000);
+    for (int m = 1; m < L; ++m) {
+      const uint32_t c = s_cell_of[m];
+      below += (c < (uint32_t)tid) ? 1 : 0;
+      if (c == (uint32_t)tid) { ++inside; thr = t.thr[m]; }
+    }
+    const uint32_t lo = t.code[below], hi = t.code[below + 1 < L ? below + 1 : L - 1];
+    s_entry[tid] = make_uint4(__float_as_uint(thr), mbq_flags_of_code(lo), mbq_flags_of_code(hi), 0u);
+    if (inside > 1) info->usable = 0;
+  }
+  __syncthreads();
+  if (info->usable)
+    for (int i = tid; i < kMbqCells * 32; i += n_threads) cells[i] = s_entry[i >> 5];
+  __syncthreads();
+}
+
+// flag bytes of the nearest level's code
+__device__ __forceinline__ uint32_t mbq_grid_flags(const uint4* cells, float scale, uint32_t lane_bytes, float x) {
+  const uint4 e = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(cells) +
+                                                  mbq_cell_offset(x, scale, lane_bytes));
+  return (x > __uint_as_float(e.x)) ? e.z : e.y;
 }
 
 // Signs of the successive residues with the given coefficients (residue method): bit j = [r_j >= 0].
@@ -203,7 +318,7 @@ __global__ void __launch_bounds__(256) mbq_residue_finalize_kernel(const MbqArgs
   __shared__ double s_part[256];
   const int tid = threadIdx.x;
   double s = 0.0;
-  for (uint32_t b = tid; b < a.n_blocks; b += 256) s += a.residue_sum[b];
+  for (uint32_t b = tid; b < a.n_residue_blocks; b += 256) s += a.residue_sum[b];
   s_part[tid] = s;
   __syncthreads();
   if (tid == 0) {
@@ -213,15 +328,140 @@ __global__ void __launch_bounds__(256) mbq_residue_finalize_kernel(const MbqArgs
   }
 }
 
-// Assign the signs, write the planes, gather the per-block sums.
+// How the signs of an element are found.
+constexpr int kMbqResidue = 0, kMbqSearch = 1, kMbqGrid = 2;
+
+// Running sums of one thread over all its tiles.
+template <int K>
+struct MbqSums {
+  double plus[K], sum_x;
+  uint32_t count, differ[3];  // of basis q = lane & 3, and of the pairs (q, q ^ d)
+};
+
+// The octets of thread tid of a tile: FULL = every element of the tile exists.
+template <bool FULL>
+__device__ __forceinline__ void mbq_load_tile(const MbqArgs& a, uint64_t tile, int tid, float (&v)[kMbqRounds][8]) {
+  const uint64_t oct0 = tile * (kMbqRounds * 256) + tid;
+#pragma unroll
+  for (int r = 0; r < kMbqRounds; ++r) {
+    const uint64_t oct = oct0 + r * 256;
+    if (FULL) {
+      ld_octet(a.x + oct * 8, v[r]);
+    } else if (oct < (a.n + 7) / 8) {
+      mbq_ld_octet(a.x, a.n, oct, v[r]);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[r][e] = 0.0f;
+    }
+  }
+}
+
+// One tile of kMbqTile elements, coded by one group of 256 threads (tid = index in the group): assign
+// the signs, write the planes, add to the thread's sums.
+template <int K, int MODE, bool FULL>
+__device__ __forceinline__ void mbq_encode_tile(const MbqArgs& a, uint64_t tile, int tid, int lane,
+                                                const float (&v)[kMbqRounds][8], const float (&alpha)[K],
+                                                const MbqTable<K>& table, const uint4* cells, float scale,
+                                                MbqSums<K>& sums) {
+  const uint64_t n_oct_stored = ((a.n + 31) / 32) * 4;
+  const uint64_t oct0 = tile * (kMbqRounds * 256) + tid;
+  const int q = lane & 3;
+  const uint32_t lane_bytes = 16u * (uint32_t)lane;
+#pragma unroll
+  for (int r = 0; r < kMbqRounds; ++r) {
+    const uint64_t oct = oct0 + r * 256;
+    uint32_t f[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      if (MODE == kMbqResidue) {
+        float res;
+        f[e] = mbq_flags_of_code(mbq_residue_code<K>(alpha, v[r][e], K, &res));
+      } else if (MODE == kMbqSearch) {
+        f[e] = mbq_flags_of_code(mbq_nearest_code<K>(table, v[r][e]));
+      } else {
+        f[e] = mbq_grid_flags(cells, scale, lane_bytes, v[r][e]);
+      }
+    }
+    if (!FULL) {
+      // elements of this octet that exist; signs past the end are zero bits (their values were loaded as 0)
+      const int valid = (oct * 8 + 8 <= a.n) ? 8 : ((oct * 8 < a.n) ? (int)(a.n - oct * 8) : 0);
+      if (valid < 8) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          if (e >= valid) f[e] = 0;
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const double xd = (double)v[r][e];  // 0 past the end
+      sums.sum_x += xd;
+      mbq_add_flagged<0>(sums.plus[0], xd, f[e]);
+      mbq_add_flagged<1>(sums.plus[1], xd, f[e]);
+      if constexpr (K > 2) mbq_add_flagged<2>(sums.plus[2], xd, f[e]);
+      if constexpr (K > 3) mbq_add_flagged<3>(sums.plus[3], xd, f[e]);
+    }
+    // after the quad transpose lane q holds the 32 signs of basis q of its group: counts of +1 and,
+    // against the words of the other three lanes of the quad, counts of differing signs
+    const uint32_t w = quad_transpose(mbq_planes_of_flags(f), lane);
+    if ((FULL || oct < n_oct_stored) && q < K) a.payload[(oct >> 2) * K + q] = w;
+    sums.count += __popc(w);
+#pragma unroll
+    for (int d = 1; d < 4; ++d) {
+      const uint32_t other = __shfl_xor_sync(0xffffffffu, w, d);
+      sums.differ[d - 1] += __popc(w ^ other);
+    }
+  }
+}
+
+// A group walks over tiles with a stride of the number of groups and keeps its sums in registers: the
+// group-level reduction and the record in the workspace are paid once per group, not once per tile.
+// The loads of a group's next tile are in flight while it codes the current one (two register
+// buffers, the loop unrolled by two so that both are addressed statically).
+template <int K, int MODE>
+__device__ __forceinline__ void mbq_encode_tiles(const MbqArgs& a, uint32_t group, int tid, int lane,
+                                                 const float (&alpha)[K], const MbqTable<K>& table, const uint4* cells,
+                                                 float scale, MbqSums<K>& sums) {
+  if (group >= a.n_blocks) return;
+  const uint64_t full_tiles = a.n / kMbqTile, stride = a.n_blocks;
+  float v0[kMbqRounds][8], v1[kMbqRounds][8];
+  uint64_t tile = group;
+  if (tile < full_tiles) mbq_load_tile<true>(a, tile, tid, v0);
+  while (tile < full_tiles) {
+    const uint64_t t1 = tile + stride;
+    if (t1 < full_tiles) mbq_load_tile<true>(a, t1, tid, v1);
+    mbq_encode_tile<K, MODE, true>(a, tile, tid, lane, v0, alpha, table, cells, scale, sums);
+    tile = t1;
+    if (t1 >= full_tiles) break;
+    const uint64_t t2 = t1 + stride;
+    if (t2 < full_tiles) mbq_load_tile<true>(a, t2, tid, v0);
+    mbq_encode_tile<K, MODE, true>(a, t1, tid, lane, v1, alpha, table, cells, scale, sums);
+    tile = t2;
+  }
+  // the ragged last tile of the tensor, if there is one, is the last tile of its group
+  if (tile < a.n_tiles) {
+    mbq_load_tile<false>(a, tile, tid, v0);
+    mbq_encode_tile<K, MODE, false>(a, tile, tid, lane, v0, alpha, table, cells, scale, sums);
+  }
+}
+
+// Assign the signs, write the planes, gather the sums.  One block of kMbqGroups groups of 256 threads
+// per SM; a group does what a 256-thread block would (its own tiles, its own record in the
+// workspace), the groups of a block share the search tables.  Dynamic shared memory: the search
+// grid (kMbqGridBytes), not needed when INIT.
 template <int K, bool INIT>
-__global__ void __launch_bounds__(256) mbq_encode_kernel(const MbqArgs a) {
+__global__ void __launch_bounds__(kMbqEncodeThreads, 1) mbq_encode_kernel(const MbqArgs a) {
   grid_dependency_handshake();
+  extern __shared__ uint4 s_cells[];
   __shared__ MbqTable<K> s_table;
+  __shared__ MbqGridInfo s_grid;
   __shared__ float s_level[16];
-  __shared__ double s_dbl[8][K + 1];
-  __shared__ uint32_t s_cnt[10];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  __shared__ double s_dbl[kMbqGroups][8][K + 1];
+  __shared__ uint32_t s_cnt[kMbqGroups][10];
+  const int lane = threadIdx.x & 31;
+  const int g = threadIdx.x >> 8;            // group in the block
+  const int tid = threadIdx.x & 255;         // thread in the group
+  const int warp = tid >> 5;                 // warp in the group
+  const uint32_t group = blockIdx.x * kMbqGroups + g;
   float alpha[K];
   if (INIT) {
 #pragma unroll
@@ -229,84 +469,41 @@ __global__ void __launch_bounds__(256) mbq_encode_kernel(const MbqArgs a) {
   } else {
 #pragma unroll
     for (int j = 0; j < K; ++j) alpha[j] = 0.0f;
-    mbq_build_table<K>(a.alpha_prev, &s_table, s_level, tid);
+    mbq_build_table<K>(a.alpha_prev, &s_table, s_level, threadIdx.x);
+    mbq_build_grid<K>(s_table, s_level, &s_grid, s_cells, threadIdx.x, kMbqEncodeThreads);
   }
-  if (tid < 10) s_cnt[tid] = 0;
+  if (tid < 10) s_cnt[g][tid] = 0;
   __syncthreads();
 
-  const uint64_t n_oct = (a.n + 7) / 8;
-  const uint64_t n_oct_stored = ((a.n + 31) / 32) * 4;
-  double plus[K], sum_x = 0.0;
-  uint32_t my_count = 0, my_differ[3] = {0, 0, 0};  // of basis q = lane & 3, and of the pairs (q, q ^ d)
+  MbqSums<K> sums;
+  sums.sum_x = 0.0;
+  sums.count = 0;
 #pragma unroll
-  for (int j = 0; j < K; ++j) plus[j] = 0.0;
+  for (int j = 0; j < K; ++j) sums.plus[j] = 0.0;
+#pragma unroll
+  for (int d = 0; d < 3; ++d) sums.differ[d] = 0;
+
+  if (INIT) mbq_encode_tiles<K, kMbqResidue>(a, group, tid, lane, alpha, s_table, s_cells, 0.0f, sums);
+  else if (s_grid.usable) mbq_encode_tiles<K, kMbqGrid>(a, group, tid, lane, alpha, s_table, s_cells, s_grid.scale, sums);
+  else mbq_encode_tiles<K, kMbqSearch>(a, group, tid, lane, alpha, s_table, s_cells, 0.0f, sums);
 
   const int q = lane & 3;
-  // a block walks over tiles with a stride of the grid and keeps its sums in registers: the block-level
-  // reduction and the record in the workspace are paid once per block, not once per tile
-  for (uint64_t tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x) {
-  float v[kMbqRounds][8];
+  double (&plus)[K] = sums.plus;
 #pragma unroll
-  for (int r = 0; r < kMbqRounds; ++r) {
-    const uint64_t oct = tile * (kMbqRounds * 256) + r * 256 + tid;
-    if (oct < n_oct) {
-      mbq_ld_octet(a.x, a.n, oct, v[r]);
-    } else {
-#pragma unroll
-      for (int e = 0; e < 8; ++e) v[r][e] = 0.0f;
-    }
-  }
-#pragma unroll
-  for (int r = 0; r < kMbqRounds; ++r) {
-    const uint64_t oct = tile * (kMbqRounds * 256) + r * 256 + tid;
-    // elements of this octet that exist (8 for all but the last octets of the tensor)
-    const int valid = (oct * 8 + 8 <= a.n) ? 8 : ((oct * 8 < a.n) ? (int)(a.n - oct * 8) : 0);
-    uint32_t c[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      if (INIT) {
-        float res;
-        c[e] = mbq_residue_code<K>(alpha, v[r][e], K, &res);
-      } else {
-        c[e] = mbq_nearest_code<K>(s_table, v[r][e]);
-      }
-    }
-    if (valid < 8) {  // codes of elements past the end are zero (their values were loaded as 0)
-#pragma unroll
-      for (int e = 0; e < 8; ++e)
-        if (e >= valid) c[e] = 0;
-    }
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const double xd = (double)v[r][e];  // 0 past the end
-      sum_x += xd;
-#pragma unroll
-      for (int j = 0; j < K; ++j) add_if(plus[j], xd, c[e] & (1u << j));
-    }
-    const uint32_t xlo = pack_bytes<0>(c[0], c[1], c[2], c[3]);
-    const uint32_t xhi = pack_bytes<0>(c[4], c[5], c[6], c[7]);
-    const bool stored = oct < n_oct_stored;
-    // after the quad transpose lane q holds the 32 signs of basis q of its group: counts of +1 and,
-    // against the words of the other three lanes of the quad, counts of differing signs
-    const uint32_t w = store_bitplane_guarded<K>(a.payload, oct >> 2, xlo, xhi, lane, stored);
-    my_count += __popc(w);
-#pragma unroll
-    for (int d = 1; d < 4; ++d) {
-      const uint32_t other = __shfl_xor_sync(0xffffffffu, w, d);
-      my_differ[d - 1] += __popc(w ^ other);
-    }
-  }
-  }  // tiles
+  for (int j = 0; j < K; ++j) plus[j] *= 0x1p767;  // the flag factor was 2^-767: exact
+  const double sum_x = sums.sum_x;
+  uint32_t my_count = sums.count;
+  uint32_t (&my_differ)[3] = sums.differ;
 
-  // block sums in a fixed order: lanes by butterfly, warps one after the other
+  // group sums in a fixed order: lanes by butterfly, warps one after the other
 #pragma unroll
   for (int j = 0; j < K; ++j) {
     const double s = warp_sum(plus[j]);
-    if (lane == 0) s_dbl[warp][j] = s;
+    if (lane == 0) s_dbl[g][warp][j] = s;
   }
   {
     const double s = warp_sum(sum_x);
-    if (lane == 0) s_dbl[warp][K] = s;
+    if (lane == 0) s_dbl[g][warp][K] = s;
   }
   // lanes with the same q hold partial counts of the same basis / pairs: add over the eight quads
 #pragma unroll
@@ -316,33 +513,33 @@ __global__ void __launch_bounds__(256) mbq_encode_kernel(const MbqArgs a) {
     for (int i = 0; i < 3; ++i) my_differ[i] += __shfl_xor_sync(0xffffffffu, my_differ[i], d);
   }
   if (lane < 4) {
-    atomicAdd(&s_cnt[q], my_count);
+    atomicAdd(&s_cnt[g][q], my_count);
 #pragma unroll
     for (int d = 1; d < 4; ++d) {
       const int other = q ^ d;
       if (q < other) {  // each pair once; pair index in the order (0,1) (0,2) (0,3) (1,2) (1,3) (2,3)
         const int pair = (q == 0) ? other - 1 : (q == 1 ? other + 1 : 5);
-        atomicAdd(&s_cnt[4 + pair], my_differ[d - 1]);
+        atomicAdd(&s_cnt[g][4 + pair], my_differ[d - 1]);
       }
     }
   }
   __syncthreads();
-  if (tid == 0) {
+  if (tid == 0 && group < a.n_blocks) {
     MbqPartial out;
 #pragma unroll
     for (int j = 0; j < 4; ++j) { out.plus[j] = 0.0; out.count[j] = 0; }
     for (int j = 0; j < K; ++j) {
       double s = 0.0;
-      for (int w = 0; w < 8; ++w) s += s_dbl[w][j];
+      for (int w = 0; w < 8; ++w) s += s_dbl[g][w][j];
       out.plus[j] = s;
-      out.count[j] = s_cnt[j];
+      out.count[j] = s_cnt[g][j];
     }
     double s = 0.0;
-    for (int w = 0; w < 8; ++w) s += s_dbl[w][K];
+    for (int w = 0; w < 8; ++w) s += s_dbl[g][w][K];
     out.sum_x = s;
-    for (int p = 0; p < 6; ++p) out.differ[p] = s_cnt[4 + p];
+    for (int p = 0; p < 6; ++p) out.differ[p] = s_cnt[g][4 + p];
     for (int p = 0; p < 12; ++p) out.pad[p] = 0;
-    a.partial[blockIdx.x] = out;
+    a.partial[group] = out;
   }
 }
 

@@ -97,6 +97,38 @@ def test_mbq_ties_duplicates_and_unsorted_coefficients():
         check_mbq(probe, k, 2, False, alpha_prev)
 
 
+@pytest.mark.parametrize("alpha_prev", [
+    [0.9, 0.5, 0.27, 0.14],                # well separated levels: the grid search is used
+    [1.5829446, 0.88997394, 0.48820832, 0.29352355],
+    [1.0, 0.5, 0.25, 0.125 + 1e-4],        # two thresholds 2e-4 apart share a cell: threshold search instead
+    [1.0, 0.5, 0.2500001],                 # nearly coinciding levels
+    [3e-30, 1.4e-30, 0.6e-30],             # tiny coefficients (the grid's scale is near 1e29)
+    [2e37, 1e37],                          # huge ones (levels up to 3e37)
+    [1e-39, 4e-40],                        # subnormal coefficients: scale overflows, no grid
+    [0.7, 0.3],
+])
+def test_mbq_level_search_at_thresholds_and_extremes(alpha_prev):
+    """Every decision of the nearest-level search: values on, just below and just above each midpoint
+    between neighbouring levels, a dense sweep over the span of the levels, and the extremes of fp32."""
+    alpha_prev = np.array(alpha_prev, dtype=np.float32)
+    k = alpha_prev.size
+    lv = np.unique(oracle.mbq_levels(alpha_prev)).astype(np.float64)
+    mid = ((lv[:-1] + lv[1:]) / 2).astype(np.float32)
+    near = [mid]
+    up, down = mid.copy(), mid.copy()
+    for _ in range(3):
+        up, down = np.nextafter(up, np.float32(np.inf)), np.nextafter(down, np.float32(-np.inf))
+        near += [up.copy(), down.copy()]
+    span = float(np.abs(lv).max())
+    sweep = np.linspace(-1.25 * span, 1.25 * span, 150001).astype(np.float32)
+    tiny = np.float32(1e-45)
+    extremes = np.array([0.0, -0.0, tiny, -tiny, 1e-38, -1e-38, 3e38, -3e38, 1.0, -1.0], dtype=np.float32)
+    probe = np.concatenate(near + [sweep, extremes, lv.astype(np.float32),
+                                   workloads.random_tensor(4000, k, "wide") * np.float32(span * 2.0 ** -20)]).astype(np.float32)
+    probe = probe[np.isfinite(probe)]
+    check_mbq(probe, k, 4, False, alpha_prev)
+
+
 def test_mbq_singular_system_keeps_alpha():
     x = np.abs(workloads.random_tensor(5000, 3, "normal")) + 10
     alpha_prev = np.array([1.0, 0.5], dtype=np.float32)
