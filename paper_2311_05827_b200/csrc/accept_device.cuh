@@ -241,18 +241,42 @@ __device__ __forceinline__ uint32_t pack_bytes(uint32_t b0, uint32_t b1, uint32_
   return __byte_perm(p01, p23, 0x5410);
 }
 
+// The same with the COMPLEMENT of the element's random word passed in: (~g) >> 8 is what Eq. 7's fixed
+// point form adds, and the complement of a lane word costs nothing extra: ~(h * M) = (-h) * M - 1
+// is one multiply-add like h * M itself, so the element is left with one add and one shift-add.
+template <int K, int RANGE>
+__device__ __forceinline__ uint32_t quantize_stochastic_word_not(float x, const Scale& sc, uint32_t g_not) {
+  constexpr int ZP = (RANGE == kAbsMax) ? (1 << (K - 1)) : 0;
+  constexpr float kTop = (RANGE == kAbsMax) ? (float)((1 << (K - 1)) - 1) : (float)((1 << K) - 1);
+  const float d = (RANGE == kAbsMax) ? x : __fsub_rn(x, sc.base);
+  const float t = fminf(__fmul_rn(d, sc.inv), kTop);
+  const float t24 = __fmul_rn(t, 16777216.0f);  // exact scaling
+  const uint32_t tc = (RANGE == kAbsMax) ? (uint32_t)__float2int_ru(t24) : __float2uint_ru(t24);
+  return (tc + ((uint32_t)ZP << 24)) + (g_not >> 8);
+}
+
+// ~lane_word(h, m), from h_not = ~h and h_neg = -h
+__device__ __forceinline__ uint32_t lane_word_not(uint32_t h_not, uint32_t h_neg, int m) {
+  return m == 0 ? h_not : h_neg * (m == 1 ? 0x9E3779B1u : (m == 2 ? 0x85EBCA77u : 0xC2B2AE3Du)) + 0xFFFFFFFFu;
+}
+
 // Stochastic codes of an octet whose first counter sits at position OFF of its quad; quad_lo/key
 // address that quad.
 template <int K, int RANGE, int OFF>
 __device__ __forceinline__ void quantize_octet_stochastic(const float (&v)[8], const Scale& sc, uint32_t quad_lo,
                                                           uint32_t key, uint32_t (&b)[8]) {
   constexpr int NQ = (OFF == 0) ? 2 : 3;
-  uint32_t h[NQ];
+  uint32_t h_not[NQ], h_neg[NQ];
 #pragma unroll
-  for (int p = 0; p < NQ; ++p) h[p] = Rng::quad_hash(quad_lo + p, key);
+  for (int p = 0; p < NQ; ++p) {
+    const uint32_t h = Rng::quad_hash(quad_lo + p, key);
+    h_not[p] = ~h;
+    h_neg[p] = 0u - h;
+  }
 #pragma unroll
   for (int e = 0; e < 8; ++e)
-    b[e] = quantize_stochastic_word<K, RANGE>(v[e], sc, lane_word(h[(e + OFF) >> 2], (e + OFF) & 3));
+    b[e] = quantize_stochastic_word_not<K, RANGE>(v[e], sc,
+                                                  lane_word_not(h_not[(e + OFF) >> 2], h_neg[(e + OFF) >> 2], (e + OFF) & 3));
 }
 
 // Quantizes an octet.  xlo holds the codes of elements 0..3 one per byte, xhi those of 4..7.
@@ -279,6 +303,50 @@ __device__ __forceinline__ void quantize_octet(const float (&v)[8], const Scale&
     for (int e = 0; e < 8; ++e) b[e] = quantize_nearest_word<K, RANGE>(v[e], sc);
     xlo = pack_bytes<0>(b[0], b[1], b[2], b[3]);
     xhi = pack_bytes<0>(b[4], b[5], b[6], b[7]);
+  }
+}
+
+// Quantizes the R octets of a thread; round r starts r * stride counters (a multiple of 8) after the
+// thread's first one.  Where a thread's counters sit in their quads, and whether the quad index
+// wraps inside the thread's span, is the same for all R octets (and, but for the wrap, for every
+// thread of the launch): the case is chosen once here and the octets are coded without further
+// branches.  No shuffles inside: threads may take different cases.
+template <int K, int RANGE, int R, int OFF>
+__device__ __forceinline__ void quantize_rounds_stochastic(const float (&v)[R][8], const Scale& sc, const RngThread& rt,
+                                                           uint32_t stride, uint32_t (&xlo)[R], uint32_t (&xhi)[R]) {
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    uint32_t b[8];
+    quantize_octet_stochastic<K, RANGE, OFF>(v[r], sc, rt.quad_lo + (stride * r) / 4, rt.key, b);
+    xlo[r] = pack_bytes<3>(b[0], b[1], b[2], b[3]);
+    xhi[r] = pack_bytes<3>(b[4], b[5], b[6], b[7]);
+  }
+}
+
+template <int K, int RANGE, int ROUND, int R>
+__device__ __forceinline__ void quantize_rounds(const float (&v)[R][8], const Scale& sc, const Rng& rng, const RngThread& rt,
+                                                uint32_t stride, uint32_t (&xlo)[R], uint32_t (&xhi)[R]) {
+  if (ROUND == kNearest) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) quantize_octet<K, RANGE, kNearest>(v[r], sc, rng, rt, 0u, xlo[r], xhi[r]);
+    return;
+  }
+  switch (rt.fast ? rt.off : 4) {
+    case 0: quantize_rounds_stochastic<K, RANGE, R, 0>(v, sc, rt, stride, xlo, xhi); break;
+    case 1: quantize_rounds_stochastic<K, RANGE, R, 1>(v, sc, rt, stride, xlo, xhi); break;
+    case 2: quantize_rounds_stochastic<K, RANGE, R, 2>(v, sc, rt, stride, xlo, xhi); break;
+    case 3: quantize_rounds_stochastic<K, RANGE, R, 3>(v, sc, rt, stride, xlo, xhi); break;
+    default:  // the quad index's low word (or the counter itself) wraps somewhere in this thread's span
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        uint32_t b[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          b[e] = quantize_stochastic_word<K, RANGE>(v[r][e], sc, rng.word(rt.ctr_first + stride * r + e));
+        xlo[r] = pack_bytes<3>(b[0], b[1], b[2], b[3]);
+        xhi[r] = pack_bytes<3>(b[4], b[5], b[6], b[7]);
+      }
+      break;
   }
 }
 

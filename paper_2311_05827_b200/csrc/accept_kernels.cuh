@@ -232,16 +232,16 @@ __global__ void __launch_bounds__(BLOCK_MAX, BLOCK_MAX == 256 ? (R <= 2 ? 6 : 4)
   const Rng rng{(uint32_t)a.seed, (uint32_t)(a.seed >> 32)};
   RngThread rt;
   if (ROUND == kStochastic) rt.init(rng, a.rng_offset + e0 + 8ull * gt, 8u * (R - 1) * tpc + 8u);
+  uint32_t xlo[R], xhi[R];
+  quantize_rounds<K, RANGE, ROUND, R>(v, sc, rng, rt, 8u * tpc, xlo, xhi);
 #pragma unroll
   for (int r = 0; r < R; ++r) {
     const uint64_t oct = e0 / 8 + (r * tpc + gt);  // global octet index
-    uint32_t xlo, xhi;
-    quantize_octet<K, RANGE, ROUND>(v[r], sc, rng, rt, 8u * r * tpc, xlo, xhi);
     if (LAYOUT == kInterleaved) {
-      if (active) store_interleaved<K>(a.payload, oct, xlo, xhi);
+      if (active) store_interleaved<K>(a.payload, oct, xlo[r], xhi[r]);
     } else {
       // shuffles inside: every lane takes part; an idle group rewrites nothing
-      if (active) store_bitplane<K>(a.payload, oct >> 2, xlo, xhi, lane);
+      if (active) store_bitplane<K>(a.payload, oct >> 2, xlo[r], xhi[r], lane);
     }
   }
 }

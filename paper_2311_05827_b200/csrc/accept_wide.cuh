@@ -180,17 +180,19 @@ __global__ void __launch_bounds__(256, R <= 2 ? 5 : 4) wide_encode_kernel(const 
 #pragma unroll
     for (int r = 0; r < R; ++r) ld_octet(a.x + (oct0 + r * 256) * 8, v[r]);
     const Scale sc = scale_from_record(rec + tile_chunk);
+    if (sc.nonfinite) {
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[r][i] = 0.0f;
+    }
+    uint32_t xlo[R], xhi[R];
+    quantize_rounds<K, RANGE, ROUND, R>(v, sc, rng, rt, 8u * 256u, xlo, xhi);
 #pragma unroll
     for (int r = 0; r < R; ++r) {
       const uint64_t oct = oct0 + r * 256;
-      if (sc.nonfinite) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) v[r][i] = 0.0f;
-      }
-      uint32_t xlo, xhi;
-      quantize_octet<K, RANGE, ROUND>(v[r], sc, rng, rt, 8u * r * 256u, xlo, xhi);
-      if (LAYOUT == kInterleaved) store_interleaved<K>(a.payload, oct, xlo, xhi);
-      else store_bitplane<K>(a.payload, oct >> 2, xlo, xhi, lane);
+      if (LAYOUT == kInterleaved) store_interleaved<K>(a.payload, oct, xlo[r], xhi[r]);
+      else store_bitplane<K>(a.payload, oct >> 2, xlo[r], xhi[r], lane);
     }
     return;
   }
