@@ -464,6 +464,8 @@ def sweep(A, torch, peak, args):
             torch.cuda.empty_cache()
         if name in ("cfg3_grad", "cfg4_hidden"):
             rows.append(sweep_per_tensor(A, torch, peak, name, spec, x_host))
+        if name == "cfg3_grad":  # the paper's backward encoder: stochastic codes packed along the batch dimension
+            rows.append(sweep_batch_groups(A, torch, peak, name, spec, x_host))
         if name == "cfg3_act":
             rows.extend(sweep_mbq(A, torch, peak, name, spec, x_host))
             rows.append(sweep_batch_groups(A, torch, peak, name, spec, x_host))
