@@ -316,6 +316,33 @@ def _modes_of(spec):
     return [(m.k, m.range, m.round, m.layout) for m in spec.headline + spec.also]
 
 
+def _random_case(i):
+    """Seeded draw of (n, chunk, mode, seed, counter offset, value kind) for the property test."""
+    rng = np.random.default_rng([20231105, i])
+    n = int(rng.choice([rng.integers(1, 600), rng.integers(600, 70000), rng.integers(70000, 400000)]))
+    chunk = int(rng.choice([32, 64, 96, 256, 512, 1024, 1504, 2048, 4096, 8192, 16384, 32768, 33024, 65536,
+                            32 * int(rng.integers(1, 3000))]))
+    mode = modes()[int(rng.integers(0, len(modes())))]
+    seed = int(rng.integers(0, 2 ** 63)) * 2 + int(rng.integers(0, 2))
+    offset = int(rng.choice([0, int(rng.integers(0, 2 ** 20)), 2 ** 32 - int(rng.integers(0, 5000)),
+                             2 ** 64 - int(rng.integers(1, 300000))]))
+    kind = str(rng.choice(["normal", "relu", "wide", "uniform"]))
+    return n, chunk, mode, seed, offset, kind
+
+
+@pytest.mark.parametrize("i", range(48))
+def test_parity_random_configurations(i):
+    """Property test over random (n, chunk, k, range rule, rounding, layout, seed, counter offset, value
+    distribution): stream and reconstruction bit-exact against the oracle, whatever path the sizes select
+    (register-resident chunks, the any-shape coder, chunks wider than 32768, a ragged tail)."""
+    n, chunk, (k, range_, round_, layout), seed, offset, kind = _random_case(i)
+    x = workloads.random_tensor(n, 7000 + i, kind)
+    if i % 7 == 3 and n > chunk:  # a constant chunk and an all-zero chunk somewhere inside
+        x[:chunk] = x[0]
+        x[-chunk:] = 0.0
+    check_roundtrip(x, chunk, k, range_, round_, layout, seed, offset)
+
+
 @pytest.mark.parametrize("name", ["cfg1_act", "cfg2_grad", "cfg5_64KB", "cfg5_1MB", "cfg5_16MB"])
 def test_workloads_full_parity_small(name):
     spec = workloads.TENSORS[name]
