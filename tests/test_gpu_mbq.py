@@ -129,6 +129,23 @@ def test_mbq_level_search_at_thresholds_and_extremes(alpha_prev):
     check_mbq(probe, k, 4, False, alpha_prev)
 
 
+@pytest.mark.parametrize("i", range(16))
+def test_mbq_parity_random_configurations(i):
+    """Seeded random (n, k, batch index, coefficients, value distribution), sizes around the 4096-element
+    tiles and the 296 groups of the encode pass."""
+    rng = np.random.default_rng([20231107, i])
+    n = int(rng.choice([int(rng.integers(1, 5000)), int(rng.integers(5000, 300000)), 4096 * 296 + int(rng.integers(-40, 9000)),
+                        4096 * int(rng.integers(1, 700))]))
+    k = int(rng.integers(2, 5))
+    t = int(rng.integers(1, 60))
+    kind = str(rng.choice(["normal", "relu", "uniform"]))
+    x = workloads.random_tensor(n, 9500 + i, kind) * np.float32(rng.choice([1.0, 1e-3, 37.0]))
+    alpha_prev = (np.abs(rng.standard_normal(k)) + 0.02).astype(np.float32) * np.float32(np.abs(x).mean() + 1e-6)
+    check_mbq(x, k, t, False, alpha_prev)
+    if i % 4 == 0:
+        check_mbq(x, k, 0, True, None)
+
+
 def test_mbq_singular_system_keeps_alpha():
     x = np.abs(workloads.random_tensor(5000, 3, "normal")) + 10
     alpha_prev = np.array([1.0, 0.5], dtype=np.float32)

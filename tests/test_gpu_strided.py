@@ -61,6 +61,24 @@ def test_strided_parity(mode, rows, stride, chunk):
     check(x, chunk, stride, k, range_, round_, layout, seed=21, rng_offset=5)
 
 
+@pytest.mark.parametrize("i", range(24))
+def test_strided_parity_random_configurations(i):
+    """Seeded random (batch rows, values per sample, chunk, mode, seed, counter offset): rows that do not fill
+    the last batch group, feature counts that do not fill the last block of 64 octets, chunks of any
+    multiple of 32 (boundaries anywhere inside rows), counters next to the 2^32 and 2^64 wraps."""
+    rng = np.random.default_rng([20231106, i])
+    rows = int(rng.choice([1, 2, 31, 32, 33, int(rng.integers(1, 200))]))
+    stride = 8 * int(rng.choice([1, 3, 63, 64, 65, int(rng.integers(1, 1200))]))
+    n = rows * stride
+    chunk = int(rng.choice([32, 96, 1024, 4096, 32 * int(rng.integers(1, 2000)), (n + 31) // 32 * 32]))
+    k, range_, round_, layout = modes()[int(rng.integers(0, len(modes())))]
+    seed = int(rng.integers(0, 2 ** 63)) * 2 + 1
+    offset = int(rng.choice([0, int(rng.integers(0, 2 ** 20)), 2 ** 32 - int(rng.integers(0, 5000)),
+                             2 ** 64 - int(rng.integers(1, 300000))]))
+    x = workloads.random_tensor(n, 9000 + i, str(rng.choice(["normal", "relu", "wide"])))
+    check(x, chunk, stride, k, range_, round_, layout, seed=seed, rng_offset=offset)
+
+
 def test_strided_largest_latent_output_of_the_paper():
     """Batch 128, 8192 values per sample (the 4096 KB output of Sec. 4.3.1), per-tensor range, both encoders."""
     x = workloads.generate("cfg2_grad").reshape(32, -1)
