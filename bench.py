@@ -131,16 +131,10 @@ class Codec:
         self.ws = A.new_workspace(self.p)
         self.calls = 0
 
-    def step(self, i: int, events=None):
+    def step(self, i: int):
         A, j = self.A, i % self.copies
-        if events is not None:
-            events[0].record()
         A.accept_compress(self.p, self.x[j], self.stream[j], self.ws)
-        if events is not None:
-            events[1].record()
         A.accept_decompress(self.p, self.stream[j], self.xhat[j], self.ws)
-        if events is not None:
-            events[2].record()
         self.calls += 2
 
     def run(self, steps: int, warmup: int):
@@ -159,12 +153,21 @@ class Codec:
         e1.record()
         torch.cuda.synchronize()
         total = e0.elapsed_time(e1)
-        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+        # one event before the first kernel and one after every kernel: the end of a step is the start of the next
+        edge = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        mid = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        A = self.A
+        edge[0].record()
         for i in range(steps):
-            self.step(warmup + steps + i, ev[i])
+            j = (warmup + steps + i) % self.copies
+            A.accept_compress(self.p, self.x[j], self.stream[j], self.ws)
+            mid[i].record()
+            A.accept_decompress(self.p, self.stream[j], self.xhat[j], self.ws)
+            edge[i + 1].record()
+        self.calls += 2 * steps
         torch.cuda.synchronize()
-        tc = sum(e[0].elapsed_time(e[1]) for e in ev) / steps
-        td = sum(e[1].elapsed_time(e[2]) for e in ev) / steps
+        tc = sum(edge[i].elapsed_time(mid[i]) for i in range(steps)) / steps
+        td = sum(mid[i].elapsed_time(edge[i + 1]) for i in range(steps)) / steps
         return total / steps, tc, td
 
     def run_isolated(self, steps: int, warmup: int = 3):
