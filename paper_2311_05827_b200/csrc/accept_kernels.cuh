@@ -234,15 +234,13 @@ __global__ void __launch_bounds__(BLOCK_MAX, BLOCK_MAX == 256 ? (R <= 2 ? 6 : 4)
   if (ROUND == kStochastic) rt.init(rng, a.rng_offset + e0 + 8ull * gt, 8u * (R - 1) * tpc + 8u);
   uint32_t xlo[R], xhi[R];
   quantize_rounds<K, RANGE, ROUND, R>(v, sc, rng, rt, 8u * tpc, xlo, xhi);
+  // an idle group (whole warps) stores nothing; the bit-plane store shuffles inside a quad, never across warps
+  if (!active) return;
 #pragma unroll
   for (int r = 0; r < R; ++r) {
     const uint64_t oct = e0 / 8 + (r * tpc + gt);  // global octet index
-    if (LAYOUT == kInterleaved) {
-      if (active) store_interleaved<K>(a.payload, oct, xlo[r], xhi[r]);
-    } else {
-      // shuffles inside: every lane takes part; an idle group rewrites nothing
-      if (active) store_bitplane<K>(a.payload, oct >> 2, xlo[r], xhi[r], lane);
-    }
+    if (LAYOUT == kInterleaved) store_interleaved<K>(a.payload, oct, xlo[r], xhi[r]);
+    else store_bitplane<K>(a.payload, oct >> 2, xlo[r], xhi[r], lane);
   }
 }
 
