@@ -252,7 +252,8 @@ __device__ __forceinline__ uint32_t quantize_stochastic_word_not(float x, const 
   const float t = fminf(__fmul_rn(d, sc.inv), kTop);
   const float t24 = __fmul_rn(t, 16777216.0f);  // exact scaling
   const uint32_t tc = (RANGE == kAbsMax) ? (uint32_t)__float2int_ru(t24) : __float2uint_ru(t24);
-  return (tc + ((uint32_t)ZP << 24)) + (g_not >> 8);
+  // (ZP : g_not) >> 8 = (g_not >> 8) + (ZP << 24): the zero point rides in on the funnel shift
+  return tc + __funnelshift_r(g_not, (uint32_t)ZP, 8);
 }
 
 // ~lane_word(h, m), from h_not = ~h and h_neg = -h
