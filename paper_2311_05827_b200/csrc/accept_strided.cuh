@@ -360,6 +360,24 @@ __global__ void __launch_bounds__(256) strided_decode_kernel(const CodecArgs a) 
   const uint64_t g = blockIdx.y;
   const uint64_t word0 = (g * F + (uint64_t)fo * 8) * K;
 
+  // Side words of the block's 32 row segments (512 values each), fetched once per block: with chunks of at
+  // least 512 values a segment touches at most two chunks, so 64 threads fetch {first chunk, next chunk} of
+  // a row each and everybody reads them from shared memory (instead of eight global loads per thread).
+  __shared__ float2 s_so[32][2];
+  __shared__ uint32_t s_first_chunk[32];
+  const bool staged = a.chunk >= 8u * kStridedOctetsPerBlock;
+  if (staged && tid < 64) {
+    const int r = tid >> 1, which = tid & 1;
+    const uint64_t row = g * 32 + r;
+    if (row < n_rows) {
+      const uint64_t first = row * F + (uint64_t)blockIdx.x * kStridedOctetsPerBlock * 8;
+      const uint64_t c0 = chunk_of(a, first);
+      const uint64_t c = c0 + which < a.n_chunks ? c0 + which : c0;
+      s_so[r][which] = __ldg(a.meta + c);
+      if (which == 0) s_first_chunk[r] = (uint32_t)c0;
+    }
+  }
+
   uint32_t ylo[8], yhi[8];
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
@@ -407,12 +425,14 @@ __global__ void __launch_bounds__(256) strided_decode_kernel(const CodecArgs a) 
 #pragma unroll
     for (int r = 0; r < 4; ++r) xhi[4 + r] = o[r];
   }
+  if (staged) __syncthreads();
 #pragma unroll
   for (int r = 0; r < 8; ++r) {
     const uint64_t row = g * 32 + sub * 8 + r;
     if (active && row < n_rows) {
       const uint64_t i0 = row * F + (uint64_t)fo * 8;
-      const float2 so = __ldg(a.meta + chunk_of(a, i0));
+      const uint64_t c = chunk_of(a, i0);
+      const float2 so = staged ? s_so[sub * 8 + r][(uint32_t)c - s_first_chunk[sub * 8 + r]] : __ldg(a.meta + c);
       float out[8];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
