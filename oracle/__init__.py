@@ -70,6 +70,8 @@ def _load():
     lib.oracle_mbq_payload_offset.argtypes = [u32]
     lib.oracle_mbq_stream_bytes.restype = u64
     lib.oracle_mbq_stream_bytes.argtypes = [u64, u32]
+    lib.oracle_reciprocal_toward_zero.restype = ctypes.c_float
+    lib.oracle_reciprocal_toward_zero.argtypes = [ctypes.c_float, ctypes.c_float]
     lib.oracle_mbq_levels.restype = None
     lib.oracle_mbq_levels.argtypes = [f32p, u32, f32p]
     lib.oracle_mbq_assign_nearest.restype = None
@@ -205,6 +207,11 @@ def mbq_payload_offset(k: int) -> int:
 
 def mbq_stream_bytes(n: int, k: int) -> int:
     return int(_load().oracle_mbq_stream_bytes(n, k))
+
+
+def reciprocal_toward_zero(L: float, r: float) -> float:
+    """The quantizer's reciprocal scale: L / r rounded toward zero in fp32."""
+    return float(_load().oracle_reciprocal_toward_zero(L, r))
 
 
 def mbq_levels(alpha) -> np.ndarray:

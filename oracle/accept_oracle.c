@@ -14,8 +14,9 @@
  * Readings of points the paper leaves open (each also listed in the design notes):
  *   - one range per chunk of C consecutive values of the vectorised tensor; C >= N is the paper's
  *     per-tensor range ("Backward Quantizer": c = max|g|);
- *   - "dividing by the scaling factor" is computed as a product with inv = L/c (one division per
- *     chunk); pinned against true division in the tests;
+ *   - "dividing by the scaling factor" is computed as a product with inv = L/c rounded toward zero
+ *     (one division per chunk; rounded down so that |x * inv| <= L as in exact arithmetic); pinned
+ *     against true division in the tests;
  *   - nearest rounding is IEEE round-half-to-even;
  *   - the uniform generator of Eq. 7 is counter based (MurmurHash3's 32-bit finaliser, see oracle_rng_hash below: one hash per four counters); U has 24 bits; pr = t - floor(t) and the test
  *     U < pr are exact;
@@ -92,6 +93,17 @@ double oracle_rng_uniform(uint64_t seed, uint64_t ctr) {
  * meta[0] = s (scaling factor), meta[1] = o (offset).  i0 is the index of x[0] in the whole
  * tensor (the random-number counter).  Returns 1 if the chunk was non-finite.
  */
+/* L / r rounded TOWARD ZERO (inf if the quotient overflows).  "Dividing by the scaling factor" s = r / L
+ * is computed as a product with this reciprocal; in the paper's exact arithmetic |g / s| never exceeds L, and
+ * rounding the reciprocal down keeps that true in fp32: r * inv <= L, hence fl(d * inv) <= L for every
+ * d <= r, so no value has to be clamped back into the code range.  The round-to-nearest quotient is above
+ * the true one exactly when its (exact, in double) product with r is above L. */
+float oracle_reciprocal_toward_zero(float L, float r) {
+  float q = L / r;
+  if (isfinite(q) && (double)q * (double)r > (double)L) q = nextafterf(q, 0.0f);
+  return q;
+}
+
 static int quantize_chunk(const float* x, uint32_t valid, uint32_t k, int range, int round_mode,
                           uint64_t seed, uint64_t rng_offset, uint64_t i0, uint8_t* u,
                           float* meta) {
@@ -109,7 +121,7 @@ static int quantize_chunk(const float* x, uint32_t valid, uint32_t k, int range,
       if (fabsf(x[i]) > c) c = fabsf(x[i]);
     float L = (float)((1 << (k - 1)) - 1);
     s = c / L;
-    inv = L / c;
+    inv = oracle_reciprocal_toward_zero(L, c);
     base = 0.0f;
     o = 0.0f;
     zero_point = 1 << (k - 1);
@@ -126,7 +138,7 @@ static int quantize_chunk(const float* x, uint32_t valid, uint32_t k, int range,
     float r = hi - lo;
     if (!nonfinite && !isfinite(r)) nonfinite = 1; /* range overflow */
     s = r / L;
-    inv = L / r;
+    inv = oracle_reciprocal_toward_zero(L, r);
     base = lo;
     o = lo + 0.0f; /* -0 becomes +0 */
     zero_point = 0;

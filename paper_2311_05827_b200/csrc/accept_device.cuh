@@ -112,6 +112,15 @@ __device__ __forceinline__ bool is_finite_bits(float a) {
   return (__float_as_uint(a) & 0x7f800000u) != 0x7f800000u;
 }
 
+// L / r rounded toward zero, from the round-to-nearest quotient: that one is above the true quotient
+// exactly when q * r - L (one fused operation: the sign is exact) is positive, and the float below a
+// positive q is the one with the next lower bit pattern.  q = inf (overflow) is returned as it is.
+__device__ __forceinline__ float reciprocal_toward_zero(float L, float r) {
+  const float q = __fdiv_rn(L, r);
+  const bool above = is_finite_bits(q) && __fmaf_rn(q, r, -L) > 0.0f;
+  return __uint_as_float(__float_as_uint(q) - (above ? 1u : 0u));
+}
+
 template <int K, int RANGE>
 __device__ __forceinline__ Scale make_scale(float hi, float lo) {
   Scale sc;
@@ -119,7 +128,7 @@ __device__ __forceinline__ Scale make_scale(float hi, float lo) {
     const float L = (float)((1 << (K - 1)) - 1);
     sc.nonfinite = !is_finite_bits(hi);
     sc.s = __fdiv_rn(hi, L);
-    sc.inv = __fdiv_rn(L, hi);
+    sc.inv = reciprocal_toward_zero(L, hi);  // hi * inv <= L, so |x * inv| <= L and nothing needs a clamp
     sc.base = 0.0f;
     sc.o = 0.0f;
     if (sc.nonfinite || !(hi > 0.0f) || !is_finite_bits(sc.inv)) { sc.s = 0.0f; sc.inv = 0.0f; }
@@ -128,7 +137,7 @@ __device__ __forceinline__ Scale make_scale(float hi, float lo) {
     const float r = __fsub_rn(hi, lo);
     sc.nonfinite = !is_finite_bits(hi) || !is_finite_bits(lo) || !is_finite_bits(r);
     sc.s = __fdiv_rn(r, L);
-    sc.inv = __fdiv_rn(L, r);
+    sc.inv = reciprocal_toward_zero(L, r);
     sc.base = lo;
     sc.o = (lo == 0.0f) ? 0.0f : lo;  // -0 is written as +0
     if (sc.nonfinite) { sc.s = 0.0f; sc.inv = 0.0f; sc.base = 0.0f; sc.o = 0.0f; }
@@ -204,7 +213,7 @@ __device__ __forceinline__ uint32_t quantize_nearest_word(float x, const Scale& 
   constexpr float kMagicZ = kMagic + (float)ZP;  // exact; even, so ties still go to even codes
   const float d = (RANGE == kAbsMax) ? x : __fsub_rn(x, sc.base);
   const float t = __fmul_rn(d, sc.inv);
-  // |t| <= L(1+2^-22): the rounded code cannot leave [zp-L, zp+L], no clamp needed
+  // |t| <= L (the reciprocal is rounded toward zero): the rounded code cannot leave [zp-L, zp+L], no clamp needed
   return __float_as_uint(__fadd_rn(t, kMagicZ));
 }
 
@@ -212,14 +221,13 @@ __device__ __forceinline__ uint32_t quantize_nearest_word(float x, const Scale& 
 //   U < t - n   <=>   r < ceil((t - n) * 2^24)          (r is an integer)
 // so  n + [U < t - n] = floor((ceil(t * 2^24) + (2^24 - 1 - r)) / 2^24), and 2^24 - 1 - r = (~h) >> 8.
 // Adding zero_point << 24 makes the sum non-negative; byte 3 of the 32-bit sum is the stored code u.
-// t is clamped to the top level first (a quotient that rounded just above L must not reach L + 1),
-// which also keeps the sum below 2^32; the low side cannot pass the lowest code.
+// |t| never exceeds the top level L (the reciprocal is rounded toward zero, see make_scale), so the
+// sum stays below 2^32 and the code cannot reach L + 1; the low side cannot pass the lowest code.
 template <int K, int RANGE>
 __device__ __forceinline__ uint32_t quantize_stochastic_word(float x, const Scale& sc, uint32_t h) {
   constexpr int ZP = (RANGE == kAbsMax) ? (1 << (K - 1)) : 0;
-  constexpr float kTop = (RANGE == kAbsMax) ? (float)((1 << (K - 1)) - 1) : (float)((1 << K) - 1);
   const float d = (RANGE == kAbsMax) ? x : __fsub_rn(x, sc.base);
-  const float t = fminf(__fmul_rn(d, sc.inv), kTop);
+  const float t = __fmul_rn(d, sc.inv);  // |t| <= L: inv is rounded toward zero
   const float t24 = __fmul_rn(t, 16777216.0f);  // exact scaling
   const uint32_t tc = (RANGE == kAbsMax) ? (uint32_t)__float2int_ru(t24) : __float2uint_ru(t24);
   return tc + ((uint32_t)ZP << 24) + ((~h) >> 8);
@@ -247,9 +255,8 @@ __device__ __forceinline__ uint32_t pack_bytes(uint32_t b0, uint32_t b1, uint32_
 template <int K, int RANGE>
 __device__ __forceinline__ uint32_t quantize_stochastic_word_not(float x, const Scale& sc, uint32_t g_not) {
   constexpr int ZP = (RANGE == kAbsMax) ? (1 << (K - 1)) : 0;
-  constexpr float kTop = (RANGE == kAbsMax) ? (float)((1 << (K - 1)) - 1) : (float)((1 << K) - 1);
   const float d = (RANGE == kAbsMax) ? x : __fsub_rn(x, sc.base);
-  const float t = fminf(__fmul_rn(d, sc.inv), kTop);
+  const float t = __fmul_rn(d, sc.inv);  // |t| <= L: inv is rounded toward zero
   const float t24 = __fmul_rn(t, 16777216.0f);  // exact scaling
   const uint32_t tc = (RANGE == kAbsMax) ? (uint32_t)__float2int_ru(t24) : __float2uint_ru(t24);
   // (ZP : g_not) >> 8 = (g_not >> 8) + (ZP << 24): the zero point rides in on the funnel shift

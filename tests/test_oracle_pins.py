@@ -166,6 +166,35 @@ def test_minmax_codes_by_hand():
     assert [float(v) for v in xhat[:6]] == [2.0, -1.0, 0.0, 0.0, 1.0, 1.0]
 
 
+def test_reciprocal_scale_is_the_quotient_rounded_toward_zero():
+    """inv = L / r rounded toward zero, against exact rational arithmetic: inv <= L/r < next float above inv,
+    hence r * inv <= L and no product x * inv with |x| <= r can leave the code range (checked in exact
+    arithmetic too, and in fp32 on the extreme element)."""
+    from fractions import Fraction
+    rng = np.random.default_rng(11)
+    ranges = np.concatenate([np.exp2(rng.uniform(-100, 100, 3000)), rng.uniform(0.5, 2.0, 3000), [1.0, 3.0, 7.0, 127.0, 255.0]])
+    for L in (1.0, 3.0, 7.0, 15.0, 127.0, 255.0):
+        for r in ranges.astype(np.float32):
+            inv = np.float32(oracle.reciprocal_toward_zero(L, float(r)))
+            exact = Fraction(L) / Fraction(float(r))
+            assert Fraction(float(inv)) <= exact < Fraction(float(np.nextafter(inv, np.float32(np.inf))))
+            assert Fraction(float(r)) * Fraction(float(inv)) <= Fraction(L)
+            assert np.float32(r) * inv <= np.float32(L)  # the fp32 product of the extreme element
+
+
+def test_extreme_element_takes_the_top_code_under_every_draw_of_eq7():
+    """With |x * inv| <= L the largest element sits exactly on or just below the top level: stochastic rounding
+    gives it L or L - 1, never L + 1 (which a clamp would have to repair), and -L or -L + 1 on the low side."""
+    for k in (2, 4, 8):
+        L = 2 ** (k - 1) - 1
+        zp = 2 ** (k - 1)
+        for c in (0.1, 1.0 / 3.0, 0.7, 3.0, 1e-3, 12345.678):
+            x = np.array([c, -c, c / 2, 0.0] * 8, dtype=np.float32)
+            for seed in range(200):
+                codes = oracle.quantize(x, x.size, k, RANGE_ABSMAX, ROUND_STOCHASTIC, seed, 0)[0].astype(int) - zp
+                assert set(codes[0::4]) <= {L, L - 1} and set(codes[1::4]) <= {-L, -L + 1}
+
+
 @pytest.mark.parametrize("k", [2, 4, 8])
 def test_per_tensor_range_matches_true_division(k):
     """One chunk >= N is the paper's per-tensor quantizer: codes = round(g / s), s = max|g|/L.
