@@ -13,15 +13,16 @@
  *   range   ABSMAX (Sec. 3.3 "Backward Quantizer"):  c = max|x|,  L = 2^(k-1)-1,  s = c/L,  o = 0
  *           MINMAX (affine extension):               lo = min x, hi = max x, L = 2^k-1,
  *                                                    s = (hi-lo)/L,  o = lo
- *   scale   inv = L/c  (resp. L/(hi-lo)); one IEEE fp32 division per chunk.  If the range is 0,
- *           or inv overflows, the chunk is degenerate: s = 0, inv = 0, every code is the zero point.
+ *   scale   inv = L/c  (resp. L/(hi-lo)) rounded toward zero, one IEEE fp32 division per chunk, so that
+ *           |x*inv| <= L as in exact arithmetic and no code is clamped.  If the range is 0, or the
+ *           quotient overflows, the chunk is degenerate: s = 0, inv = 0, every code is the zero point.
  *   codes   t = x*inv           (MINMAX: t = (x-lo)*inv), each fp32 operation rounded separately
  *           NEAREST:    q = rint(t)                      (ties to even)
  *           STOCHASTIC: q = floor(t) + [U < t-floor(t)]  (Eq. 7), U from the counter-based
  *                       generator described at accept_params.seed; the fraction t-floor(t) and
  *                       the comparison are exact (no rounding of the difference)
- *           ABSMAX: q clamped to [-2^(k-1), 2^(k-1)-1], stored code u = q + 2^(k-1)  ("+8" of the
- *           "Backward Encoder" for k = 4);  MINMAX: u = q clamped to [0, 2^k-1]
+ *           ABSMAX: q lies in [-L, L] (inside the paper's [-2^(k-1), 2^(k-1)-1]), stored code
+ *           u = q + 2^(k-1)  ("+8" of the "Backward Encoder" for k = 4);  MINMAX: u = q in [0, 2^k-1]
  *   pack    INTERLEAVED ("Backward Encoder"): code of element t of the chunk occupies bits
  *           [k*t, k*t+k) of the chunk's little-endian bit string (k = 8: plain bytes).
  *           BITPLANE ("Forward Encoder"): per group of 32 consecutive elements, k consecutive
