@@ -316,6 +316,24 @@ def _modes_of(spec):
     return [(m.k, m.range, m.round, m.layout) for m in spec.headline + spec.also]
 
 
+@pytest.mark.parametrize("mode", modes(), ids=MODE_IDS)
+def test_parity_extreme_ranges(mode):
+    """Chunks whose range sits at the ends of fp32: the reciprocal scale is subnormal (range near 3e38 with
+    k = 2), overflows (range below ~4e-37: a degenerate chunk) or is about to; values from full scale down
+    to subnormals inside each chunk."""
+    k, range_, round_, layout = mode
+    chunk = 1024
+    rng = np.random.default_rng(99)
+    parts = []
+    for top in (3.0e38, 1.2e38, 2.0e-36, 5.0e-37, 1.0e-38, 1.0e-42, 1.0):
+        v = (rng.uniform(-1, 1, chunk) * top).astype(np.float32)
+        v[:8] = np.array([top, -top, top / 2, top * 2.0 ** -30, 1e-45, -1e-45, 0.0, top * 0.999999], dtype=np.float32)
+        parts.append(v)
+    x = np.concatenate(parts).astype(np.float32)
+    assert np.all(np.isfinite(x))
+    check_roundtrip(x, chunk, k, range_, round_, layout, seed=17, rng_offset=3)
+
+
 def _random_case(i):
     """Seeded draw of (n, chunk, mode, seed, counter offset, value kind) for the property test."""
     rng = np.random.default_rng([20231105, i])
