@@ -217,16 +217,20 @@ accept_status accept_decompress_host(const accept_params* p, const void* h_strea
  *   init != 0 (batch 0 of an epoch): residue method: r = x; for j = 0..k-1: b_j = [r >= 0],
  *     alpha_j = mean |r|, r <- r - alpha_j b_j; alpha_prev is not read; no Eq. 3/4 update.
  *   The stream carries alpha_next and m_q = mean(B alpha_next - x) (Eq. 5); the receiver
- *     computes xhat = level(c) - m_q.  Sums run in double in a fixed order (results repeat from
- *     run to run; against another summation order alpha_next and m_q may differ in the last fp32
- *     bit).  Non-finite input is not supported: ACCEPT_DEV_NONFINITE is set, codes are unspecified.
+ *     computes xhat = level(c) - m_q.  The sums over the tensor behind Eq. 3 and Eq. 5 (B^T x, the sum
+ *     of x, and the mean |r| of the residue method) are taken WITHOUT rounding and rounded once to double:
+ *     alpha_next and m_q are a function of the input alone, whatever the order in which threads add (the
+ *     k x k system is then solved in double by Gaussian elimination with partial pivoting; a pivot below
+ *     1e-9 N counts as singular).  Non-finite input is not supported: ACCEPT_DEV_NONFINITE is set, such
+ *     values are left out of the sums and the codes are unspecified.
  * Stream: [0,32) header (magic, version, n low, n high, 0, k, 0, 1), [32, 32+4k) alpha_next,
  *   then m_q, zero pad to a multiple of 16, then bit planes: group g of 32 elements owns words
  *   g*k .. g*k+k-1, bit t of word g*k+j = [b_(32g+t),j = +1] ("-1 replaced by 0").
  * k in {2,3,4} (the paper's forward range); d_alpha_prev / d_alpha_next are DEVICE arrays of k
  * floats (they may be the same array), so successive batches chain without a host round trip.
- * The workspace (accept_mbq_workspace_size bytes, 16-byte aligned, zeroed once by the caller) holds
- * the status word and per-block partial sums (at most 47 KB).  Launches: 2 (plus 2k when init).  The encode
+ * The workspace (accept_mbq_workspace_size bytes = 624, 16-byte aligned, zeroed once by the caller) holds
+ * the status word, the residue coefficients and the exact sums (every call leaves them zeroed again; a
+ * workspace serves one call at a time).  Launches: 2 (plus k when init).  The encode
  * kernel of a batch >= 1 asks for 128 KB of dynamic shared memory per block (its search table).
  */
 typedef struct {

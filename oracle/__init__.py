@@ -49,6 +49,8 @@ def _load():
     lib.oracle_stream_bytes.argtypes = [u64, u32, u32]
     lib.oracle_rng_hash.restype = u32
     lib.oracle_rng_hash.argtypes = [u64, u64]
+    lib.oracle_rng_fill.restype = None
+    lib.oracle_rng_fill.argtypes = [u64, u64, u64, vp]
     lib.oracle_rng_uniform.restype = ctypes.c_double
     lib.oracle_rng_uniform.argtypes = [u64, u64]
     lib.oracle_quantize.restype = i32
@@ -72,6 +74,12 @@ def _load():
     lib.oracle_mbq_stream_bytes.argtypes = [u64, u32]
     lib.oracle_reciprocal_toward_zero.restype = ctypes.c_float
     lib.oracle_reciprocal_toward_zero.argtypes = [ctypes.c_float, ctypes.c_float]
+    lib.oracle_exact_sum.restype = ctypes.c_double
+    lib.oracle_exact_sum.argtypes = [vp, u64]
+    lib.oracle_exact_abs_sum.restype = ctypes.c_double
+    lib.oracle_exact_abs_sum.argtypes = [vp, u64]
+    lib.oracle_exact_signed_sum.restype = ctypes.c_double
+    lib.oracle_exact_signed_sum.argtypes = [vp, vp, u64, u32]
     lib.oracle_mbq_levels.restype = None
     lib.oracle_mbq_levels.argtypes = [f32p, u32, f32p]
     lib.oracle_mbq_assign_nearest.restype = None
@@ -125,6 +133,13 @@ def stream_bytes(n: int, chunk: int, k: int) -> int:
 
 def rng_hash(seed: int, ctr: int) -> int:
     return int(_load().oracle_rng_hash(seed & (2**64 - 1), ctr & (2**64 - 1)))
+
+
+def rng_words(seed: int, ctr0: int, n: int) -> np.ndarray:
+    """The 32-bit words of counters ctr0 .. ctr0+n-1 (rng_hash in bulk)."""
+    out = np.empty(n, dtype=np.uint32)
+    _load().oracle_rng_fill(seed & (2**64 - 1), ctr0 & (2**64 - 1), n, _ptr(out))
+    return out
 
 
 def rng_uniform(seed: int, ctr: int) -> float:
@@ -212,6 +227,24 @@ def mbq_stream_bytes(n: int, k: int) -> int:
 def reciprocal_toward_zero(L: float, r: float) -> float:
     """The quantizer's reciprocal scale: L / r rounded toward zero in fp32."""
     return float(_load().oracle_reciprocal_toward_zero(L, r))
+
+
+def exact_sum(x) -> float:
+    """Sum of the fp32 values of x without rounding, rounded once to double (ties to even)."""
+    x = _f32(x)
+    return float(_load().oracle_exact_sum(_ptr(x), x.size))
+
+
+def exact_abs_sum(x) -> float:
+    x = _f32(x)
+    return float(_load().oracle_exact_abs_sum(_ptr(x), x.size))
+
+
+def exact_signed_sum(x, codes, p: int) -> float:
+    """(B^T x)_p: +x where bit p of the code is set, -x elsewhere; exact, rounded once to double."""
+    x = _f32(x)
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    return float(_load().oracle_exact_signed_sum(_ptr(x), _ptr(codes), x.size, p))
 
 
 def mbq_levels(alpha) -> np.ndarray:

@@ -81,6 +81,11 @@ uint32_t oracle_rng_hash(uint64_t seed, uint64_t ctr) {
   return h * lane_mul[ctr & 3];
 }
 
+/* out[i] = oracle_rng_hash(seed, ctr0 + i): the same words in bulk, for the statistical pins. */
+void oracle_rng_fill(uint64_t seed, uint64_t ctr0, uint64_t n, uint32_t* out) {
+  for (uint64_t i = 0; i < n; ++i) out[i] = oracle_rng_hash(seed, ctr0 + i);
+}
+
 /* U in [0,1) on a grid of 2^-24: the top 24 random bits. */
 double oracle_rng_uniform(uint64_t seed, uint64_t ctr) {
   return (double)(oracle_rng_hash(seed, ctr) >> 8) / 16777216.0;
@@ -351,12 +356,17 @@ int oracle_bitwidth_schedule(int is_backward, int n_lr_changes) {
  *     exactly, whatever the magnitudes of x and the levels; a tie goes to the lower level; codes
  *     whose levels coincide: the smallest code);
  *     then alpha_cur = (B^T B)^-1 B^T x (Eq. 3) and alpha^t = beta alpha^(t-1) + (1-beta) alpha_cur
- *     with beta = min(0.9, (1+t)/(10+t)) (Eq. 4), all in double, rounded once to fp32.  If B^T B is
- *     singular (a pivot below 1e-9 N) alpha_cur = alpha^(t-1).
+ *     with beta = min(0.9, (1+t)/(10+t)) (Eq. 4).  B^T B is made of integers; every entry of B^T x is the
+ *     exact sum rounded once to double (see "exact sums" below), so neither depends on the order of the
+ *     elements; the k x k system is solved in double by Gaussian elimination with partial pivoting and
+ *     alpha^t is rounded once to fp32.  If B^T B is singular (a pivot below 1e-9 N) alpha_cur = alpha^(t-1).
  *   - the stream carries alpha^t (the coefficients after the update) and m_q = E[B alpha^t - x]
  *     (Eq. 5), so that the receiver computes B alpha^t - m_q ("Forward Dequantizer").
  *   - batch 0 of an epoch: residue method: r = x; for j = 0..k-1: b_j = sign(r) (+1 for r >= 0),
- *     alpha_j = mean |r|, r <- r - alpha_j b_j (fp32 residues, double means); no Eq. 3/4 update.
+ *     alpha_j = mean |r|, r <- r - alpha_j b_j (fp32 residues; the mean is the exact sum rounded once to
+ *     double, divided by n, rounded to fp32); no Eq. 3/4 update.
+ *   - m_q (Eq. 5) = (sum_p alpha_p * (sum of the signs of basis p) - sum of x) / n in double, the sum of x
+ *     exact and rounded once.
  * ============================================================================================ */
 
 #define MBQ_MAGIC_KIND 1u /* header word 7 */
@@ -380,6 +390,111 @@ void oracle_mbq_levels(const float* alpha, uint32_t k, float* levels) {
     }
     levels[c] = v;
   }
+}
+
+/* ---- exact sums --------------------------------------------------------------------------------
+ * Eq. 3 (B^T x) and Eq. 5 (the mean of B alpha - x) are sums over the whole tensor.  They are taken
+ * here as the paper writes them, as sums of real numbers: every fp32 value is an integer multiple of
+ * 2^-149, so the sum is held as an integer count of that unit (positive and negative parts apart,
+ * 384 bits each: 277 bits for the largest fp32 value and room for 2^64 of them) and rounded ONCE, to
+ * the nearest double (ties to even).  The result does not depend on the order of the elements. */
+
+#define EXACT_LIMBS 6
+typedef struct { uint64_t pos[EXACT_LIMBS], neg[EXACT_LIMBS]; } exact_sum;
+
+static void exact_clear(exact_sum* a) { memset(a, 0, sizeof(*a)); }
+
+/* acc += v * 2^shift (v < 2^24) */
+static void limbs_add_shifted(uint64_t* acc, uint64_t v, unsigned shift) {
+  unsigned limb = shift / 64, off = shift % 64;
+  uint64_t lo = v << off, hi = off ? (v >> (64 - off)) : 0;
+  uint64_t parts[2] = {lo, hi};
+  unsigned carry = 0;
+  for (unsigned i = limb; i < EXACT_LIMBS; ++i) {
+    uint64_t add = (i - limb < 2) ? parts[i - limb] : 0;
+    uint64_t before = acc[i];
+    uint64_t sum = before + add;
+    unsigned c1 = sum < before;
+    uint64_t sum2 = sum + carry;
+    unsigned c2 = sum2 < sum;
+    acc[i] = sum2;
+    carry = c1 | c2;
+    if (i - limb >= 1 && !carry) break;
+  }
+}
+
+/* Adds x (or -x when negate != 0).  Non-finite values are skipped: their chunk or tensor is flagged elsewhere. */
+static void exact_add(exact_sum* a, float x, int negate) {
+  uint32_t bits;
+  memcpy(&bits, &x, 4);
+  uint32_t E = (bits >> 23) & 0xFFu, frac = bits & 0x7FFFFFu;
+  int negative = (int)(bits >> 31) ^ (negate ? 1 : 0);
+  if (E == 255u) return;
+  /* x = m * 2^(E-150) with the hidden bit in m (E >= 1), or m * 2^-149 (subnormal) */
+  uint64_t m = E ? (frac | 0x800000u) : frac;
+  unsigned shift = E ? E - 1 : 0;
+  if (m) limbs_add_shifted(negative ? a->neg : a->pos, m, shift);
+}
+
+static int limbs_compare(const uint64_t* p, const uint64_t* q) {
+  for (int i = EXACT_LIMBS - 1; i >= 0; --i)
+    if (p[i] != q[i]) return p[i] > q[i] ? 1 : -1;
+  return 0;
+}
+
+/* The accumulated sum rounded to the nearest double, ties to even. */
+static double exact_round(const exact_sum* a) {
+  int cmp = limbs_compare(a->pos, a->neg);
+  if (cmp == 0) return 0.0;
+  const uint64_t* big = cmp > 0 ? a->pos : a->neg;
+  const uint64_t* small = cmp > 0 ? a->neg : a->pos;
+  uint64_t d[EXACT_LIMBS];
+  unsigned borrow = 0;
+  for (int i = 0; i < EXACT_LIMBS; ++i) {
+    uint64_t t = big[i] - small[i];
+    unsigned b1 = big[i] < small[i];
+    uint64_t t2 = t - borrow;
+    unsigned b2 = t < borrow;
+    d[i] = t2;
+    borrow = b1 | b2;
+  }
+  int top = -1; /* index of the highest set bit */
+  for (int i = EXACT_LIMBS * 64 - 1; i >= 0; --i)
+    if ((d[i / 64] >> (i % 64)) & 1u) { top = i; break; }
+  uint64_t mant = 0;
+  int low = top > 52 ? top - 52 : 0; /* the mantissa is bits [low, top] */
+  for (int i = top; i >= low; --i) mant = (mant << 1) | ((d[i / 64] >> (i % 64)) & 1u);
+  if (low > 0) {
+    int guard = (int)((d[(low - 1) / 64] >> ((low - 1) % 64)) & 1u), sticky = 0;
+    for (int i = low - 2; i >= 0 && !sticky; --i) sticky = (int)((d[i / 64] >> (i % 64)) & 1u);
+    if (guard && (sticky || (mant & 1u))) ++mant; /* 2^53 is still exact in a double */
+  }
+  double r = ldexp((double)mant, low - 149);
+  return cmp > 0 ? r : -r;
+}
+
+/* Sum of x[0..n), exactly, rounded once to double. */
+double oracle_exact_sum(const float* x, uint64_t n) {
+  exact_sum a;
+  exact_clear(&a);
+  for (uint64_t i = 0; i < n; ++i) exact_add(&a, x[i], 0);
+  return exact_round(&a);
+}
+
+/* Sum of |x[0..n)|, exactly, rounded once to double. */
+double oracle_exact_abs_sum(const float* x, uint64_t n) {
+  exact_sum a;
+  exact_clear(&a);
+  for (uint64_t i = 0; i < n; ++i) exact_add(&a, fabsf(x[i]), 0);
+  return exact_round(&a);
+}
+
+/* (B^T x)_p = sum of +x over the elements whose basis p is +1 and of -x over the others, exactly, rounded once. */
+double oracle_exact_signed_sum(const float* x, const uint8_t* codes, uint64_t n, uint32_t p) {
+  exact_sum a;
+  exact_clear(&a);
+  for (uint64_t i = 0; i < n; ++i) exact_add(&a, x[i], !((codes[i] >> p) & 1u));
+  return exact_round(&a);
 }
 
 /* s + e = a + b exactly (Knuth's two-sum; no overflow for fp32-sized inputs). */
@@ -439,8 +554,7 @@ void oracle_mbq_assign_residue(const float* x, uint64_t n, uint32_t k, uint8_t* 
   memcpy(r, x, sizeof(float) * n);
   memset(codes, 0, n);
   for (uint32_t j = 0; j < k; ++j) {
-    double sum = 0.0;
-    for (uint64_t i = 0; i < n; ++i) sum += fabs((double)r[i]);
+    double sum = oracle_exact_abs_sum(r, n);
     alpha0[j] = (float)(sum / (double)n);
     for (uint64_t i = 0; i < n; ++i) {
       if (r[i] >= 0.0f) { codes[i] |= (uint8_t)(1u << j); r[i] = r[i] - alpha0[j]; }
@@ -454,18 +568,14 @@ void oracle_mbq_assign_residue(const float* x, uint64_t n, uint32_t k, uint8_t* 
 static int mbq_least_squares(const float* x, const uint8_t* codes, uint64_t n, uint32_t k, const float* alpha_prev,
                              double* alpha_cur) {
   double G[8][8], rhs[8];
-  for (uint32_t p = 0; p < k; ++p) {
-    rhs[p] = 0.0;
-    for (uint32_t q = 0; q < k; ++q) G[p][q] = 0.0;
-  }
-  for (uint64_t i = 0; i < n; ++i) {
-    double b[8];
-    for (uint32_t p = 0; p < k; ++p) b[p] = ((codes[i] >> p) & 1u) ? 1.0 : -1.0;
-    for (uint32_t p = 0; p < k; ++p) {
-      rhs[p] += b[p] * (double)x[i];
-      for (uint32_t q = 0; q < k; ++q) G[p][q] += b[p] * b[q];
+  /* B^T B: integers (sums of +-1), exact in double; B^T x: exact sums rounded once */
+  for (uint32_t p = 0; p < k; ++p)
+    for (uint32_t q = 0; q < k; ++q) {
+      int64_t g = 0;
+      for (uint64_t i = 0; i < n; ++i) g += (((codes[i] >> p) ^ (codes[i] >> q)) & 1u) ? -1 : 1;
+      G[p][q] = (double)g;
     }
-  }
+  for (uint32_t p = 0; p < k; ++p) rhs[p] = oracle_exact_signed_sum(x, codes, n, p);
   /* Gaussian elimination with partial pivoting */
   for (uint32_t c = 0; c < k; ++c) {
     uint32_t piv = c;
@@ -505,8 +615,7 @@ void oracle_mbq_update_alpha(const float* x, const uint8_t* codes, uint64_t n, u
 
 /* Eq. 5: mean of the quantization error of B alpha. */
 float oracle_mbq_bias(const float* x, const uint8_t* codes, uint64_t n, uint32_t k, const float* alpha) {
-  double sum_x = 0.0, acc = 0.0;
-  for (uint64_t i = 0; i < n; ++i) sum_x += (double)x[i];
+  double sum_x = oracle_exact_sum(x, n), acc = 0.0;
   for (uint32_t p = 0; p < k; ++p) {
     int64_t s = 0; /* sum of the signs of basis p */
     for (uint64_t i = 0; i < n; ++i) s += ((codes[i] >> p) & 1u) ? 1 : -1;

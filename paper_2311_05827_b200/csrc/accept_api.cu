@@ -312,13 +312,11 @@ accept::MbqArgs mbq_args(const accept_mbq_params* p, void* d_stream, void* d_ws)
   a.side = reinterpret_cast<float*>(base + ACCEPT_HEADER_BYTES);
   a.payload = reinterpret_cast<uint32_t*>(base + accept_mbq_payload_offset(p));
   a.status = reinterpret_cast<uint32_t*>(ws);
-  a.alpha_init = reinterpret_cast<float*>(ws + 16);
+  a.ws = reinterpret_cast<accept::MbqWorkspace*>(ws);
   a.n = p->n_elems;
   a.n_blocks = mbq_blocks(p);
   a.n_residue_blocks = mbq_residue_blocks(p);
   a.n_tiles = mbq_tiles(p);
-  a.partial = reinterpret_cast<accept::MbqPartial*>(ws + 64);
-  a.residue_sum = reinterpret_cast<double*>(ws + 64 + (size_t)accept::kMbqPartialBytes * a.n_blocks);
   a.k = p->k;
   a.batch_index = p->batch_index;
   a.init = p->init ? 1u : 0u;
@@ -329,10 +327,7 @@ template <int K>
 void launch_mbq_compress(const accept::MbqArgs& a, cudaStream_t s) {
   const dim3 grid((a.n_blocks + accept::kMbqGroups - 1) / accept::kMbqGroups);
   if (a.init) {
-    for (int j = 0; j < K; ++j) {
-      launch_overlapped(accept::mbq_residue_sum_kernel<K>, dim3(a.n_residue_blocks), 256, s, a, j);
-      launch_overlapped(accept::mbq_residue_finalize_kernel, dim3(1), 256, s, a, j);
-    }
+    for (int j = 0; j < K; ++j) launch_overlapped(accept::mbq_residue_sum_kernel<K>, dim3(a.n_residue_blocks), 256, s, a, j);
     launch_overlapped(accept::mbq_encode_kernel<K, true>, grid, accept::kMbqEncodeThreads, s, a);
   } else {
     // the search grid needs more dynamic shared memory than a kernel gets without opting in (the
@@ -342,7 +337,7 @@ void launch_mbq_compress(const accept::MbqArgs& a, cudaStream_t s) {
     launch_overlapped_shared(fn, grid, accept::kMbqEncodeThreads, accept::kMbqGridBytes, s, a);
   }
   launch_overlapped(accept::mbq_finalize_kernel<K>, dim3(1), accept::kMbqFinalizeThreads, s, a);
-  g_launches.fetch_add(2 + (a.init ? 2 * K : 0), std::memory_order_relaxed);
+  g_launches.fetch_add(2 + (a.init ? K : 0), std::memory_order_relaxed);
 }
 
 // ---- built-in scratch for accept_compress_static ------------------------------------------------
@@ -568,9 +563,8 @@ size_t accept_mbq_compressed_size(const accept_mbq_params* p) {
 
 size_t accept_mbq_workspace_size(const accept_mbq_params* p) {
   if (accept_mbq_check_params(p) != ACCEPT_OK) return 0;
-  // status + residue coefficients (64 bytes), one 128-byte record per group of the encode pass (at most 296) and one
-  // double per block of a residue pass (at most 1184)
-  return 64 + (size_t)accept::kMbqPartialBytes * mbq_blocks(p) + 8 * (size_t)mbq_residue_blocks(p);
+  // status word, residue coefficients, the exact sums (five of 12 digits) and the sign counts
+  return sizeof(accept::MbqWorkspace);
 }
 
 accept_status accept_mbq_compress(const accept_mbq_params* p, const float* d_x, const float* d_alpha_prev,

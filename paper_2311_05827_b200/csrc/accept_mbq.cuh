@@ -6,38 +6,43 @@
 // 32-element group is basis j.  level(c) = (+-alpha_0) + ... + (+-alpha_k-1), summed in fp32 in
 // the order j = 0..k-1.  One pass over the input assigns the signs (nearest level through a
 // uniform grid over the span of the levels, one shared-memory lookup and one comparison per
-// element), writes the planes and gathers per group of 256 threads what Eq. 3-5 need: counts of +1
-// per basis, counts of differing signs per pair of bases (integers: B^T B exactly), sum of x over
-// the +1 elements of each basis and sum of x (double).  A single small block then adds the
-// partials in a fixed order, solves the k x k system, applies the moving average and writes the
-// side words.  Sums are order-fixed, so results repeat from run to run.
+// element), writes the planes and gathers what Eq. 3-5 need: counts of +1 per basis, counts of
+// differing signs per pair of bases (integers: B^T B exactly), the sum of x over the +1 elements of
+// each basis and the sum of x.  The sums of x are EXACT (accept_exact.cuh): integers all the way into
+// the workspace, rounded once to double by the single small block that then solves the k x k system,
+// applies the moving average and writes the side words.  Nothing depends on the order in which
+// threads or blocks add, so the side words are a function of the input alone.
 #pragma once
+#include "accept_exact.cuh"
 #include "accept_kernels.cuh"
 
 namespace accept {
 
 constexpr int kMbqRounds = 2;                      // octets per thread and tile
-constexpr int kMbqTile = kMbqRounds * 256 * 8;     // elements per block
-constexpr int kMbqPartialBytes = 128;              // per-block record in the workspace
-constexpr int kMbqFinalizeThreads = 256;           // threads of the single finalize block
+constexpr int kMbqTile = kMbqRounds * 256 * 8;     // elements per tile
+constexpr int kMbqFinalizeThreads = 32;            // threads of the single finalize block
 constexpr int kMbqGroups = 2;                      // 256-thread groups per block of the encode pass (one block per SM);
                                                    // 3 groups at 80 registers were slower than 2 at 113 (measured)
 constexpr int kMbqEncodeThreads = 256 * kMbqGroups;
-constexpr int kMbqMaxBlocks = 148 * kMbqGroups;    // groups of the encode pass = records in the workspace; fixed, so sums
-                                                   // repeat on any device
-constexpr int kMbqResidueBlocks = 1184;            // blocks of a residue pass (fixed for the same reason)
+constexpr int kMbqMaxBlocks = 148 * kMbqGroups;    // groups of the encode pass
+constexpr int kMbqResidueBlocks = 1184;            // blocks of a residue pass
 constexpr int kMbqCells = 256;                     // cells of the uniform search grid
 constexpr int kMbqGridBytes = kMbqCells * 32 * 16; // one 16-byte entry per cell and lane
+constexpr int kMbqSums = 5;                        // wide sums in the workspace: basis 0..3, then the sum of x
+constexpr int kMbqFlushTiles = kFlushElems / (kMbqRounds * 8);  // tiles a thread codes between two flushes
 
-// Per-block partial sums (one 128-byte record per block of the encode pass).
-struct MbqPartial {
-  double plus[4];     // sum of x over the elements whose basis j is +1
-  double sum_x;       // sum of x
-  uint32_t count[4];  // number of +1 per basis
-  uint32_t differ[6]; // pairs (0,1) (0,2) (0,3) (1,2) (1,3) (2,3): elements whose two signs differ
-  uint32_t pad[12];
+// Workspace of the forward quantizer (zeroed once by the caller; every call leaves the sums zeroed again).
+struct MbqWorkspace {
+  uint32_t status;
+  uint32_t pad0[3];
+  float alpha_init[4];            // coefficients found by the residue passes (init)
+  uint32_t blocks_done;           // blocks of a residue pass that have delivered their sum
+  uint32_t pad1[7];
+  long long wide[kMbqSums][kAccLimbs];  // exact sums, see accept_exact.cuh
+  unsigned long long count[4];    // number of +1 per basis
+  unsigned long long differ[6];   // pairs (0,1) (0,2) (0,3) (1,2) (1,3) (2,3): elements whose two signs differ
 };
-static_assert(sizeof(MbqPartial) == kMbqPartialBytes, "record size");
+static_assert(sizeof(MbqWorkspace) == 64 + 8 * kMbqSums * kAccLimbs + 80, "workspace layout");
 
 struct MbqArgs {
   const float* x;
@@ -48,13 +53,11 @@ struct MbqArgs {
   float* side;              // stream + 32: alpha (k floats), m_q
   uint32_t* payload;
   uint32_t* status;
-  MbqPartial* partial;      // workspace + 64
-  float* alpha_init;        // workspace + 16: coefficients found by the residue passes (init)
-  double* residue_sum;      // workspace + 32: scratch of the residue passes
+  MbqWorkspace* ws;         // the workspace (its first word is the status word)
   uint64_t n;
   uint64_t n_tiles;         // tiles of kMbqTile elements
-  uint32_t n_blocks;        // 256-thread groups of the encode pass = records in the workspace
-  uint32_t n_residue_blocks;  // blocks of a residue pass = doubles in the workspace
+  uint32_t n_blocks;        // 256-thread groups of the encode pass that have tiles
+  uint32_t n_residue_blocks;  // blocks of a residue pass
   uint32_t k, batch_index, init;
 };
 
@@ -265,78 +268,190 @@ __device__ __forceinline__ void mbq_ld_octet(const float* x, uint64_t n, uint64_
   }
 }
 
-// acc += x when flag != 0, as one predicated add (no branch, no 64-bit select)
-__device__ __forceinline__ void add_if(double& acc, double x, uint32_t flag) {
-  asm("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p add.rn.f64 %0, %0, %1;\n\t}" : "+d"(acc) : "d"(x), "r"(flag));
+// ---- exact sums of a block ------------------------------------------------------------------------
+
+// What the threads of a block share for their exact sums: the block's wide sums (slot j = basis j,
+// slot kMbqSums - 1 = the sum of x, or the only sum of a residue pass) and the window of the fast path.
+struct MbqBlockSums {
+  long long wide[kMbqSums][kAccLimbs];
+  ExactWindow window;
+};
+
+__device__ __forceinline__ void mbq_block_sums_clear(MbqBlockSums* bs, int tid, int n_threads) {
+  for (int i = tid; i < kMbqSums * kAccLimbs; i += n_threads) (&bs->wide[0][0])[i] = 0;
 }
 
-__device__ __forceinline__ double warp_sum(double v) {
-#pragma unroll
-  for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
-  return v;
+// A value outside the window: straight into the block's wide sums of `slots` (bit s set: slot s).
+__device__ __noinline__ void mbq_wide_add_value(MbqBlockSums* bs, uint32_t* status, float x, uint32_t slots) {
+  for (int s = 0; s < kMbqSums; ++s)
+    if ((slots >> s) & 1u)
+      if (!wide_add_float(bs->wide[s], x, false)) atomicOr(status, kDevNonFinite);
 }
 
-// Residue method, step j: per-block sum of |r_j| (r_0 = x) with the coefficients found so far.
+// Thread s < kMbqSums hands slot s of the block's wide sums to the workspace: carries propagated first, so
+// that each piece is below 2^32 and the 64-bit words of the workspace cannot overflow whatever the grid.
+// Call after a __syncthreads() that follows the last addition.
+__device__ inline void mbq_block_sums_deliver(MbqBlockSums* bs, MbqWorkspace* ws, int tid) {
+  if (tid >= kMbqSums) return;
+  long long limbs[kAccLimbs];
+  bool any = false;
+  for (int i = 0; i < kAccLimbs; ++i) { limbs[i] = bs->wide[tid][i]; any = any || limbs[i] != 0; }
+  if (!any) return;
+  wide_normalise(limbs);
+  for (int i = 0; i < kAccLimbs; ++i)
+    if (limbs[i] != 0) limb_add(&ws->wide[tid][i], limbs[i]);
+}
+
+// ---- residue method ---------------------------------------------------------------------------------
+
+// Residue method, step j: alpha_j = mean |r_j| (r_0 = x) with the coefficients found so far.  Every block
+// adds the |r_j| of its tiles exactly and hands the sum to the workspace; the block that arrives last
+// rounds the total once, divides by n and leaves the workspace clean for the next pass.  No block waits
+// for another.
 template <int K>
 __global__ void __launch_bounds__(256) mbq_residue_sum_kernel(const MbqArgs a, int j) {
   grid_dependency_handshake();
-  __shared__ double s_part[8];
+  __shared__ MbqBlockSums s_sums;
+  __shared__ float s_amax[8];
+  __shared__ uint32_t s_is_last;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int SLOT = kMbqSums - 1;
   float alpha[K];
 #pragma unroll
-  for (int i = 0; i < K; ++i) alpha[i] = (i < j) ? a.alpha_init[i] : 0.0f;
+  for (int i = 0; i < K; ++i) alpha[i] = (i < j) ? a.ws->alpha_init[i] : 0.0f;
   const uint64_t n_oct = (a.n + 7) / 8;
-  double acc = 0.0;
-  for (uint64_t tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x)
-#pragma unroll
-  for (int r = 0; r < kMbqRounds; ++r) {
-    const uint64_t oct = tile * (kMbqRounds * 256) + r * 256 + tid;
+  mbq_block_sums_clear(&s_sums, tid, 256);
+
+  // Window of the fast path: around the coefficient of the first basis once it is known; for the first
+  // pass around the largest magnitude of the block's first octets.
+  float scale = alpha[0];
+  if (j == 0) {
+    const uint64_t oct = (uint64_t)blockIdx.x * (kMbqRounds * 256) + tid;
+    float m = 0.0f;
     if (oct < n_oct) {
       float v[8];
       mbq_ld_octet(a.x, a.n, oct, v);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        float res;
-        mbq_residue_code<K>(alpha, v[e], j, &res);
-        if (oct * 8 + e < a.n) acc += (double)fabsf(res);
+      for (int e = 0; e < 8; ++e) m = fmaxf(m, fabsf(v[e]));
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+    if (lane == 0) s_amax[warp] = m;
+    __syncthreads();
+    scale = 0.0f;
+    for (int w = 0; w < 8; ++w) scale = fmaxf(scale, s_amax[w]);
+    scale *= 0.125f;  // the top of the window is 2^9 above the binade of the scale
+  }
+  if (tid == 0) s_sums.window = make_window(scale);
+  __syncthreads();
+  const ExactWindow win = s_sums.window;
+
+  double acc = 0.0;
+  long long irun = 0;
+  int since = 0, flushes = 0;
+  for (uint64_t tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x) {
+#pragma unroll
+    for (int r = 0; r < kMbqRounds; ++r) {
+      const uint64_t oct = tile * (kMbqRounds * 256) + r * 256 + tid;
+      if (oct < n_oct) {
+        float v[8], res[8];
+        mbq_ld_octet(a.x, a.n, oct, v);
+        WindowCheck chk;
+        chk.init();
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          mbq_residue_code<K>(alpha, v[e], j, &res[e]);
+          res[e] = (oct * 8 + e < a.n) ? fabsf(res[e]) : 0.0f;
+        }
+#pragma unroll
+        for (int e = 0; e < 8; e += 2) chk.add2(res[e], res[e + 1]);
+        if (!chk.ok(win)) {
+#pragma unroll
+          for (int e = 0; e < 8; ++e)
+            if (!in_window(win, res[e])) {
+              mbq_wide_add_value(&s_sums, a.status, res[e], 1u << SLOT);
+              res[e] = 0.0f;
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc += (double)res[e];
+      }
+    }
+    if (++since == kMbqFlushTiles) {
+      since = 0;
+      irun += __double2ll_rn(acc * win.to_units);
+      acc = 0.0;
+      if (++flushes == kPushFlushes) {  // the same for every thread of the block: tiles are the block's
+        flushes = 0;
+        const long long total = warp_sum_int64(irun);
+        if (lane == 0) wide_add_int64(s_sums.wide[SLOT], total, win.pos);
+        irun = 0;
       }
     }
   }
-  acc = warp_sum(acc);
-  if (lane == 0) s_part[warp] = acc;
-  __syncthreads();
-  if (tid == 0) {
-    double s = 0.0;
-    for (int w = 0; w < 8; ++w) s += s_part[w];
-    a.residue_sum[blockIdx.x] = s;
+  irun += __double2ll_rn(acc * win.to_units);
+  {
+    const long long total = warp_sum_int64(irun);
+    if (lane == 0) wide_add_int64(s_sums.wide[SLOT], total, win.pos);
   }
-}
-
-// Residue method, step j: alpha_j = mean |r_j| (block partials added in index order).
-__global__ void __launch_bounds__(256) mbq_residue_finalize_kernel(const MbqArgs a, int j) {
-  grid_dependency_handshake();
-  __shared__ double s_part[256];
-  const int tid = threadIdx.x;
-  double s = 0.0;
-  for (uint32_t b = tid; b < a.n_residue_blocks; b += 256) s += a.residue_sum[b];
-  s_part[tid] = s;
   __syncthreads();
-  if (tid == 0) {
-    double total = 0.0;
-    for (int i = 0; i < 256; ++i) total += s_part[i];
-    a.alpha_init[j] = (float)(total / (double)a.n);
+  if (tid == SLOT) mbq_block_sums_deliver(&s_sums, a.ws, tid);
+  // the last block to get here finishes the pass
+  if (tid == SLOT) {
+    __threadfence();
+    const uint32_t ticket = atomicAdd(&a.ws->blocks_done, 1u);
+    s_is_last = (ticket == gridDim.x - 1) ? 1u : 0u;
+  }
+  __syncthreads();
+  if (s_is_last && tid == 0) {
+    __threadfence();
+    long long total[kAccLimbs];
+    for (int i = 0; i < kAccLimbs; ++i) {
+      total[i] = (long long)atomicExch(reinterpret_cast<unsigned long long*>(&a.ws->wide[SLOT][i]), 0ull);
+    }
+    a.ws->alpha_init[j] = (float)(wide_to_double(total) / (double)a.n);
+    a.ws->blocks_done = 0u;
   }
 }
 
 // How the signs of an element are found.
 constexpr int kMbqResidue = 0, kMbqSearch = 1, kMbqGrid = 2;
 
-// Running sums of one thread over all its tiles.
+// Running sums of one thread over all its tiles.  plus[] and sum_x hold what the thread added since its
+// last flush (plus[] times 2^-767, the flag factor); irun[] the flushed part in units of the window.
 template <int K>
 struct MbqSums {
   double plus[K], sum_x;
+  long long irun[K + 1];      // [K]: the sum of x
   uint32_t count, differ[3];  // of basis q = lane & 3, and of the pairs (q, q ^ d)
+  int since, flushes;
 };
+
+// Accumulators -> integer units of the window, exactly (see accept_exact.cuh).
+template <int K>
+__device__ __forceinline__ void mbq_flush(MbqSums<K>& s, const MbqBlockSums* bs) {
+  const double to_units = bs->window.to_units;
+  const double flag_to_units = to_units * 0x1p767;  // the flag factor was 2^-767
+#pragma unroll
+  for (int j = 0; j < K; ++j) {
+    s.irun[j] += __double2ll_rn(s.plus[j] * flag_to_units);
+    s.plus[j] = 0.0;
+  }
+  s.irun[K] += __double2ll_rn(s.sum_x * to_units);
+  s.sum_x = 0.0;
+}
+
+// Running int64 sums of a warp -> the block's wide sums.  All lanes of the warp call.
+template <int K>
+__device__ __forceinline__ void mbq_push(MbqSums<K>& s, MbqBlockSums* bs, int lane) {
+  const int pos = bs->window.pos;
+#pragma unroll
+  for (int j = 0; j <= K; ++j) {
+    const long long total = warp_sum_int64(s.irun[j]);
+    if (lane == 0) wide_add_int64(bs->wide[j < K ? j : kMbqSums - 1], total, pos);
+    s.irun[j] = 0;
+  }
+}
 
 // The octets of thread tid of a tile: FULL = every element of the tile exists.
 template <bool FULL>
@@ -356,13 +471,24 @@ __device__ __forceinline__ void mbq_load_tile(const MbqArgs& a, uint64_t tile, i
   }
 }
 
+// A value of the encode pass that may lie outside the window.  If it does, it goes into the block's wide
+// sums (the sum of x, and the sum of every basis whose sign is +1) and 0 is returned for the thread's own
+// accumulators; otherwise the value itself is returned.
+__device__ __noinline__ float mbq_divert_value(MbqBlockSums* bs, uint32_t* status, float x, uint32_t flags) {
+  if (in_window(bs->window, x)) return x;
+  // flag bytes (0x10 per basis) -> slot bits, plus the slot of the sum of x
+  const uint32_t slots = ((((flags >> 4) * 0x00204081u) >> 21) & 0xFu) | (1u << (kMbqSums - 1));
+  mbq_wide_add_value(bs, status, x, slots);
+  return 0.0f;
+}
+
 // One tile of kMbqTile elements, coded by one group of 256 threads (tid = index in the group): assign
 // the signs, write the planes, add to the thread's sums.
 template <int K, int MODE, bool FULL>
 __device__ __forceinline__ void mbq_encode_tile(const MbqArgs& a, uint64_t tile, int tid, int lane,
                                                 const float (&v)[kMbqRounds][8], const float (&alpha)[K],
                                                 const MbqTable<K>& table, const uint4* cells, float scale,
-                                                MbqSums<K>& sums) {
+                                                MbqBlockSums* bs, float win_top, uint32_t win_ylow, MbqSums<K>& sums) {
   const uint64_t n_oct_stored = ((a.n + 31) / 32) * 4;
   const uint64_t oct0 = tile * (kMbqRounds * 256) + tid;
   const int q = lane & 3;
@@ -391,9 +517,21 @@ __device__ __forceinline__ void mbq_encode_tile(const MbqArgs& a, uint64_t tile,
           if (e >= valid) f[e] = 0;
       }
     }
+    // the values as the running sums take them: all of them, unless some lie outside the window
+    float w[8];
+    WindowCheck chk;
+    chk.init();
+#pragma unroll
+    for (int e = 0; e < 8; ++e) w[e] = v[r][e];  // 0 past the end
+#pragma unroll
+    for (int e = 0; e < 8; e += 2) chk.add2(w[e], w[e + 1]);
+    if (!(chk.amax < win_top && chk.ymin >= win_ylow)) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) w[e] = mbq_divert_value(bs, a.status, w[e], f[e]);
+    }
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-      const double xd = (double)v[r][e];  // 0 past the end
+      const double xd = (double)w[e];
       sums.sum_x += xd;
       mbq_add_flagged<0>(sums.plus[0], xd, f[e]);
       mbq_add_flagged<1>(sums.plus[1], xd, f[e]);
@@ -402,26 +540,37 @@ __device__ __forceinline__ void mbq_encode_tile(const MbqArgs& a, uint64_t tile,
     }
     // after the quad transpose lane q holds the 32 signs of basis q of its group: counts of +1 and,
     // against the words of the other three lanes of the quad, counts of differing signs
-    const uint32_t w = quad_transpose(mbq_planes_of_flags(f), lane);
-    if ((FULL || oct < n_oct_stored) && q < K) a.payload[(oct >> 2) * K + q] = w;
-    sums.count += __popc(w);
+    const uint32_t word = quad_transpose(mbq_planes_of_flags(f), lane);
+    if ((FULL || oct < n_oct_stored) && q < K) a.payload[(oct >> 2) * K + q] = word;
+    sums.count += __popc(word);
 #pragma unroll
     for (int d = 1; d < 4; ++d) {
-      const uint32_t other = __shfl_xor_sync(0xffffffffu, w, d);
-      sums.differ[d - 1] += __popc(w ^ other);
+      const uint32_t other = __shfl_xor_sync(0xffffffffu, word, d);
+      sums.differ[d - 1] += __popc(word ^ other);
+    }
+  }
+  // every thread of the group has coded the same number of tiles: flushes and pushes are taken together
+  if (++sums.since == kMbqFlushTiles) {
+    sums.since = 0;
+    mbq_flush<K>(sums, bs);
+    if (++sums.flushes == kPushFlushes) {
+      sums.flushes = 0;
+      mbq_push<K>(sums, bs, lane);
     }
   }
 }
 
 // A group walks over tiles with a stride of the number of groups and keeps its sums in registers: the
-// group-level reduction and the record in the workspace are paid once per group, not once per tile.
+// group-level reduction is paid once per group, not once per tile.
 // The loads of a group's next tile are in flight while it codes the current one (two register
 // buffers, the loop unrolled by two so that both are addressed statically).
 template <int K, int MODE>
 __device__ __forceinline__ void mbq_encode_tiles(const MbqArgs& a, uint32_t group, int tid, int lane,
                                                  const float (&alpha)[K], const MbqTable<K>& table, const uint4* cells,
-                                                 float scale, MbqSums<K>& sums) {
+                                                 float scale, MbqBlockSums* bs, MbqSums<K>& sums) {
   if (group >= a.n_blocks) return;
+  const float win_top = bs->window.top;
+  const uint32_t win_ylow = bs->window.ylow;
   const uint64_t full_tiles = a.n / kMbqTile, stride = a.n_blocks;
   float v0[kMbqRounds][8], v1[kMbqRounds][8];
   uint64_t tile = group;
@@ -429,82 +578,83 @@ __device__ __forceinline__ void mbq_encode_tiles(const MbqArgs& a, uint32_t grou
   while (tile < full_tiles) {
     const uint64_t t1 = tile + stride;
     if (t1 < full_tiles) mbq_load_tile<true>(a, t1, tid, v1);
-    mbq_encode_tile<K, MODE, true>(a, tile, tid, lane, v0, alpha, table, cells, scale, sums);
+    mbq_encode_tile<K, MODE, true>(a, tile, tid, lane, v0, alpha, table, cells, scale, bs, win_top, win_ylow, sums);
     tile = t1;
     if (t1 >= full_tiles) break;
     const uint64_t t2 = t1 + stride;
     if (t2 < full_tiles) mbq_load_tile<true>(a, t2, tid, v0);
-    mbq_encode_tile<K, MODE, true>(a, t1, tid, lane, v1, alpha, table, cells, scale, sums);
+    mbq_encode_tile<K, MODE, true>(a, t1, tid, lane, v1, alpha, table, cells, scale, bs, win_top, win_ylow, sums);
     tile = t2;
   }
   // the ragged last tile of the tensor, if there is one, is the last tile of its group
   if (tile < a.n_tiles) {
     mbq_load_tile<false>(a, tile, tid, v0);
-    mbq_encode_tile<K, MODE, false>(a, tile, tid, lane, v0, alpha, table, cells, scale, sums);
+    mbq_encode_tile<K, MODE, false>(a, tile, tid, lane, v0, alpha, table, cells, scale, bs, win_top, win_ylow, sums);
   }
 }
 
 // Assign the signs, write the planes, gather the sums.  One block of kMbqGroups groups of 256 threads
-// per SM; a group does what a 256-thread block would (its own tiles, its own record in the
-// workspace), the groups of a block share the search tables.  Dynamic shared memory: the search
-// grid (kMbqGridBytes), not needed when INIT.
+// per SM; a group does what a 256-thread block would (its own tiles), the groups of a block share the
+// search tables and the block's wide sums.  Dynamic shared memory: the search grid (kMbqGridBytes), not
+// needed when INIT.
 template <int K, bool INIT>
 __global__ void __launch_bounds__(kMbqEncodeThreads, 1) mbq_encode_kernel(const MbqArgs a) {
   grid_dependency_handshake();
   extern __shared__ uint4 s_cells[];
   __shared__ MbqTable<K> s_table;
   __shared__ MbqGridInfo s_grid;
+  __shared__ MbqBlockSums s_sums;
   __shared__ float s_level[16];
-  __shared__ double s_dbl[kMbqGroups][8][K + 1];
-  __shared__ uint32_t s_cnt[kMbqGroups][10];
+  __shared__ uint32_t s_cnt[10];
   const int lane = threadIdx.x & 31;
   const int g = threadIdx.x >> 8;            // group in the block
   const int tid = threadIdx.x & 255;         // thread in the group
-  const int warp = tid >> 5;                 // warp in the group
   const uint32_t group = blockIdx.x * kMbqGroups + g;
   float alpha[K];
+  mbq_block_sums_clear(&s_sums, threadIdx.x, kMbqEncodeThreads);
+  if (threadIdx.x < 10) s_cnt[threadIdx.x] = 0;
   if (INIT) {
 #pragma unroll
-    for (int j = 0; j < K; ++j) alpha[j] = a.alpha_init[j];
+    for (int j = 0; j < K; ++j) alpha[j] = a.ws->alpha_init[j];
+    // window of the exact sums: around the mean magnitude of the data
+    if (threadIdx.x == 0) s_sums.window = make_window(alpha[0]);
   } else {
 #pragma unroll
     for (int j = 0; j < K; ++j) alpha[j] = 0.0f;
     mbq_build_table<K>(a.alpha_prev, &s_table, s_level, threadIdx.x);
     mbq_build_grid<K>(s_table, s_level, &s_grid, s_cells, threadIdx.x, kMbqEncodeThreads);
+    // window of the exact sums: around the largest level (values the levels were fitted to)
+    if (threadIdx.x == 0) {
+      float amax = 0.0f;
+      for (int c = 0; c < (1 << K); ++c) amax = fmaxf(amax, fabsf(s_level[c]));
+      s_sums.window = make_window(amax * 0.125f);
+    }
   }
-  if (tid < 10) s_cnt[g][tid] = 0;
   __syncthreads();
 
   MbqSums<K> sums;
   sums.sum_x = 0.0;
   sums.count = 0;
+  sums.since = 0;
+  sums.flushes = 0;
 #pragma unroll
   for (int j = 0; j < K; ++j) sums.plus[j] = 0.0;
 #pragma unroll
+  for (int j = 0; j <= K; ++j) sums.irun[j] = 0;
+#pragma unroll
   for (int d = 0; d < 3; ++d) sums.differ[d] = 0;
 
-  if (INIT) mbq_encode_tiles<K, kMbqResidue>(a, group, tid, lane, alpha, s_table, s_cells, 0.0f, sums);
-  else if (s_grid.usable) mbq_encode_tiles<K, kMbqGrid>(a, group, tid, lane, alpha, s_table, s_cells, s_grid.scale, sums);
-  else mbq_encode_tiles<K, kMbqSearch>(a, group, tid, lane, alpha, s_table, s_cells, 0.0f, sums);
+  if (INIT) mbq_encode_tiles<K, kMbqResidue>(a, group, tid, lane, alpha, s_table, s_cells, 0.0f, &s_sums, sums);
+  else if (s_grid.usable) mbq_encode_tiles<K, kMbqGrid>(a, group, tid, lane, alpha, s_table, s_cells, s_grid.scale, &s_sums, sums);
+  else mbq_encode_tiles<K, kMbqSearch>(a, group, tid, lane, alpha, s_table, s_cells, 0.0f, &s_sums, sums);
+
+  // what is left in the accumulators, then the warp's total into the block's wide sums
+  mbq_flush<K>(sums, &s_sums);
+  mbq_push<K>(sums, &s_sums, lane);
 
   const int q = lane & 3;
-  double (&plus)[K] = sums.plus;
-#pragma unroll
-  for (int j = 0; j < K; ++j) plus[j] *= 0x1p767;  // the flag factor was 2^-767: exact
-  const double sum_x = sums.sum_x;
   uint32_t my_count = sums.count;
   uint32_t (&my_differ)[3] = sums.differ;
-
-  // group sums in a fixed order: lanes by butterfly, warps one after the other
-#pragma unroll
-  for (int j = 0; j < K; ++j) {
-    const double s = warp_sum(plus[j]);
-    if (lane == 0) s_dbl[g][warp][j] = s;
-  }
-  {
-    const double s = warp_sum(sum_x);
-    if (lane == 0) s_dbl[g][warp][K] = s;
-  }
   // lanes with the same q hold partial counts of the same basis / pairs: add over the eight quads
 #pragma unroll
   for (int d = 4; d <= 16; d <<= 1) {
@@ -513,92 +663,60 @@ __global__ void __launch_bounds__(kMbqEncodeThreads, 1) mbq_encode_kernel(const 
     for (int i = 0; i < 3; ++i) my_differ[i] += __shfl_xor_sync(0xffffffffu, my_differ[i], d);
   }
   if (lane < 4) {
-    atomicAdd(&s_cnt[g][q], my_count);
+    atomicAdd(&s_cnt[q], my_count);
 #pragma unroll
     for (int d = 1; d < 4; ++d) {
       const int other = q ^ d;
       if (q < other) {  // each pair once; pair index in the order (0,1) (0,2) (0,3) (1,2) (1,3) (2,3)
         const int pair = (q == 0) ? other - 1 : (q == 1 ? other + 1 : 5);
-        atomicAdd(&s_cnt[g][4 + pair], my_differ[d - 1]);
+        atomicAdd(&s_cnt[4 + pair], my_differ[d - 1]);
       }
     }
   }
   __syncthreads();
-  if (tid == 0 && group < a.n_blocks) {
-    MbqPartial out;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) { out.plus[j] = 0.0; out.count[j] = 0; }
-    for (int j = 0; j < K; ++j) {
-      double s = 0.0;
-      for (int w = 0; w < 8; ++w) s += s_dbl[g][w][j];
-      out.plus[j] = s;
-      out.count[j] = s_cnt[g][j];
-    }
-    double s = 0.0;
-    for (int w = 0; w < 8; ++w) s += s_dbl[g][w][K];
-    out.sum_x = s;
-    for (int p = 0; p < 6; ++p) out.differ[p] = s_cnt[g][4 + p];
-    for (int p = 0; p < 12; ++p) out.pad[p] = 0;
-    a.partial[group] = out;
+  mbq_block_sums_deliver(&s_sums, a.ws, threadIdx.x);
+  if (threadIdx.x >= 32 && threadIdx.x < 42) {
+    const int i = threadIdx.x - 32;
+    const unsigned long long c = s_cnt[i];
+    if (c) atomicAdd(i < 4 ? &a.ws->count[i] : &a.ws->differ[i - 4], c);
   }
 }
 
-// Adds the per-block partials (fixed order), then Eq. 3 (least squares by Gaussian elimination with
-// partial pivoting, in double), Eq. 4 (moving average), Eq. 5 (bias), and writes header, side
-// words and alpha_next.  One block.
+// Rounds the exact sums once, then Eq. 3 (least squares by Gaussian elimination with partial pivoting, in
+// double), Eq. 4 (moving average), Eq. 5 (bias), and writes header, side words and alpha_next; leaves the
+// sums of the workspace zeroed for the next call.  One warp.
 template <int K>
 __global__ void __launch_bounds__(kMbqFinalizeThreads) mbq_finalize_kernel(const MbqArgs a) {
   grid_dependency_handshake();
-  __shared__ double s_dbl[kMbqFinalizeThreads / 32][K + 1];
-  __shared__ unsigned long long s_int[kMbqFinalizeThreads / 32][10];
+  __shared__ double s_val[K + 1];  // [j] = (B^T x)_j, [K] = sum of x
   const int tid = threadIdx.x;
-  double d[K + 1];
+  MbqWorkspace* ws = a.ws;
+  if (tid <= K) {
+    long long lazy[kAccLimbs];
+    for (int i = 0; i < kAccLimbs; ++i) {
+      const long long sx = ws->wide[kMbqSums - 1][i];
+      // sum over the +1 elements minus sum over the -1 elements = 2 * (sum over +1) - (sum of all), digit by digit
+      lazy[i] = (tid < K) ? 2 * ws->wide[tid][i] - sx : sx;
+    }
+    s_val[tid] = wide_to_double(lazy);
+  }
   unsigned long long c[10];
 #pragma unroll
-  for (int j = 0; j <= K; ++j) d[j] = 0.0;
+  for (int j = 0; j < 4; ++j) c[j] = ws->count[j];
 #pragma unroll
-  for (int j = 0; j < 10; ++j) c[j] = 0;
-  // thread t adds records t, t + T, t + 2T, ... in that order
-#pragma unroll 4
-  for (uint32_t b = tid; b < a.n_blocks; b += kMbqFinalizeThreads) {
-    const MbqPartial& p = a.partial[b];
-#pragma unroll
-    for (int j = 0; j < K; ++j) { d[j] += p.plus[j]; c[j] += p.count[j]; }
-    d[K] += p.sum_x;
-#pragma unroll
-    for (int j = 0; j < 6; ++j) c[4 + j] += p.differ[j];
-  }
-  // fixed-order tree: butterfly over the lanes of each warp, then the warps one after the other
-#pragma unroll
-  for (int j = 0; j <= K; ++j) d[j] = warp_sum(d[j]);
-#pragma unroll
-  for (int j = 0; j < 10; ++j) {
-#pragma unroll
-    for (int sh = 16; sh >= 1; sh >>= 1) c[j] += __shfl_xor_sync(0xffffffffu, c[j], sh);
-  }
-  if ((tid & 31) == 0) {
-#pragma unroll
-    for (int j = 0; j <= K; ++j) s_dbl[tid >> 5][j] = d[j];
-#pragma unroll
-    for (int j = 0; j < 10; ++j) s_int[tid >> 5][j] = c[j];
-  }
+  for (int j = 0; j < 6; ++j) c[4 + j] = ws->differ[j];
   __syncthreads();
+  // the next call starts from zero
+  for (int i = tid; i < kMbqSums * kAccLimbs; i += kMbqFinalizeThreads) (&ws->wide[0][0])[i] = 0;
+  if (tid < 4) ws->count[tid] = 0;
+  if (tid < 6) ws->differ[tid] = 0;
   if (tid != 0) return;
-#pragma unroll
-  for (int j = 0; j <= K; ++j) d[j] = 0.0;
-#pragma unroll
-  for (int j = 0; j < 10; ++j) c[j] = 0;
-  for (int i = 0; i < kMbqFinalizeThreads / 32; ++i) {
-#pragma unroll
-    for (int j = 0; j <= K; ++j) d[j] += s_dbl[i][j];
-#pragma unroll
-    for (int j = 0; j < 10; ++j) c[j] += s_int[i][j];
-  }
-  const double N = (double)a.n, sum_x = d[K];
+
+  const double N = (double)a.n, sum_x = s_val[K];
   float alpha_next[K];
   if (a.init) {
 #pragma unroll
-    for (int j = 0; j < K; ++j) alpha_next[j] = a.alpha_init[j];
+    for (int j = 0; j < K; ++j) alpha_next[j] = ws->alpha_init[j];
   } else {
     double G[K][K], rhs[K], cur[K], prev[K];
     int pair = 0;
@@ -607,7 +725,7 @@ __global__ void __launch_bounds__(kMbqFinalizeThreads) mbq_finalize_kernel(const
         if (j < K) G[i][j] = G[j][i] = N - 2.0 * (double)c[4 + pair];
     for (int j = 0; j < K; ++j) {
       G[j][j] = N;
-      rhs[j] = 2.0 * d[j] - sum_x;  // sum over +1 minus sum over -1
+      rhs[j] = s_val[j];
       prev[j] = (double)__ldg(a.alpha_prev + j);
     }
     bool singular = false;
@@ -647,7 +765,6 @@ __global__ void __launch_bounds__(kMbqFinalizeThreads) mbq_finalize_kernel(const
   a.side[K] = m_q;
   // pad up to the payload
   for (uint32_t* w = reinterpret_cast<uint32_t*>(a.side + K + 1); w < a.payload; ++w) *w = 0u;
-  if (!is_finite_bits((float)sum_x)) atomicOr(a.status, kDevNonFinite);
 }
 
 // Receiver: planes -> codes -> level(c) - m_q.

@@ -77,7 +77,7 @@ def test_mbq_size_queries_match_oracle(A):
         assert A.accept_mbq_check_params(p) == 0
         assert A.accept_mbq_compressed_size(p) == oracle.mbq_stream_bytes(n, k)
         assert A.accept_mbq_payload_offset(p) == oracle.mbq_payload_offset(k)
-        assert A.accept_mbq_workspace_size(p) == 64 + 128 * min(296, -(-n // 4096)) + 8 * min(1184, -(-n // 4096))
+        assert A.accept_mbq_workspace_size(p) == 64 + 8 * 5 * 12 + 80  # status and coefficients, five exact sums of 12 digits, ten counts
     assert A.accept_mbq_compressed_size(A.MbqParams(10, 7)) == 0
 
 

@@ -157,6 +157,81 @@ def test_residue_initialisation():
     assert np.array_equal(codes & 1, (x >= 0).astype(np.uint8))
 
 
+def test_residue_initialisation_worked_by_hand_k2():
+    """Eight values, two bases, every number worked by hand (all of them exact in binary):
+         x   =  3     -1     0.5   -2.5    1    -0.5    2    -3.5      sum |x| = 14   -> alpha_0 = 1.75
+         b_0 =  +      -      +     -      +     -      +     -
+         r_1 =  1.25   0.75  -1.25 -0.75  -0.75  1.25   0.25 -1.75     sum |r_1| = 8  -> alpha_1 = 1
+         b_1 =  +      +      -     -      -     +      +     -
+       code = [b_0 = +] + 2 [b_1 = +]."""
+    x = np.array([3, -1, 0.5, -2.5, 1, -0.5, 2, -3.5], dtype=np.float32)
+    codes, alpha = oracle.mbq_assign_residue(x, 2)
+    assert alpha.tolist() == [1.75, 1.0]
+    assert codes.tolist() == [3, 2, 1, 0, 1, 2, 3, 0]
+    # the levels of these coefficients and the reconstruction B alpha of every element, again by hand
+    assert oracle.mbq_levels(alpha).tolist() == [-2.75, 0.75, -0.75, 2.75]
+    stream, nxt = oracle.mbq_compress(x, 2, 0, True)
+    assert nxt.tolist() == [1.75, 1.0]
+    # B alpha = 2.75 -0.75 0.75 -2.75 0.75 -0.75 2.75 -2.75; mean(B alpha - x) = (-0.25+0.25+0.25-0.25-0.25-0.25+0.75+0.75)/8
+    m_q = float(stream[32 + 8:32 + 12].view(np.float32)[0])
+    assert m_q == 1.0 / 8
+    assert oracle.mbq_decompress(stream, 8).tolist() == [2.625, -0.875, 0.625, -2.875, 0.625, -0.875, 2.625, -2.875]
+
+
+def _fraction_sum(values):
+    from fractions import Fraction
+    return float(sum((Fraction(float(v)) for v in values), Fraction(0)))  # Fraction -> float rounds to nearest, ties to even
+
+
+def test_exact_sums_against_rational_arithmetic():
+    """The sums behind Eq. 3 and Eq. 5 are exact and rounded once: against Python's rational arithmetic and
+    math.fsum on magnitudes spread over the whole fp32 range, on sums that cancel, on subnormals, and on exact
+    ties between two doubles (which go to the even one)."""
+    import math
+    rng = np.random.default_rng(2024)
+    cases = [
+        rng.standard_normal(3000).astype(np.float32),
+        (rng.standard_normal(3000) * 10.0 ** rng.uniform(-44, 38, 3000)).astype(np.float32),
+        np.float32([2.0 ** 53, 1.0]),                 # 2^53 + 1: tie, the even neighbour is 2^53
+        np.float32([2.0 ** 53, 2.0, 1.0]),            # 2^53 + 3: tie, the even neighbour is 2^53 + 4
+        np.float32([2.0 ** 53, 1.0, 2.0 ** -149]),    # just above the tie: rounds up
+        np.float32([2.0 ** 100, -(2.0 ** 100), 2.0 ** -149, 2.0 ** -149]),
+        np.float32([3.0e38] * 500 + [-3.0e38] * 499 + [1e-45] * 7),
+        (rng.integers(-(1 << 22), 1 << 22, 999).astype(np.float64) * 2.0 ** -149).astype(np.float32),
+    ]
+    v = rng.standard_normal(2000).astype(np.float32)
+    cases.append(np.concatenate([v, -v[::-1], np.float32([1e-30])]))
+    for x in cases:
+        x = x[np.isfinite(x)]
+        want = _fraction_sum(x)
+        assert oracle.exact_sum(x) == want == math.fsum(float(t) for t in x)
+        assert oracle.exact_abs_sum(x) == _fraction_sum(np.abs(x))
+        codes = rng.integers(0, 4, x.size).astype(np.uint8)
+        for p in (0, 1):
+            signed = np.where((codes >> p) & 1, x, -x)
+            assert oracle.exact_signed_sum(x, codes, p) == _fraction_sum(signed)
+    assert oracle.exact_sum(np.float32([2.0 ** 53, 1.0])) == 2.0 ** 53
+    assert oracle.exact_sum(np.float32([2.0 ** 53, 2.0, 1.0])) == 2.0 ** 53 + 4
+    # an order-independent result: any permutation gives the same bits
+    x = cases[1]
+    assert oracle.exact_sum(x) == oracle.exact_sum(x[::-1]) == oracle.exact_sum(np.sort(x))
+
+
+def test_alpha_update_does_not_depend_on_the_order_of_the_elements():
+    """Eq. 3-5 are sums over the tensor: permuting the elements (and their codes with them) leaves alpha^t and m_q
+    unchanged bit for bit, also where a plain left-to-right float sum would not."""
+    rng = np.random.default_rng(8)
+    x = (rng.standard_normal(20000) * 10.0 ** rng.uniform(-6, 6, 20000)).astype(np.float32)
+    alpha_prev = np.array([40.0, 9.0, 1.5], dtype=np.float32)
+    codes = oracle.mbq_assign_nearest(x, alpha_prev)
+    a0 = oracle.mbq_update_alpha(x, codes, alpha_prev, 4)
+    m0 = oracle.mbq_bias(x, codes, a0)
+    for seed in (1, 2, 3):
+        perm = np.random.default_rng(seed).permutation(x.size)
+        assert np.array_equal(oracle.mbq_update_alpha(x[perm], codes[perm], alpha_prev, 4).view(np.uint32), a0.view(np.uint32))
+        assert oracle.mbq_bias(x[perm], codes[perm], a0) == m0
+
+
 @pytest.mark.parametrize("k", [2, 3, 4])
 def test_stream_layout_and_size(k):
     """Side words: alpha (k floats) and m_q, the 32(k+1) bits of Eq. 8; payload k bits per element as planes."""

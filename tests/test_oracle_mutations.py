@@ -28,6 +28,9 @@ MUTATIONS = [
      "float term = ((c >> j) & 1u) ? -alpha[j] : alpha[j];"),
     ("MBQ: moving average weights swapped", "(float)(beta * (double)alpha_prev[p] + (1.0 - beta) * cur[p]);",
      "(float)((1.0 - beta) * (double)alpha_prev[p] + beta * cur[p]);"),
+    ("weak lane multiplier in the generator of Eq. 7", "{1u, 0x9E3779B1u, 0x85EBCA77u, 0xC2B2AE3Du}", "{1u, 0x00010001u, 0x85EBCA77u, 0xC2B2AE3Du}"),
+    ("exact sum drops the part below 2^-149 * 2^64", "uint64_t lo = v << off, hi = off ? (v >> (64 - off)) : 0;", "uint64_t lo = v << off, hi = 0;"),
+    ("exact sum rounds half up instead of to even", "if (guard && (sticky || (mant & 1u))) ++mant;", "if (guard) ++mant;"),
     ("MBQ: bias with the wrong sign", "return (float)((acc - sum_x) / (double)n);", "return (float)((sum_x - acc) / (double)n);"),
 ]
 
@@ -36,9 +39,11 @@ PIN_FUNCS = [getattr(pins, n) for n in dir(pins) if n.startswith("test_")] + \
 
 
 def _run_all_pins():
-    """Number of pin functions that fail (parametrized ones are run over their parameter sets)."""
+    """1 as soon as a pin function fails (parametrized ones are run over their parameter sets), else 0."""
     failed = 0
     for fn in PIN_FUNCS:
+        if failed:
+            return failed
         marks = [m for m in getattr(fn, "pytestmark", []) if m.name == "parametrize"]
         cases = [{}]
         for m in marks:
