@@ -69,13 +69,14 @@ typedef enum {
   ACCEPT_ERR_NONFINITE = 8,     /* reported through the device status word only */
   ACCEPT_ERR_BAD_SIZE = 9,      /* n_elems = 0 */
   ACCEPT_ERR_MISALIGNED = 10,   /* a device pointer is not 16-byte aligned */
-  ACCEPT_ERR_SCRATCH_LIMIT = 11 /* accept_compress_static: the call needs more scratch than the built-in array holds */
+  ACCEPT_ERR_SCRATCH_LIMIT = 11, /* accept_compress_static: the call needs more scratch than the built-in array holds */
+  ACCEPT_ERR_UNCHECKED_BUILD = 12 /* accept_bounds_check_report: this library was built without access checks */
 } accept_status;
 
 /* Bits of the device status word (word 0 of the workspace); sticky until the caller clears it. */
 #define ACCEPT_DEV_NONFINITE 1u   /* some chunk held NaN/Inf (or an overflowing MINMAX range) */
 #define ACCEPT_DEV_BAD_HEADER 2u  /* accept_decompress: stream header differs from the parameters */
-#define ACCEPT_DEV_COPY_TIMEOUT 4u /* an asynchronous copy inside a kernel did not complete within a second; output invalid */
+#define ACCEPT_DEV_COPY_TIMEOUT 4u /* an asynchronous copy inside a kernel did not complete within 0.2 s; output invalid */
 
 typedef enum { ACCEPT_RANGE_ABSMAX = 0, ACCEPT_RANGE_MINMAX = 1 } accept_range;
 typedef enum { ACCEPT_ROUND_NEAREST = 0, ACCEPT_ROUND_STOCHASTIC = 1 } accept_round;
@@ -87,9 +88,9 @@ typedef enum { ACCEPT_LAYOUT_INTERLEAVED = 0, ACCEPT_LAYOUT_BITPLANE = 1 } accep
  *   chunk_elems  C, multiple of 32, >= 32: elements sharing one range.
  *   k            bit width: 2, 3 (BITPLANE only), 4 or 8.
  *   group_stride 0, or F = values per sample (w*h*c): the tensor is (n_elems/F) x F and a pack group is
- *                made of the 32 BATCH neighbours (rows 32g..32g+31) of one feature f, as the paper's
- *                encoders do (Sec. 3.3: "concatenates the quantized data along the batch size
- *                dimension"): group index G = g*F + f, words G*k .. G*k+k-1 of the payload, element
+ *                made of the 32 BATCH neighbours (rows 32g..32g+31) of one feature f: pack groups run
+ *                along the batch dimension as in Sec. 3.3, "Forward Encoder" / "Backward Encoder".
+ *                Group index G = g*F + f, words G*k .. G*k+k-1 of the payload, element
  *                (row b, feature f) at position t = b % 32 of its group; rows past the last are zero
  *                bits; payload = 4*k*ceil(rows/32)*F bytes.  Ranges stay per chunk of consecutive
  *                values.  Needs F % 8 == 0, n_elems % F == 0, 32-byte aligned tensors, and not
@@ -135,6 +136,8 @@ size_t accept_payload_offset(const accept_params* p);
  * (such chunks do not fit on chip: their ranges are gathered in the workspace first, and the input
  * is read twice).  Word 0 is the device status word; the caller zeroes the workspace once (and
  * whenever it wants to clear the status); the workspace must be 16-byte aligned.  0 if p is invalid.
+ * This is what accept_compress needs.  accept_decompress touches the status word only: 16 bytes
+ * (4-byte aligned) are enough for it, whatever the parameters.
  */
 size_t accept_workspace_size(const accept_params* p);
 
@@ -155,7 +158,8 @@ accept_status accept_compress(const accept_params* p, const float* d_x, void* d_
  * in one kernel launch.  p carries what the receiver agreed on with the sender (n_elems,
  * chunk_elems, k, range, layout; round/seed are ignored); the kernel compares it with the header
  * words and or-s ACCEPT_DEV_BAD_HEADER into the status word on a mismatch (the output is then
- * unspecified but every access stays inside the buffers as sized by p).
+ * unspecified but every access stays inside the buffers as sized by p).  The workspace needs 16 bytes
+ * only (the status word), also for wide chunks and batch groups.
  */
 accept_status accept_decompress(const accept_params* p, const void* d_stream, size_t stream_bytes,
                                 float* d_xhat, void* d_ws, size_t ws_bytes, void* cuda_stream);
@@ -182,7 +186,11 @@ accept_status accept_decompress(const accept_params* p, const void* d_stream, si
  *     that first call before any stream capture begins on that device;
  *   - all calls on a device share the one array.  The status word in it is cleared at the start of every
  *     call (so it does not accumulate across calls as a caller-owned workspace does), and two calls that
- *     overlap on the GPU (different streams) race on it: issue them on one stream, or order them.
+ *     overlap on the GPU (different streams) race on it: issue them on one stream, or order them.  Calls
+ *     from several host threads must be serialised by the caller even on one stream: a call enqueues a
+ *     clear, its kernels and the status copy one after the other, and two threads could interleave them;
+ *   - d_x must live on the current device (checked: ACCEPT_ERR_CUDA otherwise), and cuda_stream must
+ *     belong to it.
  */
 #define ACCEPT_STATIC_SCRATCH_BYTES 256u
 accept_status accept_compress_static(const accept_params* p, const float* d_x, void* d_stream,
@@ -273,6 +281,19 @@ int accept_bitwidth_schedule(int is_backward, int n_lr_changes);
 
 /* Number of kernels the library has launched in this process (all entry points). */
 uint64_t accept_launch_count(void);
+
+/*
+ * For the checking build of this library (the same sources compiled with -DACCEPT_BOUNDS_CHECK, which the
+ * tests load in place of a memory checker): every access of a kernel to caller memory is compared with
+ * the byte ranges of the call (input, stream up to accept_compressed_size, workspace up to its size
+ * query, output), and one that falls outside -- or a write into the input -- is skipped and counted
+ * instead of performed.  This call synchronises cuda_stream, returns the number of skipped accesses since
+ * the previous report in *violations and, optionally, the address of the first one and its size (low 32
+ * bits) and kind (bit 32: write), then clears the count.  The paper has no counterpart.  In the normal
+ * build nothing is checked: *violations = 0 and the result is ACCEPT_ERR_UNCHECKED_BUILD.
+ */
+accept_status accept_bounds_check_report(void* cuda_stream, uint32_t* violations, uint64_t* first_address,
+                                         uint64_t* first_size_and_kind);
 
 #ifdef __cplusplus
 }

@@ -25,14 +25,14 @@ STATUS_NAMES = {
     0: "ACCEPT_OK", 1: "ACCEPT_ERR_NULL", 2: "ACCEPT_ERR_BAD_K", 3: "ACCEPT_ERR_BAD_CHUNK",
     4: "ACCEPT_ERR_BAD_ENUM", 5: "ACCEPT_ERR_TOO_SMALL", 6: "ACCEPT_ERR_BAD_STREAM_HEADER",
     7: "ACCEPT_ERR_CUDA", 8: "ACCEPT_ERR_NONFINITE", 9: "ACCEPT_ERR_BAD_SIZE", 10: "ACCEPT_ERR_MISALIGNED",
-    11: "ACCEPT_ERR_SCRATCH_LIMIT",
+    11: "ACCEPT_ERR_SCRATCH_LIMIT", 12: "ACCEPT_ERR_UNCHECKED_BUILD",
 }
 
 EXPORTS = [
     "accept_check_params", "accept_compressed_size", "accept_payload_offset", "accept_workspace_size",
     "accept_compress", "accept_decompress", "accept_compress_host", "accept_decompress_host",
     "accept_last_device_status", "accept_parse_header", "accept_bitwidth_schedule", "accept_launch_count",
-    "accept_compress_static",
+    "accept_compress_static", "accept_bounds_check_report",
     "accept_mbq_check_params", "accept_mbq_compressed_size", "accept_mbq_payload_offset", "accept_mbq_workspace_size",
     "accept_mbq_compress", "accept_mbq_decompress",
 ]
@@ -98,7 +98,14 @@ def lib() -> ctypes.CDLL:
         return _lib
     if not os.path.exists(LIB_PATH):
         raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2311_05827_b200.build`")
-    L = ctypes.CDLL(LIB_PATH)
+    _lib = load(LIB_PATH)
+    return _lib
+
+
+def load(path: str) -> ctypes.CDLL:
+    """Loads a build of the library (the product, or one of the tests-only variants of build.py) and
+    declares the argument types of its entry points."""
+    L = ctypes.CDLL(path)
     P, vp, sz, u64 = ctypes.POINTER(CParams), ctypes.c_void_p, ctypes.c_size_t, ctypes.c_uint64
     L.accept_check_params.restype = ctypes.c_int
     L.accept_check_params.argtypes = [P]
@@ -133,7 +140,8 @@ def lib() -> ctypes.CDLL:
     L.accept_mbq_decompress.argtypes = [MP, vp, sz, vp, vp, sz, vp]
     L.accept_launch_count.restype = u64
     L.accept_launch_count.argtypes = []
-    _lib = L
+    L.accept_bounds_check_report.restype = ctypes.c_int
+    L.accept_bounds_check_report.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), ctypes.POINTER(u64), ctypes.POINTER(u64)]
     return L
 
 
@@ -220,6 +228,13 @@ def accept_decompress_host(p: Params, h_stream, h_xhat, d_stream, d_xhat, d_ws, 
                                         d_stream.data_ptr(), d_xhat.data_ptr(), d_ws.data_ptr(),
                                         d_ws.numel() * d_ws.element_size(), _stream_handle(stream)),
            "accept_decompress_host")
+
+
+def accept_bounds_check_report(stream=None):
+    """-> (return code, skipped accesses, address of the first, its size, whether it was a write)."""
+    count, addr, info = ctypes.c_uint32(0), ctypes.c_uint64(0), ctypes.c_uint64(0)
+    code = lib().accept_bounds_check_report(_stream_handle(stream), ctypes.byref(count), ctypes.byref(addr), ctypes.byref(info))
+    return int(code), int(count.value), int(addr.value), int(info.value & 0xFFFFFFFF), bool(info.value >> 32)
 
 
 def accept_last_device_status(d_ws, stream=None) -> int:

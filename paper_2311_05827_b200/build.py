@@ -1,4 +1,12 @@
-"""Builds the CUDA library in-tree with nvcc for sm_100a (``libaccept.so`` beside this file)."""
+"""Builds the CUDA library in-tree with nvcc for sm_100a (``libaccept.so`` beside this file).
+
+Besides the product there are two tests-only variants of the same sources (never loaded by the binding
+unless a test asks for them):
+  bounds  -DACCEPT_BOUNDS_CHECK: every access of a kernel to caller memory is checked against the byte
+          ranges of the call, counted and skipped when outside (``libaccept_bounds.so``);
+  stall   -DACCEPT_TEST_COPY_STALL: the staged batch-group encoder announces bytes that never arrive, so
+          its bounded waits run out after 2 ms (``libaccept_stall.so``).
+"""
 from __future__ import annotations
 
 import os
@@ -17,23 +25,58 @@ NVCC_FLAGS = [
     "-shared", "-Xcompiler", "-fPIC",
 ]
 
+VARIANTS = {
+    "bounds": (os.path.join(HERE, "libaccept_bounds.so"), ["-DACCEPT_BOUNDS_CHECK"]),
+    "stall": (os.path.join(HERE, "libaccept_stall.so"), ["-DACCEPT_TEST_COPY_STALL"]),
+}
+
+
+def _stale(lib: str) -> bool:
+    if not os.path.exists(lib):
+        return True
+    t = os.path.getmtime(lib)
+    return any(os.path.getmtime(s) > t for s in DEPENDS)
+
 
 def needs_build() -> bool:
-    if not os.path.exists(LIB):
-        return True
-    t = os.path.getmtime(LIB)
-    return any(os.path.getmtime(s) > t for s in DEPENDS)
+    return _stale(LIB)
+
+
+def _command(lib: str, defines, verbose: bool):
+    nvcc = os.environ.get("NVCC", "nvcc")
+    return [nvcc] + NVCC_FLAGS + list(defines) + (["-Xptxas", "-v"] if verbose else []) + ["-o", lib] + SOURCES
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
-    nvcc = os.environ.get("NVCC", "nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + SOURCES
-    subprocess.run(cmd, check=True)
+    subprocess.run(_command(LIB, [], verbose), check=True)
     return LIB
+
+
+def build_variant(name: str, force: bool = False) -> str:
+    """Builds (if stale) and returns the path of a tests-only variant."""
+    lib, defines = VARIANTS[name]
+    if force or _stale(lib):
+        subprocess.run(_command(lib, defines, False), check=True)
+    return lib
+
+
+def build_all(force: bool = False) -> None:
+    """The product and the tests-only variants, compiled side by side."""
+    jobs = []
+    if force or needs_build():
+        jobs.append(subprocess.Popen(_command(LIB, [], False)))
+    for lib, defines in VARIANTS.values():
+        if force or _stale(lib):
+            jobs.append(subprocess.Popen(_command(lib, defines, False)))
+    failed = [j.args for j in jobs if j.wait() != 0]
+    if failed:
+        raise subprocess.CalledProcessError(1, failed[0])
 
 
 if __name__ == "__main__":
     import sys
+    if "--all" in sys.argv:
+        build_all(force="--force" in sys.argv)
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

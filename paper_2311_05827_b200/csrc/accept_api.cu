@@ -4,6 +4,7 @@
 #include "../../include/accept.h"
 
 #include <atomic>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <utility>
@@ -90,6 +91,51 @@ cudaError_t launch_overlapped(void (*fn)(Params...), dim3 grid, unsigned block, 
   return launch_overlapped_shared(fn, grid, block, 0, s, std::forward<Args>(args)...);
 }
 
+// A launch (or any runtime call) that fails ends the entry point at once: later launches of the same call
+// are not issued, and only launches that were issued are counted.  The result is the call's own return
+// value; cudaGetLastError() is never consulted, so an error left behind by the caller's earlier work is
+// neither reported as ours nor cleared.
+#define ACCEPT_LAUNCH(call)                                         \
+  do {                                                              \
+    if ((call) != cudaSuccess) return ACCEPT_ERR_CUDA;              \
+    g_launches.fetch_add(1, std::memory_order_relaxed);             \
+  } while (0)
+
+// ---- tests-only build: byte ranges the kernels of a call may touch ------------------------------------
+#ifdef ACCEPT_BOUNDS_CHECK
+// ACCEPT_BOUNDS_TEST_SHRINK=<bytes> in the environment cuts that many bytes off the end of every writable
+// range: the test of the checker itself, which shows that the last stores of a call are then counted and
+// skipped (nothing is written there, nothing faults).
+size_t bounds_test_shrink() {
+  const char* text = std::getenv("ACCEPT_BOUNDS_TEST_SHRINK");
+  return text ? (size_t)std::strtoull(text, nullptr, 10) : 0;
+}
+
+struct BoundsList {
+  accept::BoundsTable table{};
+  void add(const void* p, size_t bytes, bool writable) {
+    if (!p || table.n >= accept::kMaxBoundsRanges) return;
+    if (writable) bytes -= bounds_test_shrink() < bytes ? bounds_test_shrink() : bytes;
+    table.lo[table.n] = (unsigned long long)p;
+    table.hi[table.n] = (unsigned long long)p + bytes;
+    table.writable[table.n] = writable ? 1u : 0u;
+    ++table.n;
+  }
+  // ordered with the call's kernels on its stream (the source is pageable host memory: staged before return)
+  cudaError_t install(cudaStream_t s) const {
+    return cudaMemcpyToSymbolAsync(accept::g_bounds, &table, sizeof(table), 0, cudaMemcpyHostToDevice, s);
+  }
+};
+#define ACCEPT_BOUNDS(stream, ...)                                              \
+  do {                                                                          \
+    BoundsList bounds_list;                                                     \
+    __VA_ARGS__;                                                                \
+    if (bounds_list.install(stream) != cudaSuccess) return ACCEPT_ERR_CUDA;     \
+  } while (0)
+#else
+#define ACCEPT_BOUNDS(stream, ...) do { } while (0)
+#endif
+
 // ---- kernel tables -------------------------------------------------------------------------
 
 using KernelFn = void (*)(const CodecArgs);
@@ -166,28 +212,27 @@ KernelFn select_decompress(const accept_params* p, bool aligned, int rounds) {
 constexpr int kWideOctetsNearest = 2, kWideOctetsStochastic = 4;
 
 template <int K, int LAYOUT, int RANGE>
-void launch_wide_encode(int round, const CodecArgs& a, const accept::ChunkRecord* rec, uint64_t n_oct_stored, cudaStream_t s) {
+cudaError_t launch_wide_encode(int round, const CodecArgs& a, const accept::ChunkRecord* rec, uint64_t n_oct_stored, cudaStream_t s) {
   if (round == accept::kNearest) {
     const unsigned grid = (unsigned)((n_oct_stored + kWideOctetsNearest * 256 - 1) / (kWideOctetsNearest * 256));
-    launch_overlapped(accept::wide_encode_kernel<K, LAYOUT, RANGE, accept::kNearest, kWideOctetsNearest>, dim3(grid), 256, s, a, rec);
-  } else {
-    const unsigned grid = (unsigned)((n_oct_stored + kWideOctetsStochastic * 256 - 1) / (kWideOctetsStochastic * 256));
-    launch_overlapped(accept::wide_encode_kernel<K, LAYOUT, RANGE, accept::kStochastic, kWideOctetsStochastic>, dim3(grid), 256, s, a, rec);
+    return launch_overlapped(accept::wide_encode_kernel<K, LAYOUT, RANGE, accept::kNearest, kWideOctetsNearest>, dim3(grid), 256, s, a, rec);
   }
+  const unsigned grid = (unsigned)((n_oct_stored + kWideOctetsStochastic * 256 - 1) / (kWideOctetsStochastic * 256));
+  return launch_overlapped(accept::wide_encode_kernel<K, LAYOUT, RANGE, accept::kStochastic, kWideOctetsStochastic>, dim3(grid), 256, s, a, rec);
 }
 
 template <int RANGE>
-void launch_wide_encode_for(const accept_params* p, const CodecArgs& a, const accept::ChunkRecord* rec, uint64_t grid,
-                            cudaStream_t s) {
+cudaError_t launch_wide_encode_for(const accept_params* p, const CodecArgs& a, const accept::ChunkRecord* rec, uint64_t grid,
+                                   cudaStream_t s) {
   const bool bp = p->layout == ACCEPT_LAYOUT_BITPLANE;
   switch (p->k) {
-    case 2: bp ? launch_wide_encode<2, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
-               : launch_wide_encode<2, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s); break;
-    case 3: launch_wide_encode<3, accept::kBitplane, RANGE>(p->round, a, rec, grid, s); break;
-    case 4: bp ? launch_wide_encode<4, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
-               : launch_wide_encode<4, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s); break;
-    default: bp ? launch_wide_encode<8, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
-                : launch_wide_encode<8, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s); break;
+    case 2: return bp ? launch_wide_encode<2, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
+                      : launch_wide_encode<2, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s);
+    case 3: return launch_wide_encode<3, accept::kBitplane, RANGE>(p->round, a, rec, grid, s);
+    case 4: return bp ? launch_wide_encode<4, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
+                      : launch_wide_encode<4, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s);
+    default: return bp ? launch_wide_encode<8, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
+                       : launch_wide_encode<8, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s);
   }
 }
 
@@ -200,16 +245,15 @@ accept_status launch_wide(const accept_params* p, const CodecArgs& a, uint8_t* r
   const unsigned fin_grid = (unsigned)((a.n_chunks + 255) / 256);
   const uint64_t enc_grid = ((p->n_elems + 31) / 32) * 4;  // octets the encode pass stores
   if (p->range == ACCEPT_RANGE_ABSMAX) {
-    launch_overlapped(accept::wide_range_kernel<accept::kAbsMax, 4>, dim3(range_grid), 256, s, a, rec);
-    launch_overlapped(accept::wide_finalize_kernel<accept::kAbsMax>, dim3(fin_grid), 256, s, a, rec);
-    launch_wide_encode_for<accept::kAbsMax>(p, a, rec, enc_grid, s);
+    ACCEPT_LAUNCH(launch_overlapped(accept::wide_range_kernel<accept::kAbsMax, 4>, dim3(range_grid), 256, s, a, rec));
+    ACCEPT_LAUNCH(launch_overlapped(accept::wide_finalize_kernel<accept::kAbsMax>, dim3(fin_grid), 256, s, a, rec));
+    ACCEPT_LAUNCH(launch_wide_encode_for<accept::kAbsMax>(p, a, rec, enc_grid, s));
   } else {
-    launch_overlapped(accept::wide_range_kernel<accept::kMinMax, 4>, dim3(range_grid), 256, s, a, rec);
-    launch_overlapped(accept::wide_finalize_kernel<accept::kMinMax>, dim3(fin_grid), 256, s, a, rec);
-    launch_wide_encode_for<accept::kMinMax>(p, a, rec, enc_grid, s);
+    ACCEPT_LAUNCH(launch_overlapped(accept::wide_range_kernel<accept::kMinMax, 4>, dim3(range_grid), 256, s, a, rec));
+    ACCEPT_LAUNCH(launch_overlapped(accept::wide_finalize_kernel<accept::kMinMax>, dim3(fin_grid), 256, s, a, rec));
+    ACCEPT_LAUNCH(launch_wide_encode_for<accept::kMinMax>(p, a, rec, enc_grid, s));
   }
-  g_launches.fetch_add(3, std::memory_order_relaxed);
-  return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+  return ACCEPT_OK;
 }
 
 // ---- pack groups along the batch dimension ---------------------------------------------------------
@@ -218,15 +262,14 @@ accept_status launch_wide(const accept_params* p, const CodecArgs& a, uint8_t* r
 constexpr unsigned kStridedEncodeBlocks = 3 * 148;
 
 template <int K, int LAYOUT, int RANGE>
-void launch_strided_encode(int round, const CodecArgs& a, const accept::ChunkRecord* rec, dim3 tiles, cudaStream_t s) {
-  if (round != accept::kNearest) {  // instruction bound: one tile per block, rows in registers
-    launch_overlapped(accept::strided_encode_direct_kernel<K, LAYOUT, RANGE, accept::kStochastic>, tiles, 256, s, a, rec);
-    return;
-  }
+cudaError_t launch_strided_encode(int round, const CodecArgs& a, const accept::ChunkRecord* rec, dim3 tiles, cudaStream_t s) {
+  if (round != accept::kNearest)  // instruction bound: one tile per block, rows in registers
+    return launch_overlapped(accept::strided_encode_direct_kernel<K, LAYOUT, RANGE, accept::kStochastic>, tiles, 256, s, a, rec);
   // memory bound: persistent blocks with a staged tile, which needs more dynamic shared memory than a
   // kernel gets without opting in (the attribute is per device: set every time)
   auto fn = accept::strided_encode_kernel<K, LAYOUT, RANGE, accept::kNearest>;
-  if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, accept::kStridedSmemBytes) != cudaSuccess) return;
+  const cudaError_t err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, accept::kStridedSmemBytes);
+  if (err != cudaSuccess) return err;
   const uint64_t n_tiles = (uint64_t)tiles.x * tiles.y;
   const unsigned grid = (unsigned)(n_tiles < kStridedEncodeBlocks ? n_tiles : kStridedEncodeBlocks);
   accept::StridedTiling t;
@@ -235,33 +278,33 @@ void launch_strided_encode(int round, const CodecArgs& a, const accept::ChunkRec
   t.n_rows = (uint32_t)(a.n / a.group_stride);
   t.step_x = grid % tiles.x;
   t.step_y = grid / tiles.x;
-  launch_overlapped_shared(fn, dim3(grid), 256, accept::kStridedSmemBytes, s, a, rec, t);
+  return launch_overlapped_shared(fn, dim3(grid), 256, accept::kStridedSmemBytes, s, a, rec, t);
 }
 
 template <int RANGE>
-void launch_strided_encode_for(const accept_params* p, const CodecArgs& a, const accept::ChunkRecord* rec, dim3 grid,
-                               cudaStream_t s) {
+cudaError_t launch_strided_encode_for(const accept_params* p, const CodecArgs& a, const accept::ChunkRecord* rec, dim3 grid,
+                                      cudaStream_t s) {
   const bool bp = p->layout == ACCEPT_LAYOUT_BITPLANE;
   switch (p->k) {
-    case 2: bp ? launch_strided_encode<2, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
-               : launch_strided_encode<2, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s); break;
-    case 3: launch_strided_encode<3, accept::kBitplane, RANGE>(p->round, a, rec, grid, s); break;
-    case 4: bp ? launch_strided_encode<4, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
-               : launch_strided_encode<4, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s); break;
-    default: launch_strided_encode<8, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s); break;
+    case 2: return bp ? launch_strided_encode<2, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
+                      : launch_strided_encode<2, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s);
+    case 3: return launch_strided_encode<3, accept::kBitplane, RANGE>(p->round, a, rec, grid, s);
+    case 4: return bp ? launch_strided_encode<4, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
+                      : launch_strided_encode<4, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s);
+    default: return launch_strided_encode<8, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s);
   }
 }
 
 template <int RANGE>
-void launch_strided_decode_for(const accept_params* p, const CodecArgs& a, dim3 grid, cudaStream_t s) {
+cudaError_t launch_strided_decode_for(const accept_params* p, const CodecArgs& a, dim3 grid, cudaStream_t s) {
   const bool bp = p->layout == ACCEPT_LAYOUT_BITPLANE;
   switch (p->k) {
-    case 2: bp ? launch_overlapped(accept::strided_decode_kernel<2, accept::kBitplane, RANGE>, dim3(grid), 256, s, a)
-               : launch_overlapped(accept::strided_decode_kernel<2, accept::kInterleaved, RANGE>, dim3(grid), 256, s, a); break;
-    case 3: launch_overlapped(accept::strided_decode_kernel<3, accept::kBitplane, RANGE>, dim3(grid), 256, s, a); break;
-    case 4: bp ? launch_overlapped(accept::strided_decode_kernel<4, accept::kBitplane, RANGE>, dim3(grid), 256, s, a)
-               : launch_overlapped(accept::strided_decode_kernel<4, accept::kInterleaved, RANGE>, dim3(grid), 256, s, a); break;
-    default: launch_overlapped(accept::strided_decode_kernel<8, accept::kInterleaved, RANGE>, dim3(grid), 256, s, a); break;
+    case 2: return bp ? launch_overlapped(accept::strided_decode_kernel<2, accept::kBitplane, RANGE>, dim3(grid), 256, s, a)
+                      : launch_overlapped(accept::strided_decode_kernel<2, accept::kInterleaved, RANGE>, dim3(grid), 256, s, a);
+    case 3: return launch_overlapped(accept::strided_decode_kernel<3, accept::kBitplane, RANGE>, dim3(grid), 256, s, a);
+    case 4: return bp ? launch_overlapped(accept::strided_decode_kernel<4, accept::kBitplane, RANGE>, dim3(grid), 256, s, a)
+                      : launch_overlapped(accept::strided_decode_kernel<4, accept::kInterleaved, RANGE>, dim3(grid), 256, s, a);
+    default: return launch_overlapped(accept::strided_decode_kernel<8, accept::kInterleaved, RANGE>, dim3(grid), 256, s, a);
   }
 }
 
@@ -278,16 +321,15 @@ accept_status launch_strided(const accept_params* p, const CodecArgs& a, uint8_t
   const unsigned range_grid = (unsigned)((n_oct + 4 * 256 - 1) / (4 * 256));
   const unsigned fin_grid = (unsigned)((a.n_chunks + 255) / 256);
   if (p->range == ACCEPT_RANGE_ABSMAX) {
-    launch_overlapped(accept::wide_range_kernel<accept::kAbsMax, 4>, dim3(range_grid), 256, s, a, rec);
-    launch_overlapped(accept::wide_finalize_kernel<accept::kAbsMax>, dim3(fin_grid), 256, s, a, rec);
-    launch_strided_encode_for<accept::kAbsMax>(p, a, rec, strided_grid(p), s);
+    ACCEPT_LAUNCH(launch_overlapped(accept::wide_range_kernel<accept::kAbsMax, 4>, dim3(range_grid), 256, s, a, rec));
+    ACCEPT_LAUNCH(launch_overlapped(accept::wide_finalize_kernel<accept::kAbsMax>, dim3(fin_grid), 256, s, a, rec));
+    ACCEPT_LAUNCH(launch_strided_encode_for<accept::kAbsMax>(p, a, rec, strided_grid(p), s));
   } else {
-    launch_overlapped(accept::wide_range_kernel<accept::kMinMax, 4>, dim3(range_grid), 256, s, a, rec);
-    launch_overlapped(accept::wide_finalize_kernel<accept::kMinMax>, dim3(fin_grid), 256, s, a, rec);
-    launch_strided_encode_for<accept::kMinMax>(p, a, rec, strided_grid(p), s);
+    ACCEPT_LAUNCH(launch_overlapped(accept::wide_range_kernel<accept::kMinMax, 4>, dim3(range_grid), 256, s, a, rec));
+    ACCEPT_LAUNCH(launch_overlapped(accept::wide_finalize_kernel<accept::kMinMax>, dim3(fin_grid), 256, s, a, rec));
+    ACCEPT_LAUNCH(launch_strided_encode_for<accept::kMinMax>(p, a, rec, strided_grid(p), s));
   }
-  g_launches.fetch_add(3, std::memory_order_relaxed);
-  return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+  return ACCEPT_OK;
 }
 
 // ---- multi-bit quantization --------------------------------------------------------------------
@@ -324,20 +366,22 @@ accept::MbqArgs mbq_args(const accept_mbq_params* p, void* d_stream, void* d_ws)
 }
 
 template <int K>
-void launch_mbq_compress(const accept::MbqArgs& a, cudaStream_t s) {
+accept_status launch_mbq_compress(const accept::MbqArgs& a, cudaStream_t s) {
   const dim3 grid((a.n_blocks + accept::kMbqGroups - 1) / accept::kMbqGroups);
   if (a.init) {
-    for (int j = 0; j < K; ++j) launch_overlapped(accept::mbq_residue_sum_kernel<K>, dim3(a.n_residue_blocks), 256, s, a, j);
-    launch_overlapped(accept::mbq_encode_kernel<K, true>, grid, accept::kMbqEncodeThreads, s, a);
+    for (int j = 0; j < K; ++j)
+      ACCEPT_LAUNCH(launch_overlapped(accept::mbq_residue_sum_kernel<K>, dim3(a.n_residue_blocks), 256, s, a, j));
+    ACCEPT_LAUNCH(launch_overlapped(accept::mbq_encode_kernel<K, true>, grid, accept::kMbqEncodeThreads, s, a));
   } else {
     // the search grid needs more dynamic shared memory than a kernel gets without opting in (the
     // attribute is per device: set every time)
     auto fn = accept::mbq_encode_kernel<K, false>;
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, accept::kMbqGridBytes) != cudaSuccess) return;
-    launch_overlapped_shared(fn, grid, accept::kMbqEncodeThreads, accept::kMbqGridBytes, s, a);
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, accept::kMbqGridBytes) != cudaSuccess)
+      return ACCEPT_ERR_CUDA;
+    ACCEPT_LAUNCH(launch_overlapped_shared(fn, grid, accept::kMbqEncodeThreads, accept::kMbqGridBytes, s, a));
   }
-  launch_overlapped(accept::mbq_finalize_kernel<K>, dim3(1), accept::kMbqFinalizeThreads, s, a);
-  g_launches.fetch_add(2 + (a.init ? K : 0), std::memory_order_relaxed);
+  ACCEPT_LAUNCH(launch_overlapped(accept::mbq_finalize_kernel<K>, dim3(1), accept::kMbqFinalizeThreads, s, a));
+  return ACCEPT_OK;
 }
 
 // ---- built-in scratch for accept_compress_static ------------------------------------------------
@@ -364,12 +408,15 @@ void* static_scratch_address() {
   return g_scratch_address[dev];
 }
 
+// ws_need: bytes of workspace the call touches (the compress side: accept_workspace_size; the decode side:
+// the status word only, whatever the parameters).
 accept_status check_buffers(const accept_params* p, const void* d_tensor, const void* d_stream,
-                            size_t stream_bytes, const void* d_ws, size_t ws_bytes) {
+                            size_t stream_bytes, const void* d_ws, size_t ws_bytes, bool decode) {
   if (!p || !d_tensor || !d_stream || !d_ws) return ACCEPT_ERR_NULL;
   accept_status st = accept_check_params(p);
   if (st != ACCEPT_OK) return st;
-  if (stream_bytes < accept_compressed_size(p) || ws_bytes < accept_workspace_size(p)) return ACCEPT_ERR_TOO_SMALL;
+  const size_t ws_need = decode ? 16 : accept_workspace_size(p);
+  if (stream_bytes < accept_compressed_size(p) || ws_bytes < ws_need) return ACCEPT_ERR_TOO_SMALL;
   if (!is_aligned(d_tensor, 16) || !is_aligned(d_stream, 16) || !is_aligned(d_ws, 4)) return ACCEPT_ERR_MISALIGNED;
   return ACCEPT_OK;
 }
@@ -416,10 +463,12 @@ size_t accept_workspace_size(const accept_params* p) {
 
 accept_status accept_compress(const accept_params* p, const float* d_x, void* d_stream, size_t stream_bytes,
                               void* d_ws, size_t ws_bytes, void* cuda_stream) {
-  accept_status st = check_buffers(p, d_x, d_stream, stream_bytes, d_ws, ws_bytes);
+  accept_status st = check_buffers(p, d_x, d_stream, stream_bytes, d_ws, ws_bytes, false);
   if (st != ACCEPT_OK) return st;
   CodecArgs a = make_args(p, d_stream, d_ws);
   a.x = d_x;
+  ACCEPT_BOUNDS(static_cast<cudaStream_t>(cuda_stream), bounds_list.add(d_x, 4 * p->n_elems, false);
+                bounds_list.add(d_stream, accept_compressed_size(p), true); bounds_list.add(d_ws, accept_workspace_size(p), true));
 
   if (is_strided(p)) {
     if (!is_aligned(d_x, 32) || !is_aligned(d_ws, 16)) return ACCEPT_ERR_MISALIGNED;
@@ -451,39 +500,38 @@ accept_status accept_compress(const accept_params* p, const float* d_x, void* d_
   a.fast_blocks = (uint32_t)fast_blocks;
   const uint64_t grid = fast_blocks + (a.n_chunks - a.n_fast_chunks);
   KernelFn fn = select_compress(p, fast ? g.rounds : 2, block <= 256);
-  const cudaError_t err = launch_overlapped(fn, (unsigned)grid, block, static_cast<cudaStream_t>(cuda_stream), a);
-  g_launches.fetch_add(1, std::memory_order_relaxed);
-  return err == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+  ACCEPT_LAUNCH(launch_overlapped(fn, (unsigned)grid, block, static_cast<cudaStream_t>(cuda_stream), a));
+  return ACCEPT_OK;
 }
 
 accept_status accept_decompress(const accept_params* p, const void* d_stream, size_t stream_bytes, float* d_xhat,
                                 void* d_ws, size_t ws_bytes, void* cuda_stream) {
-  accept_status st = check_buffers(p, d_xhat, d_stream, stream_bytes, d_ws, ws_bytes);
+  accept_status st = check_buffers(p, d_xhat, d_stream, stream_bytes, d_ws, ws_bytes, true);
   if (st != ACCEPT_OK) return st;
   CodecArgs a = make_args(p, const_cast<void*>(d_stream), d_ws);
   a.xhat = d_xhat;
+  ACCEPT_BOUNDS(static_cast<cudaStream_t>(cuda_stream), bounds_list.add(d_stream, accept_compressed_size(p), false);
+                bounds_list.add(d_xhat, 4 * p->n_elems, true); bounds_list.add(d_ws, 16, true));
   if (is_strided(p)) {
     if (!is_aligned(d_xhat, 32)) return ACCEPT_ERR_MISALIGNED;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    if (p->range == ACCEPT_RANGE_ABSMAX) launch_strided_decode_for<accept::kAbsMax>(p, a, strided_grid(p), s);
-    else launch_strided_decode_for<accept::kMinMax>(p, a, strided_grid(p), s);
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+    if (p->range == ACCEPT_RANGE_ABSMAX) ACCEPT_LAUNCH(launch_strided_decode_for<accept::kAbsMax>(p, a, strided_grid(p), s));
+    else ACCEPT_LAUNCH(launch_strided_decode_for<accept::kMinMax>(p, a, strided_grid(p), s));
+    return ACCEPT_OK;
   }
   const bool aligned = is_aligned(d_xhat, 32);
   const int rounds = 2;  // octets per thread
   KernelFn fn = select_decompress(p, aligned, rounds);
   const uint64_t per_block = aligned ? 2048ull * rounds : 256;  // elements per block
   const uint64_t grid = (p->n_elems + per_block - 1) / per_block;
-  const cudaError_t err = launch_overlapped(fn, (unsigned)grid, 256, static_cast<cudaStream_t>(cuda_stream), a);
-  g_launches.fetch_add(1, std::memory_order_relaxed);
-  return err == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+  ACCEPT_LAUNCH(launch_overlapped(fn, (unsigned)grid, 256, static_cast<cudaStream_t>(cuda_stream), a));
+  return ACCEPT_OK;
 }
 
 accept_status accept_compress_host(const accept_params* p, const float* h_x, void* h_stream, size_t stream_bytes,
                                    float* d_x, void* d_stream, void* d_ws, size_t ws_bytes, void* cuda_stream) {
   if (!h_x || !h_stream) return ACCEPT_ERR_NULL;
-  accept_status st = check_buffers(p, d_x, d_stream, stream_bytes, d_ws, ws_bytes);
+  accept_status st = check_buffers(p, d_x, d_stream, stream_bytes, d_ws, ws_bytes, false);
   if (st != ACCEPT_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   if (cudaMemcpyAsync(d_x, h_x, p->n_elems * sizeof(float), cudaMemcpyHostToDevice, s) != cudaSuccess)
@@ -499,7 +547,7 @@ accept_status accept_decompress_host(const accept_params* p, const void* h_strea
                                      float* h_xhat, void* d_stream, float* d_xhat, void* d_ws, size_t ws_bytes,
                                      void* cuda_stream) {
   if (!h_stream || !h_xhat) return ACCEPT_ERR_NULL;
-  accept_status st = check_buffers(p, d_xhat, d_stream, stream_bytes, d_ws, ws_bytes);
+  accept_status st = check_buffers(p, d_xhat, d_stream, stream_bytes, d_ws, ws_bytes, true);
   if (st != ACCEPT_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   if (cudaMemcpyAsync(d_stream, h_stream, accept_compressed_size(p), cudaMemcpyHostToDevice, s) != cudaSuccess)
@@ -583,12 +631,14 @@ accept_status accept_mbq_compress(const accept_mbq_params* p, const float* d_x, 
   a.alpha_prev = d_alpha_prev;
   a.alpha_next = d_alpha_next;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  ACCEPT_BOUNDS(s, bounds_list.add(d_x, 4 * p->n_elems, false); bounds_list.add(d_alpha_prev, 4 * p->k, false);
+                bounds_list.add(d_alpha_next, 4 * p->k, true); bounds_list.add(d_stream, accept_mbq_compressed_size(p), true);
+                bounds_list.add(d_ws, accept_mbq_workspace_size(p), true));
   switch (p->k) {
-    case 2: launch_mbq_compress<2>(a, s); break;
-    case 3: launch_mbq_compress<3>(a, s); break;
-    default: launch_mbq_compress<4>(a, s); break;
+    case 2: return launch_mbq_compress<2>(a, s);
+    case 3: return launch_mbq_compress<3>(a, s);
+    default: return launch_mbq_compress<4>(a, s);
   }
-  return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
 }
 
 accept_status accept_mbq_decompress(const accept_mbq_params* p, const void* d_stream, size_t stream_bytes,
@@ -602,16 +652,40 @@ accept_status accept_mbq_decompress(const accept_mbq_params* p, const void* d_st
   a.xhat = d_xhat;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   const unsigned grid = (unsigned)((p->n_elems + 4095) / 4096);
+  ACCEPT_BOUNDS(s, bounds_list.add(d_stream, accept_mbq_compressed_size(p), false); bounds_list.add(d_xhat, 4 * p->n_elems, true);
+                bounds_list.add(d_ws, 16, true));
   switch (p->k) {
-    case 2: launch_overlapped(accept::mbq_decode_kernel<2>, dim3(grid), 256, s, a); break;
-    case 3: launch_overlapped(accept::mbq_decode_kernel<3>, dim3(grid), 256, s, a); break;
-    default: launch_overlapped(accept::mbq_decode_kernel<4>, dim3(grid), 256, s, a); break;
+    case 2: ACCEPT_LAUNCH(launch_overlapped(accept::mbq_decode_kernel<2>, dim3(grid), 256, s, a)); break;
+    case 3: ACCEPT_LAUNCH(launch_overlapped(accept::mbq_decode_kernel<3>, dim3(grid), 256, s, a)); break;
+    default: ACCEPT_LAUNCH(launch_overlapped(accept::mbq_decode_kernel<4>, dim3(grid), 256, s, a)); break;
   }
-  g_launches.fetch_add(1, std::memory_order_relaxed);
-  return cudaGetLastError() == cudaSuccess ? ACCEPT_OK : ACCEPT_ERR_CUDA;
+  return ACCEPT_OK;
 }
 
 uint64_t accept_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+accept_status accept_bounds_check_report(void* cuda_stream, uint32_t* violations, uint64_t* first_address,
+                                         uint64_t* first_size_and_kind) {
+  if (!violations) return ACCEPT_ERR_NULL;
+#ifndef ACCEPT_BOUNDS_CHECK
+  (void)cuda_stream;
+  *violations = 0;
+  if (first_address) *first_address = 0;
+  if (first_size_and_kind) *first_size_and_kind = 0;
+  return ACCEPT_ERR_UNCHECKED_BUILD;
+#else
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  unsigned long long first[2] = {0, 0};
+  const unsigned int zero = 0;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return ACCEPT_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(violations, accept::g_bounds_violations, sizeof(uint32_t)) != cudaSuccess) return ACCEPT_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(first, accept::g_bounds_first, sizeof(first)) != cudaSuccess) return ACCEPT_ERR_CUDA;
+  if (cudaMemcpyToSymbol(accept::g_bounds_violations, &zero, sizeof(zero)) != cudaSuccess) return ACCEPT_ERR_CUDA;
+  if (first_address) *first_address = first[0];
+  if (first_size_and_kind) *first_size_and_kind = first[1];
+  return ACCEPT_OK;
+#endif
+}
 
 accept_status accept_compress_static(const accept_params* p, const float* d_x, void* d_stream, size_t stream_bytes,
                                      uint32_t* d_status_out, void* cuda_stream) {
@@ -623,6 +697,12 @@ accept_status accept_compress_static(const accept_params* p, const float* d_x, v
   if (stream_bytes < accept_compressed_size(p)) return ACCEPT_ERR_TOO_SMALL;
   if (!is_aligned(d_x, 16) || !is_aligned(d_stream, 16) || !is_aligned(d_status_out, 4)) return ACCEPT_ERR_MISALIGNED;
 
+  // the built-in array is looked up on the CURRENT device: an input that lives on another one would make the
+  // kernel run there with this device's scratch address
+  int current = -1;
+  cudaPointerAttributes where{};
+  if (cudaGetDevice(&current) != cudaSuccess || cudaPointerGetAttributes(&where, d_x) != cudaSuccess) return ACCEPT_ERR_CUDA;
+  if (where.type == cudaMemoryTypeDevice && where.device != current) return ACCEPT_ERR_CUDA;
   void* scratch = static_scratch_address();
   if (!scratch) return ACCEPT_ERR_CUDA;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);

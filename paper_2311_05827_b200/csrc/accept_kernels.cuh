@@ -60,16 +60,16 @@ constexpr int kGenericBlock = 256;  // threads per block of the any-shape path
 template <int K>
 __device__ __forceinline__ void store_interleaved(uint32_t* payload, uint64_t oct, uint32_t xlo, uint32_t xhi) {
   if (K == 8) {
-    reinterpret_cast<uint2*>(payload)[oct] = make_uint2(xlo, xhi);
+    st_c(reinterpret_cast<uint2*>(payload) + oct, make_uint2(xlo, xhi));
   } else if (K == 4) {
     // bytes u0|u1<<4 and u2|u3<<4 sit in bytes 0 and 2 of x | x>>4
     const uint32_t ylo = xlo | (xlo >> 4), yhi = xhi | (xhi >> 4);
-    payload[oct] = __byte_perm(ylo, yhi, 0x6420);
+    st_c(payload + oct, __byte_perm(ylo, yhi, 0x6420));
   } else {  // K == 2
     uint32_t ylo = xlo | (xlo >> 6), yhi = xhi | (xhi >> 6);
     ylo |= ylo >> 12;
     yhi |= yhi >> 12;
-    reinterpret_cast<uint16_t*>(payload)[oct] = (uint16_t)__byte_perm(ylo, yhi, 0x0040);
+    st_c(reinterpret_cast<uint16_t*>(payload) + oct, (uint16_t)__byte_perm(ylo, yhi, 0x0040));
   }
 }
 
@@ -82,7 +82,7 @@ __device__ __forceinline__ uint32_t store_bitplane_guarded(uint32_t* payload, ui
   const int q = lane & 3;
   if (K <= 4) {
     const uint32_t w = quad_transpose(planes_nibbles(merge_nibbles(xlo, xhi)), lane);
-    if (store && q < K) payload[group * K + q] = w;
+    if (store && q < K) st_c(payload + group * K + q, w);
     return w;
   } else {
     const uint32_t lo = merge_nibbles(xlo & 0x0F0F0F0Fu, xhi & 0x0F0F0F0Fu);
@@ -90,8 +90,8 @@ __device__ __forceinline__ uint32_t store_bitplane_guarded(uint32_t* payload, ui
     const uint32_t w0 = quad_transpose(planes_nibbles(lo), lane);
     const uint32_t w1 = quad_transpose(planes_nibbles(hi), lane);
     if (store) {
-      payload[group * 8 + q] = w0;
-      payload[group * 8 + 4 + q] = w1;
+      st_c(payload + group * 8 + q, w0);
+      st_c(payload + group * 8 + 4 + q, w1);
     }
     return 0u;
   }
@@ -118,7 +118,7 @@ __device__ void compress_chunk_generic(const CodecArgs& a, uint64_t m, float* s_
 
   Range<RANGE> rg;
   rg.init();
-  for (uint32_t i = tid; i < valid; i += blockDim.x) rg.add(__ldg(x + i));
+  for (uint32_t i = tid; i < valid; i += blockDim.x) rg.add(ldg_c(x + i));
   rg.warp_reduce();
   __syncthreads();  // protects s_hi/s_lo against a previous use
   if (lane == 0) { s_hi[warp] = rg.hi; s_lo[warp] = rg.lo; }
@@ -128,7 +128,7 @@ __device__ void compress_chunk_generic(const CodecArgs& a, uint64_t m, float* s_
 
   Scale sc = make_scale<K, RANGE>(rg.hi, rg.lo);
   if (tid == 0) {
-    a.meta[m] = make_float2(sc.s, sc.o);
+    st_c(a.meta + m, make_float2(sc.s, sc.o));
     if (sc.nonfinite) atomicOr(a.status, kDevNonFinite);
   }
   Rng rng{(uint32_t)a.seed, (uint32_t)(a.seed >> 32)};
@@ -137,7 +137,7 @@ __device__ void compress_chunk_generic(const CodecArgs& a, uint64_t m, float* s_
     const uint32_t t = g * 32 + lane;
     uint32_t u = 0;
     if (t < valid) {
-      float v = __ldg(x + t);
+      float v = ldg_c(x + t);
       if (sc.nonfinite) v = 0.0f;
       uint32_t h = 0;
       if (ROUND == kStochastic) h = rng.word(a.rng_offset + i0 + t);
@@ -155,7 +155,7 @@ __device__ void compress_chunk_generic(const CodecArgs& a, uint64_t m, float* s_
         bit = (__shfl_sync(0xffffffffu, u, pos / K) >> (pos % K)) & 1u;
       }
       const uint32_t word = __ballot_sync(0xffffffffu, bit);
-      if (lane == w) a.payload[word0 + w] = word;
+      if (lane == w) st_c(a.payload + word0 + w, word);
     }
   }
 }
@@ -178,8 +178,8 @@ __global__ void __launch_bounds__(BLOCK_MAX, BLOCK_MAX == 256 ? (R <= 2 ? 6 : 4)
 
   if (blockIdx.x == 0 && tid < 8) {
     // stream header and the pad between the side words and the payload
-    a.header[tid] = header_word(a, tid);
-    if ((a.n_chunks & 1) && tid < 2) reinterpret_cast<uint32_t*>(a.meta + a.n_chunks)[tid] = 0u;
+    st_c(a.header + tid, header_word(a, tid));
+    if ((a.n_chunks & 1) && tid < 2) st_c(reinterpret_cast<uint32_t*>(a.meta + a.n_chunks) + tid, 0u);
   }
 
   if (blockIdx.x >= a.fast_blocks) {
@@ -219,7 +219,7 @@ __global__ void __launch_bounds__(BLOCK_MAX, BLOCK_MAX == 256 ? (R <= 2 ? 6 : 4)
 
   Scale sc = make_scale<K, RANGE>(rg.hi, rg.lo);
   if (gt == 0 && active) {
-    a.meta[m] = make_float2(sc.s, sc.o);
+    st_c(a.meta + m, make_float2(sc.s, sc.o));
     if (sc.nonfinite) atomicOr(a.status, kDevNonFinite);
   }
   if (sc.nonfinite) {
@@ -260,12 +260,12 @@ __device__ __forceinline__ RawOctet load_raw(const CodecArgs& a, uint64_t oct, u
   if (LAYOUT == kInterleaved) {
     if (oct < n_oct) {
       if (K == 8) {
-        const uint2 w = __ldg(reinterpret_cast<const uint2*>(a.payload) + oct);
+        const uint2 w = ldg_c(reinterpret_cast<const uint2*>(a.payload) + oct);
         raw.w0 = w.x; raw.w1 = w.y;
       } else if (K == 4) {
-        raw.w0 = __ldg(a.payload + oct);
+        raw.w0 = ldg_c(a.payload + oct);
       } else {
-        raw.w0 = __ldg(reinterpret_cast<const uint16_t*>(a.payload) + oct);
+        raw.w0 = ldg_c(reinterpret_cast<const uint16_t*>(a.payload) + oct);
       }
     }
   } else {
@@ -274,17 +274,17 @@ __device__ __forceinline__ RawOctet load_raw(const CodecArgs& a, uint64_t oct, u
     const uint64_t group = oct >> 2;
     if (group < n_groups) {
       if (K <= 4) {
-        if (q < K) raw.w0 = __ldg(a.payload + group * K + q);
+        if (q < K) raw.w0 = ldg_c(a.payload + group * K + q);
       } else {
-        raw.w0 = __ldg(a.payload + group * 8 + q);
-        raw.w1 = __ldg(a.payload + group * 8 + 4 + q);
+        raw.w0 = ldg_c(a.payload + group * 8 + q);
+        raw.w1 = ldg_c(a.payload + group * 8 + 4 + q);
       }
     }
   }
   if (oct < n_oct) {
     const uint64_t e = oct * 8;
     const uint64_t m = (a.chunk_shift >= 0) ? (e >> a.chunk_shift) : (e / a.chunk);
-    raw.so = __ldg(a.meta + m);
+    raw.so = ldg_c(a.meta + m);
   }
   return raw;
 }
@@ -344,7 +344,7 @@ __device__ __forceinline__ void decode_tile(const CodecArgs& a, const RawOctet (
         st_octet(a.xhat + e, out);
       } else {
         for (int i = 0; i < 8; ++i)
-          if (e + i < a.n) a.xhat[e + i] = out[i];
+          if (e + i < a.n) st_c(a.xhat + e + i, out[i]);
       }
     }
   }
@@ -381,14 +381,14 @@ __global__ void __launch_bounds__(256) decompress_unaligned_kernel(const CodecAr
   uint32_t u = 0;
   if (LAYOUT == kInterleaved) {
     const uint64_t bit = i * K;
-    u = (a.payload[bit >> 5] >> (bit & 31)) & ((1u << K) - 1);
+    u = (ldg_c(a.payload + (bit >> 5)) >> (bit & 31)) & ((1u << K) - 1);
   } else {
     const uint64_t w0 = (i >> 5) * K;
-    for (int j = 0; j < K; ++j) u |= ((a.payload[w0 + j] >> (i & 31)) & 1u) << j;
+    for (int j = 0; j < K; ++j) u |= ((ldg_c(a.payload + w0 + j) >> (i & 31)) & 1u) << j;
   }
   const uint64_t m = (a.chunk_shift >= 0) ? (i >> a.chunk_shift) : (i / a.chunk);
-  const float2 so = a.meta[m];
-  a.xhat[i] = dequantize_code<K, RANGE>(u, so.x, so.y);
+  const float2 so = ldg_c(a.meta + m);
+  st_c(a.xhat + i, dequantize_code<K, RANGE>(u, so.x, so.y));
 }
 
 }  // namespace accept

@@ -102,7 +102,7 @@ __device__ void mbq_build_table(const float* alpha_global, MbqTable<K>* t, float
   __shared__ float s_sorted[16];
   float alpha[K];
 #pragma unroll
-  for (int j = 0; j < K; ++j) alpha[j] = __ldg(alpha_global + j);
+  for (int j = 0; j < K; ++j) alpha[j] = ldg_c(alpha_global + j);
   if (tid < L) s_level[tid] = mbq_level<K>(alpha, tid);
   __syncthreads();
   if (tid < L) {
@@ -264,7 +264,7 @@ __device__ __forceinline__ void mbq_ld_octet(const float* x, uint64_t n, uint64_
     ld_octet(x + e, v);
   } else {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = (e + i < n) ? __ldg(x + e + i) : 0.0f;
+    for (int i = 0; i < 8; ++i) v[i] = (e + i < n) ? ldg_c(x + e + i) : 0.0f;
   }
 }
 
@@ -541,7 +541,7 @@ __device__ __forceinline__ void mbq_encode_tile(const MbqArgs& a, uint64_t tile,
     // after the quad transpose lane q holds the 32 signs of basis q of its group: counts of +1 and,
     // against the words of the other three lanes of the quad, counts of differing signs
     const uint32_t word = quad_transpose(mbq_planes_of_flags(f), lane);
-    if ((FULL || oct < n_oct_stored) && q < K) a.payload[(oct >> 2) * K + q] = word;
+    if ((FULL || oct < n_oct_stored) && q < K) st_c(a.payload + (oct >> 2) * K + q, word);
     sums.count += __popc(word);
 #pragma unroll
     for (int d = 1; d < 4; ++d) {
@@ -726,7 +726,7 @@ __global__ void __launch_bounds__(kMbqFinalizeThreads) mbq_finalize_kernel(const
     for (int j = 0; j < K; ++j) {
       G[j][j] = N;
       rhs[j] = s_val[j];
-      prev[j] = (double)__ldg(a.alpha_prev + j);
+      prev[j] = (double)ldg_c(a.alpha_prev + j);
     }
     bool singular = false;
     for (int col = 0; col < K && !singular; ++col) {
@@ -760,11 +760,11 @@ __global__ void __launch_bounds__(kMbqFinalizeThreads) mbq_finalize_kernel(const
   double acc = 0.0;
   for (int j = 0; j < K; ++j) acc += (double)alpha_next[j] * (2.0 * (double)c[j] - N);
   const float m_q = (float)((acc - sum_x) / N);
-  for (int i = 0; i < 8; ++i) a.header[i] = mbq_header_word(a, i);
-  for (int j = 0; j < K; ++j) { a.side[j] = alpha_next[j]; a.alpha_next[j] = alpha_next[j]; }
-  a.side[K] = m_q;
+  for (int i = 0; i < 8; ++i) st_c(a.header + i, mbq_header_word(a, i));
+  for (int j = 0; j < K; ++j) { st_c(a.side + j, alpha_next[j]); st_c(a.alpha_next + j, alpha_next[j]); }
+  st_c(a.side + K, m_q);
   // pad up to the payload
-  for (uint32_t* w = reinterpret_cast<uint32_t*>(a.side + K + 1); w < a.payload; ++w) *w = 0u;
+  for (uint32_t* w = reinterpret_cast<uint32_t*>(a.side + K + 1); w < a.payload; ++w) st_c(w, 0u);
 }
 
 // Receiver: planes -> codes -> level(c) - m_q.
@@ -777,8 +777,8 @@ __global__ void __launch_bounds__(256, 8) mbq_decode_kernel(const MbqArgs a) {
   if (tid < (1 << K)) {
     float alpha[K];
 #pragma unroll
-    for (int j = 0; j < K; ++j) alpha[j] = __ldg(a.side + j);
-    s_value[tid] = __fsub_rn(mbq_level<K>(alpha, tid), __ldg(a.side + K));
+    for (int j = 0; j < K; ++j) alpha[j] = ldg_c(a.side + j);
+    s_value[tid] = __fsub_rn(mbq_level<K>(alpha, tid), ldg_c(a.side + K));
   }
   __syncthreads();
   const uint64_t n_oct = (a.n + 7) / 8, n_groups = (a.n + 31) / 32;
@@ -788,7 +788,7 @@ __global__ void __launch_bounds__(256, 8) mbq_decode_kernel(const MbqArgs a) {
     const uint64_t oct = (uint64_t)blockIdx.x * 512 + r * 256 + tid;
     const uint64_t group = oct >> 2;
     uint32_t w = 0;
-    if (group < n_groups && q < K) w = __ldg(a.payload + group * K + q);
+    if (group < n_groups && q < K) w = ldg_c(a.payload + group * K + q);
     const uint32_t nib = planes_nibbles(quad_transpose(w, lane));
     if (oct < n_oct) {
       float out[8];
@@ -802,7 +802,7 @@ __global__ void __launch_bounds__(256, 8) mbq_decode_kernel(const MbqArgs a) {
         st_octet(a.xhat + e, out);
       } else {
         for (int i = 0; i < 8; ++i)
-          if (e + i < a.n) a.xhat[e + i] = out[i];
+          if (e + i < a.n) st_c(a.xhat + e + i, out[i]);
       }
     }
   }

@@ -28,6 +28,7 @@ __device__ __forceinline__ float from_sortable_key(uint32_t k) {
 
 template <int RANGE>
 __device__ __forceinline__ void merge_into_record(ChunkRecord* rec, float hi, float lo) {
+  if (!bounds_ok(rec, sizeof(ChunkRecord), true)) return;
   if (RANGE == kAbsMax) {
     atomicMax(&rec->a, __float_as_uint(hi));  // hi = max|x| >= 0 (or NaN): magnitude bits order as integers
   } else {
@@ -43,9 +44,9 @@ __device__ __forceinline__ void ld_octet_guarded(const CodecArgs& a, uint64_t oc
   if (e + 8 <= a.n) {
     ld_octet(a.x + e, v);
   } else {
-    const float fill = repeat_first ? __ldg(a.x + e) : 0.0f;
+    const float fill = repeat_first ? ldg_c(a.x + e) : 0.0f;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = (e + i < a.n) ? __ldg(a.x + e + i) : fill;
+    for (int i = 0; i < 8; ++i) v[i] = (e + i < a.n) ? ldg_c(a.x + e + i) : fill;
   }
 }
 
@@ -124,11 +125,12 @@ __global__ void __launch_bounds__(256) wide_finalize_kernel(const CodecArgs a, C
   const uint64_t m = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (m >= a.n_chunks) return;
   float hi, lo = 0.0f;
+  const ChunkRecord gathered = ld_c(rec + m);
   if (RANGE == kAbsMax) {
-    hi = __uint_as_float(rec[m].a);
+    hi = __uint_as_float(gathered.a);
   } else {
-    hi = from_sortable_key(rec[m].a);
-    lo = from_sortable_key(~rec[m].b);
+    hi = from_sortable_key(gathered.a);
+    lo = from_sortable_key(~gathered.b);
   }
   Scale sc;
   switch (a.k) {
@@ -137,19 +139,21 @@ __global__ void __launch_bounds__(256) wide_finalize_kernel(const CodecArgs a, C
     case 4: sc = make_scale<4, RANGE>(hi, lo); break;
     default: sc = make_scale<8, RANGE>(hi, lo); break;
   }
-  a.meta[m] = make_float2(sc.s, sc.o);
+  st_c(a.meta + m, make_float2(sc.s, sc.o));
   if (sc.nonfinite) atomicOr(a.status, kDevNonFinite);
-  rec[m].a = sc.nonfinite ? 1u : 0u;
-  rec[m].b = 0u;
-  rec[m].inv = sc.nonfinite ? -0.0f : sc.inv;
-  rec[m].base = sc.base;
+  ChunkRecord constants;
+  constants.a = sc.nonfinite ? 1u : 0u;
+  constants.b = 0u;
+  constants.inv = sc.nonfinite ? -0.0f : sc.inv;
+  constants.base = sc.base;
+  st_c(rec + m, constants);
 }
 
 // Pass 3: quantize + pack with the constants of each octet's chunk.  A tile that lies inside the
 // tensor and inside one chunk (all but the tiles on a chunk boundary and the last one) reads its
 // record once and skips the per-octet guards.
 __device__ __forceinline__ Scale scale_from_record(const ChunkRecord* rec) {
-  const uint4 raw = __ldg(reinterpret_cast<const uint4*>(rec));
+  const uint4 raw = ldg_c(reinterpret_cast<const uint4*>(rec));
   Scale sc;
   sc.s = 0.0f; sc.o = 0.0f;
   sc.inv = fabsf(__uint_as_float(raw.z));
@@ -163,8 +167,8 @@ __global__ void __launch_bounds__(256, R <= 2 ? 5 : 4) wide_encode_kernel(const 
   grid_dependency_handshake();
   const int tid = threadIdx.x, lane = tid & 31;
   if (blockIdx.x == 0 && tid < 8) {
-    a.header[tid] = header_word(a, tid);
-    if ((a.n_chunks & 1) && tid < 2) reinterpret_cast<uint32_t*>(a.meta + a.n_chunks)[tid] = 0u;
+    st_c(a.header + tid, header_word(a, tid));
+    if ((a.n_chunks & 1) && tid < 2) st_c(reinterpret_cast<uint32_t*>(a.meta + a.n_chunks) + tid, 0u);
   }
   const uint64_t n_oct_stored = ((a.n + 31) / 32) * 4;  // whole pack groups are stored
   const uint64_t tile_oct = (uint64_t)blockIdx.x * (R * 256);

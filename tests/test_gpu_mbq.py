@@ -10,6 +10,7 @@ import pytest
 
 import oracle
 import workloads
+from tests import gpu_util
 
 pytestmark = pytest.mark.gpu
 
@@ -24,14 +25,20 @@ def _A():
 def gpu_mbq_compress(x, k, t, init, alpha_prev):
     A = _A()
     p = A.MbqParams(x.size, k, t, init)
-    d_x = torch.from_numpy(x).cuda()
-    d_prev = None if alpha_prev is None else torch.from_numpy(np.asarray(alpha_prev, dtype=np.float32)).cuda()
-    d_next = torch.full((k,), float("nan"), dtype=torch.float32, device="cuda")
-    d_stream = A.new_stream_buffer(p)
-    d_stream.fill_(0x77)
-    d_ws = A.new_workspace(p)
-    A.accept_mbq_compress(p, d_x, d_prev, d_next, d_stream, d_ws)
+    g_x = gpu_util.guarded_input(torch, x)
+    g_prev = None if alpha_prev is None else gpu_util.guarded_input(torch, np.asarray(alpha_prev, dtype=np.float32))
+    g_next = gpu_util.guarded_floats(torch, k)
+    g_stream = gpu_util.guarded_stream(A, torch, p, 0x77)
+    g_ws = gpu_util.guarded_workspace(A, torch, p)
+    d_stream, d_ws, d_next = g_stream.bytes, g_ws.view(torch.int32), g_next.view(torch.float32)
+    A.accept_mbq_compress(p, g_x.view(torch.float32), None if g_prev is None else g_prev.view(torch.float32), d_next,
+                          d_stream, d_ws)
     status = A.accept_last_device_status(d_ws)
+    for g, what in ((g_x, "input"), (g_prev, "alpha_prev"), (g_next, "alpha_next"), (g_stream, "stream"), (g_ws, "workspace")):
+        if g is not None:
+            g.check(what)
+    # the call leaves everything but the status word and the residue coefficients of its workspace zeroed
+    assert not bool(d_ws.view(torch.uint8)[64:].any()), "exact sums not cleared"
     return p, d_stream, d_next.cpu().numpy(), status, d_ws
 
 
@@ -51,9 +58,11 @@ def check_mbq(x, k, t, init, alpha_prev):
     bad = np.nonzero(got[off:].view(np.uint32) != ref_stream[off:].view(np.uint32))[0]
     assert bad.size == 0, f"{bad.size} plane words differ, first {bad[:5]}"
     # receiver: the GPU decodes its own stream; the oracle decodes the same bytes
-    d_xhat = torch.full((x.size,), float("nan"), dtype=torch.float32, device="cuda")
+    g_xhat = gpu_util.guarded_floats(torch, x.size)
+    d_xhat = g_xhat.view(torch.float32)
     A.accept_mbq_decompress(p, d_stream, d_xhat, d_ws)
     assert A.accept_last_device_status(d_ws) == 0
+    g_xhat.check("reconstruction")
     want = oracle.mbq_decompress(got, x.size)
     assert np.array_equal(d_xhat.cpu().numpy().view(np.uint32), want.view(np.uint32))
     return alpha_next, side_g

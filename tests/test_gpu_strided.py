@@ -4,6 +4,7 @@ import pytest
 
 import oracle
 import workloads
+from tests import gpu_util
 from oracle import (LAYOUT_BITPLANE, LAYOUT_INTERLEAVED, RANGE_ABSMAX, RANGE_MINMAX, ROUND_NEAREST,
                     ROUND_STOCHASTIC)
 
@@ -28,11 +29,14 @@ def check(x, chunk, stride, k, range_, round_, layout, seed=0, rng_offset=0):
     ref, flag = oracle.compress_strided(x, chunk, k, stride, range_, round_, layout, seed, rng_offset)
     p = A.Params(n, chunk, k, range_, round_, layout, seed, rng_offset, group_stride=stride)
     assert A.accept_compressed_size(p) == ref.size
-    d_stream = A.new_stream_buffer(p)
-    d_stream.fill_(0x3C)
-    d_ws = A.new_workspace(p)
-    A.accept_compress(p, torch.from_numpy(x.reshape(-1)).cuda(), d_stream, d_ws)
+    g_x = gpu_util.guarded_input(torch, x)
+    g_stream = gpu_util.guarded_stream(A, torch, p, 0x3C)
+    g_ws = gpu_util.guarded_workspace(A, torch, p)
+    d_stream, d_ws = g_stream.bytes, g_ws.view(torch.int32)
+    A.accept_compress(p, g_x.view(torch.float32), d_stream, d_ws)
     assert (A.accept_last_device_status(d_ws) & 1) == flag
+    for g, what in ((g_x, "input"), (g_stream, "stream"), (g_ws, "workspace")):
+        g.check(what)
     got = d_stream.cpu().numpy()
     if not np.array_equal(got, ref):
         off = oracle.payload_offset(n, chunk)
@@ -40,9 +44,13 @@ def check(x, chunk, stride, k, range_, round_, layout, seed=0, rng_offset=0):
         assert np.array_equal(got[32:off], ref[32:off]), "side words"
         bad = np.nonzero(got[off:].view(np.uint32) != ref[off:].view(np.uint32))[0]
         raise AssertionError(f"{bad.size} payload words differ, first {bad[:8]}")
-    d_xhat = torch.full((n,), float("nan"), dtype=torch.float32, device="cuda")
-    A.accept_decompress(p, d_stream, d_xhat, d_ws)
-    assert A.accept_last_device_status(d_ws) == flag
+    g_xhat = gpu_util.guarded_floats(torch, n)
+    d_xhat = g_xhat.view(torch.float32)
+    g_ws16 = gpu_util.guarded_workspace(A, torch, p, 16)  # the receiver needs the status word only
+    A.accept_decompress(p, d_stream, d_xhat, g_ws16.view(torch.int32))
+    assert A.accept_last_device_status(g_ws16.view(torch.int32)) == 0
+    g_xhat.check("reconstruction")
+    g_ws16.check("receiver workspace")
     want = oracle.decompress_strided(ref, n)
     assert np.array_equal(d_xhat.cpu().numpy().view(np.uint32), want.view(np.uint32))
     assert A.accept_parse_header(bytes(got[:32])).group_stride == stride
