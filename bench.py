@@ -9,6 +9,12 @@ reported on their own, each with its achieved fraction of the measured HBM copy 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--sweep]
     python bench.py --impl reference ...      # the CPU oracle on the host cores
 
+The headline (`value`) is the round trip on --workload (cfg4_hidden by default): the median over --repeats
+blocks of exactly K back-to-back steps each.  On one GPU the line also carries, under "workloads", one
+row per tensor of 100 MB or more in its headline modes (cfg3 forward and backward, cfg4, the 256 MB and
+1 GB points of the size sweep) with both kernels timed inside the step and in loops of their own, and under
+"small" the tensors of 16 MB and less replayed from CUDA graphs next to an empty kernel launched the same way.
+
 With N > 1 (launched under torch.distributed.run) every rank codes its own replica of the tensor;
 the codec has no exchange step, so there is no data-path collective (weak scaling).
 """
@@ -45,6 +51,33 @@ def mode_name(m) -> str:
 def algorithmic_bytes(n: int, chunk: int, k: int) -> float:
     """Bytes the method must move per call, either direction: 4 + k/8 + 8/C per element."""
     return n * (4.0 + k / 8.0 + 8.0 / chunk)
+
+
+def kernel_sources_digest() -> str:
+    """Digest of the CUDA sources: ncu counters stored under profiles/ are quoted only for the kernels they
+    were taken from."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2311_05827_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        if name.endswith((".cu", ".cuh")):
+            with open(os.path.join(csrc, name), "rb") as f:
+                h.update(name.encode() + b"\0" + f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(workload: str, entry_point: str):
+    """DRAM bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum) from profiles/traffic.json, or
+    None when there is no capture of this kernel on this workload or the sources have changed since."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            table = json.load(f)
+        row = table["captures"][workload][entry_point]
+        if row["sources_digest"] != kernel_sources_digest():
+            return None
+        return float(row["dram_bytes_per_launch"])
+    except Exception:
+        return None
 
 
 def measured_peak():
@@ -169,6 +202,43 @@ class Codec:
         tc = sum(edge[i].elapsed_time(mid[i]) for i in range(steps)) / steps
         td = sum(mid[i].elapsed_time(edge[i + 1]) for i in range(steps)) / steps
         return total / steps, tc, td
+
+    def run_blocks(self, steps: int, repeats: int):
+        """`repeats` blocks of exactly `steps` back-to-back steps, one pair of events round each block:
+        -> ms per step of every block."""
+        torch = self.torch
+        out = []
+        for r in range(repeats):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(steps):
+                self.step(r * steps + i)
+            e1.record()
+            torch.cuda.synchronize()
+            out.append(e0.elapsed_time(e1) / steps)
+        return out
+
+    def run_isolated_blocks(self, steps: int, repeats: int, warmup: int = 3):
+        """Each kernel in loops of its own: -> (ms per compress of every block, ms per decompress of every block)."""
+        torch, A = self.torch, self.A
+        out = []
+        for fn in (lambda j: A.accept_compress(self.p, self.x[j], self.stream[j], self.ws),
+                   lambda j: A.accept_decompress(self.p, self.stream[j], self.xhat[j], self.ws)):
+            for i in range(warmup):
+                fn(i % self.copies)
+            torch.cuda.synchronize()
+            blocks = []
+            for r in range(repeats):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for i in range(steps):
+                    fn((r * steps + i) % self.copies)
+                e1.record()
+                torch.cuda.synchronize()
+                blocks.append(e0.elapsed_time(e1) / steps)
+            self.calls += warmup + steps * repeats
+            out.append(blocks)
+        return out[0], out[1]
 
     def run_isolated(self, steps: int, warmup: int = 3):
         """Each kernel in a loop of its own (rotating buffers): -> (ms per compress, ms per decompress).
@@ -333,6 +403,113 @@ def job_throughput(n_elems_per_rank: int, world: int, ms: float) -> float:
     return world * 4.0 * n_elems_per_rank / (ms * 1e-3) / 1e9
 
 
+def spread(values) -> dict:
+    v = sorted(float(t) for t in values)
+    return {"median": float(np.median(v)), "min": v[0], "max": v[-1], "blocks": len(v)}
+
+
+def generate_on_all_cores(name: str) -> np.ndarray:
+    """The whole tensor, its blocks drawn on one thread per host core (numpy's generators drop the interpreter lock)."""
+    from concurrent.futures import ThreadPoolExecutor
+    n, step = workloads.TENSORS[name].n, 1 << 22
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    with ThreadPoolExecutor(max_workers=max(1, cores)) as pool:
+        parts = list(pool.map(lambda s0: workloads.generate(name, s0, min(step, n - s0)), range(0, n, step)))
+    return np.concatenate(parts) if len(parts) > 1 else parts[0]
+
+
+def kernel_figures(n: int, alg: float, us_in_step: float, us_alone: dict, peak: float) -> dict:
+    """One kernel of a row: microseconds inside the step and in a loop of its own, GB/s of fp32, and the
+    algorithmic bytes over the time as a fraction of the measured copy bandwidth and of 8 TB/s."""
+    gbs = lambda nbytes, us: nbytes / (us * 1e-6) / 1e9
+    return {"us_in_step": us_in_step, "us_alone": us_alone,
+            "gbs_fp32_in_step": gbs(4 * n, us_in_step), "gbs_fp32_alone": gbs(4 * n, us_alone["median"]),
+            "frac_of_measured_in_step": gbs(alg, us_in_step) / peak, "frac_of_measured_alone": gbs(alg, us_alone["median"]) / peak,
+            "frac_of_8TBs_in_step": gbs(alg, us_in_step) / 8000.0, "frac_of_8TBs_alone": gbs(alg, us_alone["median"]) / 8000.0}
+
+
+def measure_row(A, torch, name: str, mode, x_host, steps: int, repeats: int, warmup: int, peak: float):
+    """compress + decompress of one tensor in one mode: `repeats` blocks of `steps` steps, then each kernel
+    between events inside the step, then each kernel in loops of its own.  -> (row, codec)."""
+    spec = workloads.TENSORS[name]
+    codec = Codec(A, torch, x_host, spec.chunk, mode, spec.seed)
+    for i in range(warmup):
+        codec.step(i)
+    torch.cuda.synchronize()
+    before = A.accept_launch_count()
+    step_ms = codec.run_blocks(steps, repeats)
+    launches = (A.accept_launch_count() - before) // repeats
+    _, ms_c, ms_d = codec.run(steps, 0)
+    iso_c, iso_d = codec.run_isolated_blocks(steps, repeats)
+    assert codec.status() == 0
+    alg = algorithmic_bytes(spec.n, spec.chunk, mode.k)
+    step_us = spread(1e3 * t for t in step_ms)
+    row = {"workload": name, "mode": mode_name(mode), "mbytes": spec.n * 4 / 2 ** 20, "buffer_sets": codec.copies,
+           "algorithmic_bytes_per_launch": alg, "step_us": step_us,
+           "step_gbs_fp32": 4 * spec.n / (step_us["median"] * 1e-6) / 1e9,
+           "step_frac_of_measured": 2 * alg / (step_us["median"] * 1e-6) / 1e9 / peak,
+           "step_frac_of_8TBs": 2 * alg / (step_us["median"] * 1e-6) / 1e9 / 8000.0,
+           "compress": kernel_figures(spec.n, alg, 1e3 * ms_c, spread(1e3 * t for t in iso_c), peak),
+           "decompress": kernel_figures(spec.n, alg, 1e3 * ms_d, spread(1e3 * t for t in iso_d), peak),
+           "launches_per_block": launches}
+    return row, codec
+
+
+def small_rows(A, torch, peak: float):
+    """Tensors of 16 MB and less: the time of a call is set by launching, not by bytes.  Each kernel is
+    replayed from a CUDA graph of 64 calls over rotating buffers (cold) next to an EMPTY kernel of the same
+    grid launched the same way (same launch attribute, same graph): the floor.  What is left above the
+    floor is set against the time the algorithmic bytes take at the measured copy bandwidth."""
+    rows = []
+    for name in ("cfg1_act", "cfg2_grad", "cfg5_64KB", "cfg5_1MB", "cfg5_16MB"):
+        spec = workloads.TENSORS[name]
+        x_host = workloads.generate(name)
+        for mode in spec.headline:
+            codec = Codec(A, torch, x_host, spec.chunk, mode, spec.seed)
+            g_c, g_d = codec.run_graphed()
+            blocks = -(-spec.n // 4096)
+            floor_c, floor_d = null_graph_ms(A, torch, blocks, 128), null_graph_ms(A, torch, blocks, 256)
+            alg = algorithmic_bytes(spec.n, spec.chunk, mode.k)
+            bytes_us = alg / peak / 1e3  # microseconds the bytes take at the measured copy bandwidth
+            rows.append({"workload": name, "mode": mode_name(mode), "kbytes": spec.n * 4 / 1024,
+                         "bytes_us_at_measured_copy": bytes_us,
+                         "compress_us_graph": 1e3 * g_c, "decompress_us_graph": 1e3 * g_d,
+                         "empty_kernel_us_graph": {"blocks": blocks, "threads_128": 1e3 * floor_c, "threads_256": 1e3 * floor_d},
+                         "compress_us_above_floor": 1e3 * (g_c - floor_c), "decompress_us_above_floor": 1e3 * (g_d - floor_d),
+                         "compress_frac_of_measured": bytes_us / (1e3 * g_c), "decompress_frac_of_measured": bytes_us / (1e3 * g_d)})
+            assert codec.status() == 0
+            del codec
+            torch.cuda.empty_cache()
+    return rows
+
+
+def null_graph_ms(A, torch, blocks: int, threads: int, launches: int = 64, replays: int = 10) -> float:
+    """ms per launch of the library's empty kernel, captured and replayed like Codec.run_graphed."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        A.accept_launch_null(blocks, threads, side)
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(launches):
+                A.accept_launch_null(blocks, threads, side)
+        graph.replay()
+        side.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(side)
+        for _ in range(replays):
+            graph.replay()
+        e1.record(side)
+        side.synchronize()
+    torch.cuda.current_stream().wait_stream(side)
+    return e0.elapsed_time(e1) / (replays * launches)
+
+
+# tensors of 100 MB or more besides the headline workload, each in its headline modes
+LARGE_ROWS = ("cfg3_act", "cfg3_grad", "cfg5_256MB", "cfg5_1GB")
+
+
 def run_gpu(args):
     import torch
     import paper_2311_05827_b200 as A
@@ -353,32 +530,44 @@ def run_gpu(args):
 
     spec = workloads.TENSORS[args.workload]
     mode = (spec.headline + spec.also)[args.mode_index]
-    x_host = workloads.generate(args.workload)
+    x_host = generate_on_all_cores(args.workload)
     n = spec.n
     peak, peak_src = measured_peak()
-
-    codec = Codec(A, torch, x_host, spec.chunk, mode, spec.seed)
-    launches0 = A.accept_launch_count()
-    sampler = ClockSampler(local_rank)
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(args.warmup):
-        codec.step(i)
+    sampler = ClockSampler(local_rank)
     barrier()
     sampler.start()
-    launches_before = A.accept_launch_count()
-    ms_step, ms_c, ms_d = codec.run(args.steps, 0)
-    launches_timed = (A.accept_launch_count() - launches_before) // 2  # the step pass; the per-kernel pass repeats it
+    head, codec = measure_row(A, torch, args.workload, mode, x_host, args.steps, args.repeats, args.warmup, peak)
     barrier()
-    iso_c, iso_d = codec.run_isolated(args.steps)
-    clocks = sampler.stop()
-    assert codec.status() == 0
+    # the slowest rank defines the job: per block, then the median over blocks
+    ms_step = max_over_ranks([head["step_us"]["median"] * 1e-3], dist, "cuda")[0]
+    ms_c, ms_d = max_over_ranks([head["compress"]["us_in_step"] * 1e-3, head["decompress"]["us_in_step"] * 1e-3], dist, "cuda")
+    iso_c, iso_d = max_over_ranks([head["compress"]["us_alone"]["median"] * 1e-3,
+                                   head["decompress"]["us_alone"]["median"] * 1e-3], dist, "cuda")
+    launches_timed = head["launches_per_block"]
 
-    ms_step, ms_c, ms_d, iso_c, iso_d = max_over_ranks([ms_step, ms_c, ms_d, iso_c, iso_d], dist, "cuda")
+    rows, small = [head], []
+    if world == 1 and not args.kernels_only and not args.headline_only:
+        for name in LARGE_ROWS:
+            if name == args.workload:
+                continue
+            xr = generate_on_all_cores(name)
+            for m in workloads.TENSORS[name].headline:
+                row, c = measure_row(A, torch, name, m, xr, args.steps, args.repeats, args.warmup, peak)
+                rows.append(row)
+                del c
+                torch.cuda.empty_cache()
+            del xr
+        small = small_rows(A, torch, peak)
+    clocks = sampler.stop()
+    if clocks.get("sm_mhz"):
+        for row in rows:
+            row["step_mcycles"] = row["step_us"]["median"] * clocks["sm_mhz"] * 1e-6  # time x median SM clock
 
     # end to end through host buffers
     e2e_steps = max(2, min(args.steps, 6))
@@ -398,27 +587,28 @@ def run_gpu(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "shape": list(spec.shape), "n_elems": n, "chunk": spec.chunk,
                    "mode": mode_name(mode), "l2": "inputs larger than L2 and %d rotating buffer sets" % codec.copies,
-                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "timing": "median of %d blocks of exactly %d back-to-back steps, CUDA events round each block" % (args.repeats, args.steps)},
+        "ms_per_step_blocks": {k: (v * 1e-3 if k != "blocks" else v) for k, v in head["step_us"].items()},
         "step_hbm": {"algorithmic_bytes": 2 * alg, "gbs": gbs(2 * alg, ms_step), "frac_of_measured_copy": gbs(2 * alg, ms_step) / peak,
                      "frac_of_8TBs": gbs(2 * alg, ms_step) / 8000.0},
-        "compress": {"ms_in_step": ms_c, "ms_alone": iso_c, "gbs_fp32_in": gbs(4 * n, iso_c), "hbm_gbs": gbs(alg, iso_c),
-                     "frac_of_measured_copy": gbs(alg, iso_c) / peak, "frac_of_8TBs": gbs(alg, iso_c) / 8000.0},
-        "decompress": {"ms_in_step": ms_d, "ms_alone": iso_d, "gbs_fp32_out": gbs(4 * n, iso_d), "hbm_gbs": gbs(alg, iso_d),
-                       "frac_of_measured_copy": gbs(alg, iso_d) / peak, "frac_of_8TBs": gbs(alg, iso_d) / 8000.0},
         "roofline": {"bound": "hbm", "kernel": dominant, "achieved": gbs(alg, ms_dom), "peak": peak, "peak_source": peak_src,
-                     "unit": "GB/s", "frac": gbs(alg, ms_dom) / peak, "traffic": TRAFFIC.get((args.workload, dominant)),
+                     "unit": "GB/s", "frac": gbs(alg, ms_dom) / peak, "traffic": recorded_traffic(args.workload, dominant),
                      # the same kernel in a loop of its own: inside a step it also pays for the write-back of the dirty
                      # lines its predecessor left in L2 (the step as a whole is in step_hbm)
                      "achieved_alone": gbs(alg, iso_c if dominant == "accept_compress" else iso_d),
                      "frac_alone": gbs(alg, iso_c if dominant == "accept_compress" else iso_d) / peak},
         "e2e": {"value": job_throughput(n, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "streams": 2},
+                "d2h_bytes_per_step": d2h, "streams": 2, "steps": e2e_steps},
         "gpu_launches": launches_timed,
         "clocks": clocks,
+        "workloads": rows,
     }
+    if small:
+        out["small"] = small
 
     if args.sweep and rank == 0:
-        out["workloads"] = sweep(A, torch, peak, args)
+        out["sweep"] = sweep(A, torch, peak, args)
 
     if rank == 0 and world == 1 and not (args.no_cpu_baseline or args.kernels_only):
         tc, td, reps = time_oracle(x_host, spec.chunk, mode, spec.seed, budget_s=args.cpu_budget)
@@ -435,10 +625,6 @@ def run_gpu(args):
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(out))
-
-
-# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch, filled from profiles/ once captured
-TRAFFIC = {("cfg4_hidden", "accept_compress"): 318.96e6, ("cfg4_hidden", "accept_decompress"): 277.38e6}
 
 
 def sweep(A, torch, peak, args):
@@ -613,6 +799,8 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--repeats", type=int, default=10, help="blocks of --steps steps; the headline is their median")
+    ap.add_argument("--headline-only", action="store_true", help="skip the rows of the other workloads")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(workloads.TENSORS))

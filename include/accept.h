@@ -238,7 +238,7 @@ accept_status accept_decompress_host(const accept_params* p, const void* h_strea
  * floats (they may be the same array), so successive batches chain without a host round trip.
  * The workspace (accept_mbq_workspace_size bytes = 624, 16-byte aligned, zeroed once by the caller) holds
  * the status word, the residue coefficients and the exact sums (every call leaves them zeroed again; a
- * workspace serves one call at a time).  Launches: 2 (plus k when init).  The encode
+ * workspace serves one call at a time).  Launches: 1 (plus k when init).  The encode
  * kernel of a batch >= 1 asks for 128 KB of dynamic shared memory per block (its search table).
  */
 typedef struct {
@@ -281,6 +281,15 @@ int accept_bitwidth_schedule(int is_backward, int n_lr_changes);
 
 /* Number of kernels the library has launched in this process (all entry points). */
 uint64_t accept_launch_count(void);
+
+/*
+ * Launches an EMPTY kernel of `blocks` blocks of `threads` threads on cuda_stream exactly as every kernel of
+ * this library is launched (same launch attribute, same first instructions).  It measures what a launch
+ * costs where a call is bound by launching rather than by bytes (tensors of a few MB): replayed from a
+ * CUDA graph beside the codec's own kernels it gives the floor under their times.  The paper has no
+ * counterpart.  blocks in [1, 2^31), threads in [32, 1024].
+ */
+accept_status accept_launch_null(uint32_t blocks, uint32_t threads, void* cuda_stream);
 
 /*
  * For the checking build of this library (the same sources compiled with -DACCEPT_BOUNDS_CHECK, which the

@@ -32,7 +32,7 @@ EXPORTS = [
     "accept_check_params", "accept_compressed_size", "accept_payload_offset", "accept_workspace_size",
     "accept_compress", "accept_decompress", "accept_compress_host", "accept_decompress_host",
     "accept_last_device_status", "accept_parse_header", "accept_bitwidth_schedule", "accept_launch_count",
-    "accept_compress_static", "accept_bounds_check_report",
+    "accept_compress_static", "accept_bounds_check_report", "accept_launch_null",
     "accept_mbq_check_params", "accept_mbq_compressed_size", "accept_mbq_payload_offset", "accept_mbq_workspace_size",
     "accept_mbq_compress", "accept_mbq_decompress",
 ]
@@ -140,6 +140,8 @@ def load(path: str) -> ctypes.CDLL:
     L.accept_mbq_decompress.argtypes = [MP, vp, sz, vp, vp, sz, vp]
     L.accept_launch_count.restype = u64
     L.accept_launch_count.argtypes = []
+    L.accept_launch_null.restype = ctypes.c_int
+    L.accept_launch_null.argtypes = [ctypes.c_uint32, ctypes.c_uint32, vp]
     L.accept_bounds_check_report.restype = ctypes.c_int
     L.accept_bounds_check_report.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), ctypes.POINTER(u64), ctypes.POINTER(u64)]
     return L
@@ -228,6 +230,10 @@ def accept_decompress_host(p: Params, h_stream, h_xhat, d_stream, d_xhat, d_ws, 
                                         d_stream.data_ptr(), d_xhat.data_ptr(), d_ws.data_ptr(),
                                         d_ws.numel() * d_ws.element_size(), _stream_handle(stream)),
            "accept_decompress_host")
+
+
+def accept_launch_null(blocks: int, threads: int, stream=None) -> None:
+    _check(lib().accept_launch_null(blocks, threads, _stream_handle(stream)), "accept_launch_null")
 
 
 def accept_bounds_check_report(stream=None):

@@ -336,8 +336,9 @@ accept_status launch_strided(const accept_params* p, const CodecArgs& a, uint8_t
 
 uint64_t mbq_tiles(const accept_mbq_params* p) { return (p->n_elems + accept::kMbqTile - 1) / accept::kMbqTile; }
 
+// blocks of the encode pass: one per tile of 256 groups, at most two per SM of a B200 (the blocks are persistent)
 uint32_t mbq_blocks(const accept_mbq_params* p) {
-  const uint64_t tiles = mbq_tiles(p);
+  const uint64_t tiles = (p->n_elems + accept::kMbqGroupTile - 1) / accept::kMbqGroupTile;
   return (uint32_t)(tiles < (uint64_t)accept::kMbqMaxBlocks ? tiles : (uint64_t)accept::kMbqMaxBlocks);
 }
 
@@ -367,20 +368,22 @@ accept::MbqArgs mbq_args(const accept_mbq_params* p, void* d_stream, void* d_ws)
 
 template <int K>
 accept_status launch_mbq_compress(const accept::MbqArgs& a, cudaStream_t s) {
-  const dim3 grid((a.n_blocks + accept::kMbqGroups - 1) / accept::kMbqGroups);
+  const dim3 grid(a.n_blocks);
+  // the search grid and the staged tiles need more dynamic shared memory than a kernel gets without opting in
+  // (the attribute is per device: set every time)
   if (a.init) {
     for (int j = 0; j < K; ++j)
       ACCEPT_LAUNCH(launch_overlapped(accept::mbq_residue_sum_kernel<K>, dim3(a.n_residue_blocks), 256, s, a, j));
-    ACCEPT_LAUNCH(launch_overlapped(accept::mbq_encode_kernel<K, true>, grid, accept::kMbqEncodeThreads, s, a));
-  } else {
-    // the search grid needs more dynamic shared memory than a kernel gets without opting in (the
-    // attribute is per device: set every time)
-    auto fn = accept::mbq_encode_kernel<K, false>;
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, accept::kMbqGridBytes) != cudaSuccess)
+    auto fn = accept::mbq_encode_kernel<K, true>;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, accept::kMbqEncodeSmemBytes) != cudaSuccess)
       return ACCEPT_ERR_CUDA;
-    ACCEPT_LAUNCH(launch_overlapped_shared(fn, grid, accept::kMbqEncodeThreads, accept::kMbqGridBytes, s, a));
+    ACCEPT_LAUNCH(launch_overlapped_shared(fn, grid, accept::kMbqEncodeThreads, accept::kMbqEncodeSmemBytes, s, a));
+  } else {
+    auto fn = accept::mbq_encode_kernel<K, false>;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, accept::kMbqEncodeSmemBytes) != cudaSuccess)
+      return ACCEPT_ERR_CUDA;
+    ACCEPT_LAUNCH(launch_overlapped_shared(fn, grid, accept::kMbqEncodeThreads, accept::kMbqEncodeSmemBytes, s, a));
   }
-  ACCEPT_LAUNCH(launch_overlapped(accept::mbq_finalize_kernel<K>, dim3(1), accept::kMbqFinalizeThreads, s, a));
   return ACCEPT_OK;
 }
 
@@ -663,6 +666,12 @@ accept_status accept_mbq_decompress(const accept_mbq_params* p, const void* d_st
 }
 
 uint64_t accept_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+accept_status accept_launch_null(uint32_t blocks, uint32_t threads, void* cuda_stream) {
+  if (blocks == 0 || blocks > 0x7fffffffu || threads < 32 || threads > 1024) return ACCEPT_ERR_BAD_SIZE;
+  ACCEPT_LAUNCH(launch_overlapped(accept::null_kernel, dim3(blocks), threads, static_cast<cudaStream_t>(cuda_stream)));
+  return ACCEPT_OK;
+}
 
 accept_status accept_bounds_check_report(void* cuda_stream, uint32_t* violations, uint64_t* first_address,
                                          uint64_t* first_size_and_kind) {

@@ -49,34 +49,40 @@ struct ExactWindow {
 // Window for data whose magnitudes are expected around `scale` (any value; 0, NaN and Inf fall back to 1):
 // the top is 2^9 times the binade of scale, the bottom 2^24 below that.
 __device__ inline ExactWindow make_window(float scale) {
+  // binade of the scale from its exponent field (subnormal scales count as 2^-126)
   int e = 0;
-  if (scale > 0.0f && is_finite_bits(scale)) e = ilogbf(scale);
+  if (scale > 0.0f && is_finite_bits(scale)) {
+    const int field = (int)((__float_as_uint(scale) >> 23) & 0xFFu);
+    e = (field ? field : 1) - 127;
+  }
   int e_top = e + 9;
   if (e_top > 127) e_top = 127;
   if (e_top < -126 + 24) e_top = -126 + 24;  // keeps the bottom a normal number
   const int q = e_top - kWindowTopBits;
   ExactWindow w;
-  w.top = ldexpf(1.0f, e_top);
-  const float bottom = ldexpf(1.0f, e_top - 24);
-  w.top_bits = __float_as_uint(w.top);
-  w.bottom_bits = __float_as_uint(bottom);
+  w.top_bits = (uint32_t)(e_top + 127) << 23;          // 2^e_top
+  w.bottom_bits = (uint32_t)(e_top - 24 + 127) << 23;  // 2^(e_top - 24)
+  w.top = __uint_as_float(w.top_bits);
   w.ylow = 2u * w.bottom_bits - 2u;
   w.pos = q + 149;
-  w.to_units = ldexp(1.0, -q);
+  w.to_units = __hiloint2double((1023 - q) << 20, 0);  // 2^-q
   return w;
 }
 
-// Are all values seen so far inside the window (or zero)?  Per pair of values: one 3-input maximum of the
-// magnitudes (NaN survives, and then fails the comparison with the top) and one 3-input unsigned minimum
-// of y = 2 * bits - 2, which drops the sign, sends zero to the largest numbers and keeps the order of
-// all other magnitudes, so that "no non-zero value below the bottom" is one comparison at the end.
+// 2 * v - 2 (mod 2^32) as one integer multiply-add, which the FMA pipe takes (the ALU pipe is the busy one)
+__device__ __forceinline__ uint32_t twice_minus_two(uint32_t v) {
+  uint32_t r;
+  asm("mad.lo.u32 %0, %1, 2, 0xFFFFFFFE;" : "=r"(r) : "r"(v));
+  return r;
+}
+
 struct WindowCheck {
   float amax;
   uint32_t ymin;
   __device__ __forceinline__ void init() { amax = 0.0f; ymin = 0xFFFFFFFFu; }
   __device__ __forceinline__ void add2(float a, float b) {
     amax = max3_nan(amax, fabsf(a), fabsf(b));
-    ymin = __vimin3_u32(ymin, 2u * __float_as_uint(a) - 2u, 2u * __float_as_uint(b) - 2u);
+    ymin = __vimin3_u32(ymin, twice_minus_two(__float_as_uint(a)), twice_minus_two(__float_as_uint(b)));
   }
   __device__ __forceinline__ bool ok(const ExactWindow& w) const { return amax < w.top && ymin >= w.ylow; }
 };
@@ -126,8 +132,9 @@ __device__ __forceinline__ long long warp_sum_int64(long long v) {
 }
 
 // Carries propagated: digits 0..kAccLimbs-2 end in [0, 2^32), the last one keeps the sign.
-__device__ inline void wide_normalise(long long (&limbs)[kAccLimbs]) {
+__device__ __forceinline__ void wide_normalise(long long (&limbs)[kAccLimbs]) {
   long long carry = 0;
+#pragma unroll
   for (int i = 0; i < kAccLimbs - 1; ++i) {
     const long long t = limbs[i] + carry;
     limbs[i] = (long long)((uint64_t)t & 0xFFFFFFFFull);
@@ -137,15 +144,18 @@ __device__ inline void wide_normalise(long long (&limbs)[kAccLimbs]) {
 }
 
 // The wide sum (digits with pending carries) rounded to the nearest double, ties to even.
-__device__ inline double wide_to_double(const long long* lazy) {
+// d: scratch of kAccLimbs + 1 words that may be indexed by a variable: give it shared memory (an array of
+// the thread's own would live in local memory, whose misses cost microseconds in a block that runs alone).
+__device__ inline double wide_to_double(const long long* lazy, uint32_t* d) {
   long long limbs[kAccLimbs];
+#pragma unroll
   for (int i = 0; i < kAccLimbs; ++i) limbs[i] = lazy[i];
   wide_normalise(limbs);
   const bool negative = limbs[kAccLimbs - 1] < 0;
-  uint32_t d[kAccLimbs + 1];
   if (negative) {
     // magnitude of a two's complement number: complement every digit, add one
     uint64_t carry = 1;
+#pragma unroll
     for (int i = 0; i < kAccLimbs - 1; ++i) {
       const uint64_t t = (uint64_t)(~(uint32_t)limbs[i]) + carry;
       d[i] = (uint32_t)t;
@@ -153,6 +163,7 @@ __device__ inline double wide_to_double(const long long* lazy) {
     }
     d[kAccLimbs - 1] = (uint32_t)((uint64_t)(~limbs[kAccLimbs - 1]) + carry);
   } else {
+#pragma unroll
     for (int i = 0; i < kAccLimbs; ++i) d[i] = (uint32_t)limbs[i];
   }
   d[kAccLimbs] = 0u;

@@ -51,6 +51,9 @@ __device__ __forceinline__ void grid_dependency_handshake() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// Nothing but the handshake every kernel starts with: what a launch of this library costs (accept_launch_null).
+__global__ void null_kernel() { grid_dependency_handshake(); }
+
 constexpr int kFastBlock = 128;     // threads per block when a chunk needs at most 128 threads (finer tail than 256: measured)
 constexpr int kGenericBlock = 256;  // threads per block of the any-shape path
 

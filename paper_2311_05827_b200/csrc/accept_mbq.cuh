@@ -13,31 +13,42 @@
 // applies the moving average and writes the side words.  Nothing depends on the order in which
 // threads or blocks add, so the side words are a function of the input alone.
 #pragma once
+#include "accept_async.cuh"
 #include "accept_exact.cuh"
 #include "accept_kernels.cuh"
 
 namespace accept {
 
-constexpr int kMbqRounds = 2;                      // octets per thread and tile
-constexpr int kMbqTile = kMbqRounds * 256 * 8;     // elements per tile
-constexpr int kMbqFinalizeThreads = 32;            // threads of the single finalize block
-constexpr int kMbqGroups = 2;                      // 256-thread groups per block of the encode pass (one block per SM);
-                                                   // 3 groups at 80 registers were slower than 2 at 113 (measured)
-constexpr int kMbqEncodeThreads = 256 * kMbqGroups;
-constexpr int kMbqMaxBlocks = 148 * kMbqGroups;    // groups of the encode pass
+constexpr int kMbqRounds = 2;                      // octets per thread and tile of a residue pass
+constexpr int kMbqTile = kMbqRounds * 256 * 8;     // elements per tile of a residue pass
 constexpr int kMbqResidueBlocks = 1184;            // blocks of a residue pass
-constexpr int kMbqCells = 256;                     // cells of the uniform search grid
-constexpr int kMbqGridBytes = kMbqCells * 32 * 16; // one 16-byte entry per cell and lane
 constexpr int kMbqSums = 5;                        // wide sums in the workspace: basis 0..3, then the sum of x
-constexpr int kMbqFlushTiles = kFlushElems / (kMbqRounds * 8);  // tiles a thread codes between two flushes
+constexpr int kMbqFlushTiles = kFlushElems / (kMbqRounds * 8);  // tiles a thread of a residue pass adds between two flushes
+
+// Encode pass: persistent blocks of 256 threads, two per SM.  A thread owns one pack group (32 consecutive
+// values, 128 bytes) of each tile; tiles of 256 groups (32 KB) are staged in shared memory with
+// asynchronous bulk copies, two stages per block, so a block always has its next tile in flight.
+constexpr int kMbqEncodeThreads = 256;
+constexpr int kMbqBlocksPerSm = 2;
+constexpr int kMbqMaxBlocks = 148 * kMbqBlocksPerSm;
+constexpr int kMbqGroupTile = kMbqEncodeThreads * 32;        // elements per tile of the encode pass
+constexpr int kMbqTileBytes = kMbqGroupTile * 4;
+constexpr int kMbqStages = 2;
+constexpr int kMbqCopyBytes = 8192;                          // one bulk copy; a tile is four of them
+constexpr int kMbqCells = 256;                               // cells of the uniform search grid
+constexpr int kMbqColumns = 8;                               // copies of the grid: one per lane of a quarter warp
+constexpr int kMbqGridBytes = kMbqCells * kMbqColumns * 16;  // one 16-byte entry per cell and column: 32 KB
+constexpr int kMbqEncodeSmemBytes = kMbqGridBytes + kMbqStages * kMbqTileBytes;
+constexpr int kMbqFlushGroups = kFlushElems / 32;            // groups a thread codes between two flushes
 
 // Workspace of the forward quantizer (zeroed once by the caller; every call leaves the sums zeroed again).
 struct MbqWorkspace {
   uint32_t status;
   uint32_t pad0[3];
   float alpha_init[4];            // coefficients found by the residue passes (init)
-  uint32_t blocks_done;           // blocks of a residue pass that have delivered their sum
-  uint32_t pad1[7];
+  uint32_t blocks_done;           // blocks of the running pass that have delivered their sums
+  uint32_t next_tile;             // encode pass: tiles handed out beyond every block's first two
+  uint32_t pad1[6];
   long long wide[kMbqSums][kAccLimbs];  // exact sums, see accept_exact.cuh
   unsigned long long count[4];    // number of +1 per basis
   unsigned long long differ[6];   // pairs (0,1) (0,2) (0,3) (1,2) (1,3) (2,3): elements whose two signs differ
@@ -168,7 +179,7 @@ __device__ __forceinline__ uint32_t mbq_planes_of_flags(const uint32_t (&f)[8]) 
 }
 
 // Nearest level through a uniform grid.  The span of the levels (with a margin) is cut into 256
-// cells; cell_offset() is a non-decreasing function of x, so every x of a cell below the cell of a
+// cells; mbq_cell() is a non-decreasing function of x, so every x of a cell below the cell of a
 // threshold lies below that threshold and every x of a cell above it lies above.  When no cell
 // holds more than one threshold, one comparison with "the threshold inside my cell" finishes the
 // search: entry = {that threshold (+inf if the cell has none), flag bytes of the code below it,
@@ -176,23 +187,24 @@ __device__ __forceinline__ uint32_t mbq_planes_of_flags(const uint32_t (&f)[8]) 
 // when two thresholds share a cell (coinciding or very close levels), or a level is not finite,
 // the grid is marked unusable and the kernel searches the sorted thresholds instead.
 //
-// The table is stored once per lane, entry (cell, lane) at byte 512 * cell + 16 * lane: whatever
-// cells the 32 lanes of a warp ask for, lane l only ever touches its own 16-byte column of the
-// banks, so a lookup is one 128-bit shared load without bank conflicts (a single shared copy
-// cost 8.6 wavefronts per load on post-ReLU data and bound the pass).  128 KB per block.
+// The grid is stored eight times, entry (cell, column) at byte 128 * cell + 16 * column, and lane l
+// reads column l & 7: a 128-bit shared load is served a quarter warp at a time, and the eight lanes of a
+// quarter warp then touch eight different 16-byte columns of the banks whatever cells they ask for: no
+// bank conflicts (a single copy cost 8.6 wavefronts per load on post-ReLU data).  32 KB per block.
 struct MbqGridInfo {
-  float scale;  // 1 / (2 * span)
+  float scale;  // 1 / (2 * 1.03125 * largest |level|)
   int usable;
 };
 
-// Byte offset of entry (cell of x, lane); lane_bytes = 16 * lane.  Two fused multiply-adds on the
-// FMA pipe and one logic operation: the first maps the span onto [0, 1] and saturates, the second
-// leaves round(255 * 512 * t) in the low mantissa bits; keeping bits 9..16 of it gives
-// 512 * floor(that / 512).  NaN goes to cell 0.
-__device__ __forceinline__ uint32_t mbq_cell_offset(float x, float scale, uint32_t lane_bytes) {
+// Byte offset of the cell of x inside a column of the grid (128 * cell, cell = 0 .. 255).  Two fused
+// multiply-adds on the FMA pipe and one logic operation: the first maps the span onto [0, 1] and saturates
+// (NaN goes to 0), the second leaves round(255 * 128 * t) in the low mantissa bits; keeping bits 7..14 of it
+// gives 128 * floor(that / 128).  Non-decreasing in x.  (A float-to-integer conversion would do the same in
+// one instruction less, but it runs on the conversion unit, which this kernel already keeps busy: measured.)
+__device__ __forceinline__ uint32_t mbq_cell_offset(float x, float scale) {
   float t;
   asm("fma.rn.sat.f32 %0, %1, %2, 0f3F000000;" : "=f"(t) : "f"(x), "f"(scale));
-  return (__float_as_uint(__fmaf_rn(t, 130560.0f, kMagic)) & 0x1FE00u) | lane_bytes;
+  return __float_as_uint(__fmaf_rn(t, 32640.0f, kMagic)) & 0x7F80u;
 }
 
 // Called by all threads of the block.
@@ -214,7 +226,7 @@ __device__ void mbq_build_grid(const MbqTable<K>& t, const float* s_level, MbqGr
     info->usable = (finite && amax > 0.0f && is_finite_bits(scale)) ? 1 : 0;
   }
   __syncthreads();
-  if (tid >= 1 && tid < L) s_cell_of[tid] = mbq_cell_offset(t.thr[tid], info->scale, 0u) >> 9;
+  if (tid >= 1 && tid < L) s_cell_of[tid] = mbq_cell_offset(t.thr[tid], info->scale) >> 7;
   __syncthreads();
   if (tid < kMbqCells) {
     int below = 0, inside = 0;
@@ -230,14 +242,15 @@ __device__ void mbq_build_grid(const MbqTable<K>& t, const float* s_level, MbqGr
   }
   __syncthreads();
   if (info->usable)
-    for (int i = tid; i < kMbqCells * 32; i += n_threads) cells[i] = s_entry[i >> 5];
+    for (int i = tid; i < kMbqCells * kMbqColumns; i += n_threads) cells[i] = s_entry[i / kMbqColumns];
   __syncthreads();
 }
 
-// flag bytes of the nearest level's code
-__device__ __forceinline__ uint32_t mbq_grid_flags(const uint4* cells, float scale, uint32_t lane_bytes, float x) {
-  const uint4 e = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(cells) +
-                                                  mbq_cell_offset(x, scale, lane_bytes));
+// flag bytes of the nearest level's code; column = this lane's copy of the grid (byte address in shared memory)
+__device__ __forceinline__ uint32_t mbq_grid_flags(uint32_t column, float scale, float x) {
+  uint4 e;
+  const uint32_t addr = mbq_cell_offset(x, scale) + column;
+  asm("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(e.x), "=r"(e.y), "=r"(e.z), "=r"(e.w) : "r"(addr));
   return (x > __uint_as_float(e.x)) ? e.z : e.y;
 }
 
@@ -295,9 +308,11 @@ __device__ inline void mbq_block_sums_deliver(MbqBlockSums* bs, MbqWorkspace* ws
   if (tid >= kMbqSums) return;
   long long limbs[kAccLimbs];
   bool any = false;
+#pragma unroll
   for (int i = 0; i < kAccLimbs; ++i) { limbs[i] = bs->wide[tid][i]; any = any || limbs[i] != 0; }
   if (!any) return;
   wide_normalise(limbs);
+#pragma unroll
   for (int i = 0; i < kAccLimbs; ++i)
     if (limbs[i] != 0) limb_add(&ws->wide[tid][i], limbs[i]);
 }
@@ -406,10 +421,12 @@ __global__ void __launch_bounds__(256) mbq_residue_sum_kernel(const MbqArgs a, i
   if (s_is_last && tid == 0) {
     __threadfence();
     long long total[kAccLimbs];
+#pragma unroll
     for (int i = 0; i < kAccLimbs; ++i) {
       total[i] = (long long)atomicExch(reinterpret_cast<unsigned long long*>(&a.ws->wide[SLOT][i]), 0ull);
     }
-    a.ws->alpha_init[j] = (float)(wide_to_double(total) / (double)a.n);
+    // (the block's own wide sums have been delivered: their storage serves as scratch)
+    a.ws->alpha_init[j] = (float)(wide_to_double(total, reinterpret_cast<uint32_t*>(&s_sums.wide[0][0])) / (double)a.n);
     a.ws->blocks_done = 0u;
   }
 }
@@ -417,14 +434,23 @@ __global__ void __launch_bounds__(256) mbq_residue_sum_kernel(const MbqArgs a, i
 // How the signs of an element are found.
 constexpr int kMbqResidue = 0, kMbqSearch = 1, kMbqGrid = 2;
 
-// Running sums of one thread over all its tiles.  plus[] and sum_x hold what the thread added since its
+// Running sums of one thread over all its groups.  plus[] and sum_x hold what the thread added since its
 // last flush (plus[] times 2^-767, the flag factor); irun[] the flushed part in units of the window.
 template <int K>
 struct MbqSums {
   double plus[K], sum_x;
-  long long irun[K + 1];      // [K]: the sum of x
-  uint32_t count, differ[3];  // of basis q = lane & 3, and of the pairs (q, q ^ d)
-  int since, flushes;
+  long long irun[K + 1];   // [K]: the sum of x
+  uint32_t count[K];       // +1 signs per basis
+  uint32_t differ[6];      // pairs (0,1) (0,2) (0,3) (1,2) (1,3) (2,3): elements whose two signs differ
+  __device__ __forceinline__ void clear() {
+    sum_x = 0.0;
+#pragma unroll
+    for (int j = 0; j < K; ++j) { plus[j] = 0.0; count[j] = 0; }
+#pragma unroll
+    for (int j = 0; j <= K; ++j) irun[j] = 0;
+#pragma unroll
+    for (int d = 0; d < 6; ++d) differ[d] = 0;
+  }
 };
 
 // Accumulators -> integer units of the window, exactly (see accept_exact.cuh).
@@ -453,318 +479,484 @@ __device__ __forceinline__ void mbq_push(MbqSums<K>& s, MbqBlockSums* bs, int la
   }
 }
 
-// The octets of thread tid of a tile: FULL = every element of the tile exists.
-template <bool FULL>
-__device__ __forceinline__ void mbq_load_tile(const MbqArgs& a, uint64_t tile, int tid, float (&v)[kMbqRounds][8]) {
-  const uint64_t oct0 = tile * (kMbqRounds * 256) + tid;
+// What a thread needs to find the signs of a value.
+template <int K>
+struct MbqLookup {
+  const MbqTable<K>* table;  // sorted thresholds (kMbqSearch)
+  uint32_t column;           // shared-memory byte address of this lane's column of the grid (kMbqGrid)
+  float scale;               // of the grid
+  float alpha[K];            // coefficients of the residue method (kMbqResidue)
+};
+
+template <int K, int MODE>
+__device__ __forceinline__ uint32_t mbq_flags_of_value(const MbqLookup<K>& lk, float x) {
+  if (MODE == kMbqGrid) return mbq_grid_flags(lk.column, lk.scale, x);
+  if (MODE == kMbqSearch) return mbq_flags_of_code(mbq_nearest_code<K>(*lk.table, x));
+  float res;
+  return mbq_flags_of_code(mbq_residue_code<K>(lk.alpha, x, K, &res));
+}
+
+// x into the thread's accumulators: the sum of x, and the sum of every basis whose flag byte is set.
+template <int K>
+__device__ __forceinline__ void mbq_accumulate(MbqSums<K>& sums, float x, uint32_t flags) {
+  const double xd = (double)x;
+  sums.sum_x += xd;
+  mbq_add_flagged<0>(sums.plus[0], xd, flags);
+  mbq_add_flagged<1>(sums.plus[1], xd, flags);
+  if constexpr (K > 2) mbq_add_flagged<2>(sums.plus[2], xd, flags);
+  if constexpr (K > 3) mbq_add_flagged<3>(sums.plus[3], xd, flags);
+}
+
+// Four values of a group whose 32 values all lie inside the window: their signs, their share of the
+// sums; returns the signs as a word whose byte j holds, in its bits 4..7, basis j of the four values.
+template <int K, int MODE>
+__device__ __forceinline__ uint32_t mbq_code_four(const MbqLookup<K>& lk, const float4 v, MbqSums<K>& sums) {
+  const float w[4] = {v.x, v.y, v.z, v.w};
+  uint32_t f[4];
 #pragma unroll
-  for (int r = 0; r < kMbqRounds; ++r) {
-    const uint64_t oct = oct0 + r * 256;
-    if (FULL) {
-      ld_octet(a.x + oct * 8, v[r]);
-    } else if (oct < (a.n + 7) / 8) {
-      mbq_ld_octet(a.x, a.n, oct, v[r]);
+  for (int e = 0; e < 4; ++e) f[e] = mbq_flags_of_value<K, MODE>(lk, w[e]);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) mbq_accumulate<K>(sums, w[e], f[e]);
+  return f[0] + 2u * f[1] + 4u * f[2] + 8u * f[3];
+}
+
+// One value of a group that holds values outside the window, or fewer than 32 values (the ragged end of
+// the tensor): its signs are returned, and the value goes into the block's wide sums (the sum of x, and
+// the sum of every basis whose sign is +1) instead of the thread's accumulators -- exact wherever it lies.
+// Rare: kept out of line, and everything is passed by value so that the caller's state stays in registers.
+template <int K, int MODE>
+__device__ __noinline__ uint32_t mbq_code_value_slowly(MbqLookup<K> lk, float x, MbqBlockSums* bs, uint32_t* status) {
+  const uint32_t f = mbq_flags_of_value<K, MODE>(lk, x);
+  // flag bytes (0x10 per basis) -> slot bits, plus the slot of the sum of x
+  const uint32_t slots = ((((f >> 4) * 0x00204081u) >> 21) & 0xFu) | (1u << (kMbqSums - 1));
+  mbq_wide_add_value(bs, status, x, slots);
+  return f;
+}
+
+// The eight sign words of a group (slot c: bits 4..7 of byte j = basis j of values 4c..4c+3) -> the K plane
+// words of the group (bit t of word j = basis j of value t), counted and stored.
+template <int K>
+__device__ __forceinline__ void mbq_finish_group(const MbqArgs& a, const uint32_t (&s4)[8], uint32_t rotate_bits,
+                                                 uint64_t group, bool store, MbqSums<K>& sums) {
+  // pairs of slots: byte j = basis j of eight values
+  uint32_t b[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) b[i] = (s4[2 * i] >> 4) | s4[2 * i + 1];
+  // 4 x 4 byte transpose: word j = basis j of all 32 values, in the order of the slots
+  const uint32_t t0 = __byte_perm(b[0], b[1], 0x5140), t1 = __byte_perm(b[2], b[3], 0x5140);
+  const uint32_t t2 = __byte_perm(b[0], b[1], 0x7362), t3 = __byte_perm(b[2], b[3], 0x7362);
+  uint32_t word[4];
+  word[0] = __byte_perm(t0, t1, 0x5410);
+  word[1] = __byte_perm(t0, t1, 0x7632);
+  word[2] = __byte_perm(t2, t3, 0x5410);
+  word[3] = __byte_perm(t2, t3, 0x7632);
+  // the slots were read in an order rotated by the lane (bank conflicts): turn the words back
+#pragma unroll
+  for (int j = 0; j < K; ++j) word[j] = __funnelshift_l(word[j], word[j], rotate_bits);
+#pragma unroll
+  for (int j = 0; j < K; ++j) sums.count[j] += __popc(word[j]);
+  {
+    int pair = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = i + 1; j < 4; ++j, ++pair)
+        if (j < K) sums.differ[pair] += __popc(word[i] ^ word[j]);
+  }
+  if (store) {
+    uint32_t* out = a.payload + group * K;
+    if (K == 4) {
+      st_c(reinterpret_cast<uint4*>(out), make_uint4(word[0], word[1], word[2], word[3]));
+    } else if (K == 2) {
+      st_c(reinterpret_cast<uint2*>(out), make_uint2(word[0], word[1]));
     } else {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) v[r][e] = 0.0f;
+      for (int j = 0; j < K; ++j) st_c(out + j, word[j]);
     }
   }
 }
 
-// A value of the encode pass that may lie outside the window.  If it does, it goes into the block's wide
-// sums (the sum of x, and the sum of every basis whose sign is +1) and 0 is returned for the thread's own
-// accumulators; otherwise the value itself is returned.
-__device__ __noinline__ float mbq_divert_value(MbqBlockSums* bs, uint32_t* status, float x, uint32_t flags) {
-  if (in_window(bs->window, x)) return x;
-  // flag bytes (0x10 per basis) -> slot bits, plus the slot of the sum of x
-  const uint32_t slots = ((((flags >> 4) * 0x00204081u) >> 21) & 0xFu) | (1u << (kMbqSums - 1));
-  mbq_wide_add_value(bs, status, x, slots);
-  return 0.0f;
-}
+// Scratch of the finalize step, in shared memory: nothing of it is indexed out of a thread's own arrays.
+struct MbqFinalScratch {
+  long long wide[kMbqSums][kAccLimbs];        // the sums of the workspace
+  uint32_t digits[kMbqSums][kAccLimbs + 2];   // wide_to_double's
+  unsigned long long cnt[10];
+  double val[kMbqSums];                       // [j] = (B^T x)_j, [K] = sum of x
+  float alpha_prev[4];
+};
 
-// One tile of kMbqTile elements, coded by one group of 256 threads (tid = index in the group): assign
-// the signs, write the planes, add to the thread's sums.
-template <int K, int MODE, bool FULL>
-__device__ __forceinline__ void mbq_encode_tile(const MbqArgs& a, uint64_t tile, int tid, int lane,
-                                                const float (&v)[kMbqRounds][8], const float (&alpha)[K],
-                                                const MbqTable<K>& table, const uint4* cells, float scale,
-                                                MbqBlockSums* bs, float win_top, uint32_t win_ylow, MbqSums<K>& sums) {
-  const uint64_t n_oct_stored = ((a.n + 31) / 32) * 4;
-  const uint64_t oct0 = tile * (kMbqRounds * 256) + tid;
-  const int q = lane & 3;
-  const uint32_t lane_bytes = 16u * (uint32_t)lane;
-#pragma unroll
-  for (int r = 0; r < kMbqRounds; ++r) {
-    const uint64_t oct = oct0 + r * 256;
-    uint32_t f[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      if (MODE == kMbqResidue) {
-        float res;
-        f[e] = mbq_flags_of_code(mbq_residue_code<K>(alpha, v[r][e], K, &res));
-      } else if (MODE == kMbqSearch) {
-        f[e] = mbq_flags_of_code(mbq_nearest_code<K>(table, v[r][e]));
-      } else {
-        f[e] = mbq_grid_flags(cells, scale, lane_bytes, v[r][e]);
-      }
-    }
-    if (!FULL) {
-      // elements of this octet that exist; signs past the end are zero bits (their values were loaded as 0)
-      const int valid = (oct * 8 + 8 <= a.n) ? 8 : ((oct * 8 < a.n) ? (int)(a.n - oct * 8) : 0);
-      if (valid < 8) {
-#pragma unroll
-        for (int e = 0; e < 8; ++e)
-          if (e >= valid) f[e] = 0;
-      }
-    }
-    // the values as the running sums take them: all of them, unless some lie outside the window
-    float w[8];
-    WindowCheck chk;
-    chk.init();
-#pragma unroll
-    for (int e = 0; e < 8; ++e) w[e] = v[r][e];  // 0 past the end
-#pragma unroll
-    for (int e = 0; e < 8; e += 2) chk.add2(w[e], w[e + 1]);
-    if (!(chk.amax < win_top && chk.ymin >= win_ylow)) {
-#pragma unroll
-      for (int e = 0; e < 8; ++e) w[e] = mbq_divert_value(bs, a.status, w[e], f[e]);
-    }
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const double xd = (double)w[e];
-      sums.sum_x += xd;
-      mbq_add_flagged<0>(sums.plus[0], xd, f[e]);
-      mbq_add_flagged<1>(sums.plus[1], xd, f[e]);
-      if constexpr (K > 2) mbq_add_flagged<2>(sums.plus[2], xd, f[e]);
-      if constexpr (K > 3) mbq_add_flagged<3>(sums.plus[3], xd, f[e]);
-    }
-    // after the quad transpose lane q holds the 32 signs of basis q of its group: counts of +1 and,
-    // against the words of the other three lanes of the quad, counts of differing signs
-    const uint32_t word = quad_transpose(mbq_planes_of_flags(f), lane);
-    if ((FULL || oct < n_oct_stored) && q < K) st_c(a.payload + (oct >> 2) * K + q, word);
-    sums.count += __popc(word);
-#pragma unroll
-    for (int d = 1; d < 4; ++d) {
-      const uint32_t other = __shfl_xor_sync(0xffffffffu, word, d);
-      sums.differ[d - 1] += __popc(word ^ other);
-    }
-  }
-  // every thread of the group has coded the same number of tiles: flushes and pushes are taken together
-  if (++sums.since == kMbqFlushTiles) {
-    sums.since = 0;
-    mbq_flush<K>(sums, bs);
-    if (++sums.flushes == kPushFlushes) {
-      sums.flushes = 0;
-      mbq_push<K>(sums, bs, lane);
-    }
-  }
-}
-
-// A group walks over tiles with a stride of the number of groups and keeps its sums in registers: the
-// group-level reduction is paid once per group, not once per tile.
-// The loads of a group's next tile are in flight while it codes the current one (two register
-// buffers, the loop unrolled by two so that both are addressed statically).
-template <int K, int MODE>
-__device__ __forceinline__ void mbq_encode_tiles(const MbqArgs& a, uint32_t group, int tid, int lane,
-                                                 const float (&alpha)[K], const MbqTable<K>& table, const uint4* cells,
-                                                 float scale, MbqBlockSums* bs, MbqSums<K>& sums) {
-  if (group >= a.n_blocks) return;
-  const float win_top = bs->window.top;
-  const uint32_t win_ylow = bs->window.ylow;
-  const uint64_t full_tiles = a.n / kMbqTile, stride = a.n_blocks;
-  float v0[kMbqRounds][8], v1[kMbqRounds][8];
-  uint64_t tile = group;
-  if (tile < full_tiles) mbq_load_tile<true>(a, tile, tid, v0);
-  while (tile < full_tiles) {
-    const uint64_t t1 = tile + stride;
-    if (t1 < full_tiles) mbq_load_tile<true>(a, t1, tid, v1);
-    mbq_encode_tile<K, MODE, true>(a, tile, tid, lane, v0, alpha, table, cells, scale, bs, win_top, win_ylow, sums);
-    tile = t1;
-    if (t1 >= full_tiles) break;
-    const uint64_t t2 = t1 + stride;
-    if (t2 < full_tiles) mbq_load_tile<true>(a, t2, tid, v0);
-    mbq_encode_tile<K, MODE, true>(a, t1, tid, lane, v1, alpha, table, cells, scale, bs, win_top, win_ylow, sums);
-    tile = t2;
-  }
-  // the ragged last tile of the tensor, if there is one, is the last tile of its group
-  if (tile < a.n_tiles) {
-    mbq_load_tile<false>(a, tile, tid, v0);
-    mbq_encode_tile<K, MODE, false>(a, tile, tid, lane, v0, alpha, table, cells, scale, bs, win_top, win_ylow, sums);
-  }
-}
-
-// Assign the signs, write the planes, gather the sums.  One block of kMbqGroups groups of 256 threads
-// per SM; a group does what a 256-thread block would (its own tiles), the groups of a block share the
-// search tables and the block's wide sums.  Dynamic shared memory: the search grid (kMbqGridBytes), not
-// needed when INIT.
-template <int K, bool INIT>
-__global__ void __launch_bounds__(kMbqEncodeThreads, 1) mbq_encode_kernel(const MbqArgs a) {
-  grid_dependency_handshake();
-  extern __shared__ uint4 s_cells[];
-  __shared__ MbqTable<K> s_table;
-  __shared__ MbqGridInfo s_grid;
-  __shared__ MbqBlockSums s_sums;
-  __shared__ float s_level[16];
-  __shared__ uint32_t s_cnt[10];
-  const int lane = threadIdx.x & 31;
-  const int g = threadIdx.x >> 8;            // group in the block
-  const int tid = threadIdx.x & 255;         // thread in the group
-  const uint32_t group = blockIdx.x * kMbqGroups + g;
-  float alpha[K];
-  mbq_block_sums_clear(&s_sums, threadIdx.x, kMbqEncodeThreads);
-  if (threadIdx.x < 10) s_cnt[threadIdx.x] = 0;
-  if (INIT) {
-#pragma unroll
-    for (int j = 0; j < K; ++j) alpha[j] = a.ws->alpha_init[j];
-    // window of the exact sums: around the mean magnitude of the data
-    if (threadIdx.x == 0) s_sums.window = make_window(alpha[0]);
-  } else {
-#pragma unroll
-    for (int j = 0; j < K; ++j) alpha[j] = 0.0f;
-    mbq_build_table<K>(a.alpha_prev, &s_table, s_level, threadIdx.x);
-    mbq_build_grid<K>(s_table, s_level, &s_grid, s_cells, threadIdx.x, kMbqEncodeThreads);
-    // window of the exact sums: around the largest level (values the levels were fitted to)
-    if (threadIdx.x == 0) {
-      float amax = 0.0f;
-      for (int c = 0; c < (1 << K); ++c) amax = fmaxf(amax, fabsf(s_level[c]));
-      s_sums.window = make_window(amax * 0.125f);
-    }
-  }
-  __syncthreads();
-
-  MbqSums<K> sums;
-  sums.sum_x = 0.0;
-  sums.count = 0;
-  sums.since = 0;
-  sums.flushes = 0;
-#pragma unroll
-  for (int j = 0; j < K; ++j) sums.plus[j] = 0.0;
-#pragma unroll
-  for (int j = 0; j <= K; ++j) sums.irun[j] = 0;
-#pragma unroll
-  for (int d = 0; d < 3; ++d) sums.differ[d] = 0;
-
-  if (INIT) mbq_encode_tiles<K, kMbqResidue>(a, group, tid, lane, alpha, s_table, s_cells, 0.0f, &s_sums, sums);
-  else if (s_grid.usable) mbq_encode_tiles<K, kMbqGrid>(a, group, tid, lane, alpha, s_table, s_cells, s_grid.scale, &s_sums, sums);
-  else mbq_encode_tiles<K, kMbqSearch>(a, group, tid, lane, alpha, s_table, s_cells, 0.0f, &s_sums, sums);
-
-  // what is left in the accumulators, then the warp's total into the block's wide sums
-  mbq_flush<K>(sums, &s_sums);
-  mbq_push<K>(sums, &s_sums, lane);
-
-  const int q = lane & 3;
-  uint32_t my_count = sums.count;
-  uint32_t (&my_differ)[3] = sums.differ;
-  // lanes with the same q hold partial counts of the same basis / pairs: add over the eight quads
-#pragma unroll
-  for (int d = 4; d <= 16; d <<= 1) {
-    my_count += __shfl_xor_sync(0xffffffffu, my_count, d);
-#pragma unroll
-    for (int i = 0; i < 3; ++i) my_differ[i] += __shfl_xor_sync(0xffffffffu, my_differ[i], d);
-  }
-  if (lane < 4) {
-    atomicAdd(&s_cnt[q], my_count);
-#pragma unroll
-    for (int d = 1; d < 4; ++d) {
-      const int other = q ^ d;
-      if (q < other) {  // each pair once; pair index in the order (0,1) (0,2) (0,3) (1,2) (1,3) (2,3)
-        const int pair = (q == 0) ? other - 1 : (q == 1 ? other + 1 : 5);
-        atomicAdd(&s_cnt[4 + pair], my_differ[d - 1]);
-      }
-    }
-  }
-  __syncthreads();
-  mbq_block_sums_deliver(&s_sums, a.ws, threadIdx.x);
-  if (threadIdx.x >= 32 && threadIdx.x < 42) {
-    const int i = threadIdx.x - 32;
-    const unsigned long long c = s_cnt[i];
-    if (c) atomicAdd(i < 4 ? &a.ws->count[i] : &a.ws->differ[i - 4], c);
-  }
-}
-
-// Rounds the exact sums once, then Eq. 3 (least squares by Gaussian elimination with partial pivoting, in
-// double), Eq. 4 (moving average), Eq. 5 (bias), and writes header, side words and alpha_next; leaves the
-// sums of the workspace zeroed for the next call.  One warp.
+// Solves the K x K system G y = rhs by Gaussian elimination with partial pivoting in double, every index a
+// compile-time constant (rows are exchanged by conditional moves).  Returns false if a pivot is below
+// 1e-9 * N (singular: the caller keeps the previous coefficients).
 template <int K>
-__global__ void __launch_bounds__(kMbqFinalizeThreads) mbq_finalize_kernel(const MbqArgs a) {
-  grid_dependency_handshake();
-  __shared__ double s_val[K + 1];  // [j] = (B^T x)_j, [K] = sum of x
-  const int tid = threadIdx.x;
-  MbqWorkspace* ws = a.ws;
-  if (tid <= K) {
-    long long lazy[kAccLimbs];
-    for (int i = 0; i < kAccLimbs; ++i) {
-      const long long sx = ws->wide[kMbqSums - 1][i];
-      // sum over the +1 elements minus sum over the -1 elements = 2 * (sum over +1) - (sum of all), digit by digit
-      lazy[i] = (tid < K) ? 2 * ws->wide[tid][i] - sx : sx;
+__device__ __forceinline__ bool mbq_solve(double (&G)[K][K], double (&rhs)[K], double N, double (&y)[K]) {
+  bool singular = false;
+#pragma unroll
+  for (int col = 0; col < K; ++col) {
+    // the row, from col down, whose entry in this column is largest in magnitude: the first such row
+    int piv = col;
+    double best = fabs(G[col][col]);
+#pragma unroll
+    for (int r = col + 1; r < K; ++r) {
+      const double v = fabs(G[r][col]);
+      if (v > best) { best = v; piv = r; }
     }
-    s_val[tid] = wide_to_double(lazy);
+    if (best < 1e-9 * N) singular = true;
+#pragma unroll
+    for (int r = col + 1; r < K; ++r) {
+      if (r == piv) {
+#pragma unroll
+        for (int q = 0; q < K; ++q) { const double t = G[col][q]; G[col][q] = G[r][q]; G[r][q] = t; }
+        const double t = rhs[col]; rhs[col] = rhs[r]; rhs[r] = t;
+      }
+    }
+    if (!singular) {
+#pragma unroll
+      for (int r = col + 1; r < K; ++r) {
+        const double f = G[r][col] / G[col][col];
+#pragma unroll
+        for (int q = col; q < K; ++q) G[r][q] -= f * G[col][q];
+        rhs[r] -= f * rhs[col];
+      }
+    }
   }
-  unsigned long long c[10];
+  if (singular) return false;
 #pragma unroll
-  for (int j = 0; j < 4; ++j) c[j] = ws->count[j];
+  for (int col = K - 1; col >= 0; --col) {
+    double s = rhs[col];
 #pragma unroll
-  for (int j = 0; j < 6; ++j) c[4 + j] = ws->differ[j];
+    for (int q = col + 1; q < K; ++q) s -= G[col][q] * y[q];
+    y[col] = s / G[col][col];
+  }
+  return true;
+}
+
+// The end of the encode pass, run by the block that delivers its sums last (all threads of it call): rounds
+// the exact sums once, then Eq. 3 (least squares), Eq. 4 (moving average), Eq. 5 (bias), and writes header,
+// side words and alpha_next; leaves the sums of the workspace zeroed for the next call.
+template <int K>
+__device__ void mbq_finalize(const MbqArgs& a, int tid, MbqFinalScratch* fs) {
+  MbqWorkspace* ws = a.ws;
+  // one round trip for everything the step reads (the sums were written by other blocks' atomic adds: read
+  // them where atomics are performed)
+  if (tid < kMbqSums * kAccLimbs) (&fs->wide[0][0])[tid] = __ldcg(&ws->wide[0][0] + tid);
+  else if (tid < kMbqSums * kAccLimbs + 4) fs->cnt[tid - kMbqSums * kAccLimbs] = __ldcg(&ws->count[tid - kMbqSums * kAccLimbs]);
+  else if (tid < kMbqSums * kAccLimbs + 10) fs->cnt[tid - kMbqSums * kAccLimbs] = __ldcg(&ws->differ[tid - kMbqSums * kAccLimbs - 4]);
+  else if (tid < kMbqSums * kAccLimbs + 10 + K && !a.init) fs->alpha_prev[tid - kMbqSums * kAccLimbs - 10] = ldg_c(a.alpha_prev + (tid - kMbqSums * kAccLimbs - 10));
+  else if (tid >= 96 && tid < 96 + 8) st_c(a.header + (tid - 96), mbq_header_word(a, tid - 96));
   __syncthreads();
   // the next call starts from zero
-  for (int i = tid; i < kMbqSums * kAccLimbs; i += kMbqFinalizeThreads) (&ws->wide[0][0])[i] = 0;
-  if (tid < 4) ws->count[tid] = 0;
-  if (tid < 6) ws->differ[tid] = 0;
+  if (tid < kMbqSums * kAccLimbs) (&ws->wide[0][0])[tid] = 0;
+  if (tid >= 64 && tid < 68) ws->count[tid - 64] = 0;
+  if (tid >= 68 && tid < 74) ws->differ[tid - 68] = 0;
+  if (tid == 74) { ws->blocks_done = 0u; ws->next_tile = 0u; }
+  if (tid <= K) {
+    long long lazy[kAccLimbs];
+#pragma unroll
+    for (int i = 0; i < kAccLimbs; ++i) {
+      const long long sx = fs->wide[kMbqSums - 1][i];
+      // sum over the +1 elements minus sum over the -1 elements = 2 * (sum over +1) - (sum of all), digit by digit
+      lazy[i] = (tid < K) ? 2 * fs->wide[tid][i] - sx : sx;
+    }
+    fs->val[tid] = wide_to_double(lazy, fs->digits[tid]);
+  }
+  __syncthreads();
   if (tid != 0) return;
 
-  const double N = (double)a.n, sum_x = s_val[K];
+  const double N = (double)a.n, sum_x = fs->val[K];
   float alpha_next[K];
   if (a.init) {
 #pragma unroll
     for (int j = 0; j < K; ++j) alpha_next[j] = ws->alpha_init[j];
   } else {
     double G[K][K], rhs[K], cur[K], prev[K];
-    int pair = 0;
-    for (int i = 0; i < 4; ++i)
-      for (int j = i + 1; j < 4; ++j, ++pair)
-        if (j < K) G[i][j] = G[j][i] = N - 2.0 * (double)c[4 + pair];
+    {
+      int pair = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = i + 1; j < 4; ++j, ++pair)
+          if (j < K) G[i][j] = G[j][i] = N - 2.0 * (double)fs->cnt[4 + pair];
+    }
+#pragma unroll
     for (int j = 0; j < K; ++j) {
       G[j][j] = N;
-      rhs[j] = s_val[j];
-      prev[j] = (double)ldg_c(a.alpha_prev + j);
+      rhs[j] = fs->val[j];
+      prev[j] = (double)fs->alpha_prev[j];
+      cur[j] = 0.0;
     }
-    bool singular = false;
-    for (int col = 0; col < K && !singular; ++col) {
-      int piv = col;
-      for (int r = col + 1; r < K; ++r)
-        if (fabs(G[r][col]) > fabs(G[piv][col])) piv = r;
-      if (fabs(G[piv][col]) < 1e-9 * N) { singular = true; break; }
-      if (piv != col) {
-        for (int q = 0; q < K; ++q) { const double t = G[col][q]; G[col][q] = G[piv][q]; G[piv][q] = t; }
-        const double t = rhs[col]; rhs[col] = rhs[piv]; rhs[piv] = t;
-      }
-      for (int r = col + 1; r < K; ++r) {
-        const double f = G[r][col] / G[col][col];
-        for (int q = col; q < K; ++q) G[r][q] -= f * G[col][q];
-        rhs[r] -= f * rhs[col];
-      }
-    }
-    if (singular) {
+    if (!mbq_solve<K>(G, rhs, N, cur)) {
+#pragma unroll
       for (int j = 0; j < K; ++j) cur[j] = prev[j];
-    } else {
-      for (int col = K - 1; col >= 0; --col) {
-        double s = rhs[col];
-        for (int q = col + 1; q < K; ++q) s -= G[col][q] * cur[q];
-        cur[col] = s / G[col][col];
-      }
     }
     double beta = (1.0 + (double)a.batch_index) / (10.0 + (double)a.batch_index);
     if (beta > 0.9) beta = 0.9;
+#pragma unroll
     for (int j = 0; j < K; ++j) alpha_next[j] = (float)(beta * prev[j] + (1.0 - beta) * cur[j]);
   }
   double acc = 0.0;
-  for (int j = 0; j < K; ++j) acc += (double)alpha_next[j] * (2.0 * (double)c[j] - N);
+#pragma unroll
+  for (int j = 0; j < K; ++j) acc += (double)alpha_next[j] * (2.0 * (double)fs->cnt[j] - N);
   const float m_q = (float)((acc - sum_x) / N);
-  for (int i = 0; i < 8; ++i) st_c(a.header + i, mbq_header_word(a, i));
+#pragma unroll
   for (int j = 0; j < K; ++j) { st_c(a.side + j, alpha_next[j]); st_c(a.alpha_next + j, alpha_next[j]); }
   st_c(a.side + K, m_q);
   // pad up to the payload
   for (uint32_t* w = reinterpret_cast<uint32_t*>(a.side + K + 1); w < a.payload; ++w) st_c(w, 0u);
+}
+
+// Shared state of a block of the encode pass besides the dynamic shared memory (grid, then stages).
+template <int K>
+struct MbqEncodeShared {
+  MbqTable<K> table;
+  MbqGridInfo grid;
+  MbqBlockSums sums;
+  float level[16];
+  uint32_t cnt[10];
+  uint32_t failed;
+  uint32_t is_last;
+  uint32_t tile[kMbqStages];   // tile each stage holds or is waiting for
+  MbqFinalScratch final_step;
+  alignas(8) unsigned long long bar[kMbqStages];
+};
+
+// Thread 0 asks for a full tile: bulk copies that count their bytes on the stage's mbarrier.
+__device__ __forceinline__ void mbq_request_tile(const MbqArgs& a, uint64_t tile, uint8_t* stage, uint32_t bar) {
+  mbarrier_expect_bytes(bar, kMbqTileBytes + kCopyAnnounceExtra);
+  const uint8_t* src = reinterpret_cast<const uint8_t*>(a.x + tile * kMbqGroupTile);
+  const uint32_t dst = smem_address(stage);
+#pragma unroll
+  for (int part = 0; part < kMbqTileBytes / kMbqCopyBytes; ++part)
+    if (bounds_ok(src + part * kMbqCopyBytes, kMbqCopyBytes, false))
+      bulk_copy_to_shared(dst + part * kMbqCopyBytes, src + part * kMbqCopyBytes, kMbqCopyBytes, bar);
+}
+
+// The tiles of one block.  Full tiles are staged: thread 0 asks for a tile with four bulk copies that
+// count their bytes on the stage's mbarrier; when a tile has landed every thread codes its group out of
+// shared memory, and after the block has met at a barrier the stage is asked to fetch the tile after next.
+// A thread reads its 128 bytes as eight 16-byte slots in an order rotated by its lane, so that the eight
+// lanes of a quarter warp, whose groups are 128 bytes apart, hit eight different bank columns.  The ragged
+// last tile of the tensor is read from global memory with guards, by the block whose turn it is.
+// Returns false if a copy did not arrive in time (reported in the status word; the caller leaves).
+template <int K, int MODE>
+__device__ __forceinline__ bool mbq_encode_tiles(const MbqArgs& a, const MbqLookup<K>& lk, MbqEncodeShared<K>* sh,
+                                                 uint8_t* stages, MbqSums<K>& sums) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  MbqBlockSums* bs = &sh->sums;
+  const float win_top = bs->window.top;
+  const uint32_t win_ylow = bs->window.ylow;
+  const uint32_t bar[kMbqStages] = {smem_address(&sh->bar[0]), smem_address(&sh->bar[1])};
+  const uint64_t full_tiles = a.n / kMbqGroupTile;
+  const uint32_t stride = gridDim.x;
+  auto request = [&](uint64_t tile, int st) { mbq_request_tile(a, tile, stages + st * kMbqTileBytes, bar[st]); };
+  // (the block's first two tiles were asked for before the tables were built; see the kernel)
+  bool pending[kMbqStages] = {false, false};  // thread 0: a copy of the stage's current phase is in flight
+  if (tid == 0) {
+#pragma unroll
+    for (int st = 0; st < kMbqStages; ++st) pending[st] = sh->tile[st] < full_tiles;
+  }
+  // Tiles beyond every block's first two are handed out in the order blocks ask for them, so that the blocks end
+  // together.  Thread 0 always holds one ticket in hand: the atomic that fetches the next one has a whole tile's
+  // time to come back and never delays a request.
+  uint64_t ticket = 0;
+  if (tid == 0 && pending[kMbqStages - 1]) ticket = (uint64_t)kMbqStages * stride + atomicAdd(&a.ws->next_tile, 1u);
+  const uint32_t rot = (uint32_t)(tid & 7);  // slot c of this thread holds values 4 * ((c + rot) & 7) .. + 3 of its group
+  uint32_t slot_offset[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) slot_offset[c] = 16u * ((c + rot) & 7u);
+  uint32_t parity[kMbqStages] = {0u, 0u};
+  int since_flush = 0, since_push = 0;  // the same in every thread: all code the same number of groups
+  for (int st = 0;; st ^= 1) {
+    const uint64_t tile = sh->tile[st];  // written before the last barrier
+    if (tile >= full_tiles) break;
+    if (mbarrier_wait(bar[st], parity[st])) {
+      parity[st] ^= 1u;
+      if (tid == 0) pending[st] = false;
+    } else {
+      atomicOr(a.status, kDevCopyTimeout);
+      sh->failed = 1u;  // seen by everybody after the barrier below; this tile's values are whatever the stage holds
+    }
+    const uint8_t* mine = stages + st * kMbqTileBytes + tid * 128;
+    // first look: are all 32 values inside the window of the exact sums (or zero)?
+    WindowCheck chk;
+    chk.init();
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const float4 v = *reinterpret_cast<const float4*>(mine + slot_offset[c]);
+      chk.add2(v.x, v.y);
+      chk.add2(v.z, v.w);
+    }
+    uint32_t s4[8];
+    if (chk.amax < win_top && chk.ymin >= win_ylow) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c)
+        s4[c] = mbq_code_four<K, MODE>(lk, *reinterpret_cast<const float4*>(mine + slot_offset[c]), sums);
+    } else {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        uint32_t word = 0;
+#pragma unroll 1
+        for (int e = 0; e < 4; ++e)
+          word += mbq_code_value_slowly<K, MODE>(lk, *reinterpret_cast<const float*>(mine + slot_offset[c] + 4 * e), bs, a.status) << e;
+        s4[c] = word;
+      }
+    }
+    mbq_finish_group<K>(a, s4, 4u * rot, tile * kMbqEncodeThreads + tid, true, sums);
+    __syncthreads();  // every thread has taken its values out of the stage
+    if (sh->failed) break;
+    if (tid == 0) {
+      const uint64_t next = ticket;
+      sh->tile[st] = next < full_tiles ? (uint32_t)next : 0xFFFFFFFFu;
+      if (next < full_tiles) {
+        request(next, st);
+        pending[st] = true;
+        ticket = (uint64_t)kMbqStages * stride + atomicAdd(&a.ws->next_tile, 1u);
+      }
+    }
+    if (++since_flush == kMbqFlushGroups) {
+      since_flush = 0;
+      mbq_flush<K>(sums, bs);
+      if (++since_push == kPushFlushes) {
+        since_push = 0;
+        mbq_push<K>(sums, bs, lane);
+      }
+    }
+  }
+  if (sh->failed) {
+    // give what is still in flight a bounded time to land before the block gives its shared memory back
+    if (tid == 0) {
+#pragma unroll
+      for (int st = 0; st < kMbqStages; ++st)
+        if (pending[st]) mbarrier_wait(bar[st], parity[st]);
+    }
+    return false;
+  }
+
+  // the ragged last tile, read from global memory by the block whose turn it is
+  if (full_tiles * kMbqGroupTile < a.n && full_tiles % stride == blockIdx.x) {
+    const uint64_t first = full_tiles * kMbqGroupTile + (uint64_t)tid * 32;  // first value of this thread's group
+    const uint64_t n_groups_stored = (a.n + 31) / 32;
+    const int valid = first >= a.n ? 0 : (a.n - first >= 32 ? 32 : (int)(a.n - first));
+    uint32_t s4[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      uint32_t word = 0;
+#pragma unroll 1
+      for (int e = 0; e < 4; ++e)
+        if (4 * c + e < valid)  // values past the end have no signs and add nothing
+          word += mbq_code_value_slowly<K, MODE>(lk, ldg_c(a.x + first + 4 * c + e), bs, a.status) << e;
+      s4[c] = word;
+    }
+    const uint64_t group = full_tiles * kMbqEncodeThreads + tid;
+    mbq_finish_group<K>(a, s4, 0u, group, group < n_groups_stored, sums);
+  }
+  return true;
+}
+
+// Assign the signs, write the planes, gather the sums, and (in the block that ends last) solve Eq. 3-5:
+// the whole forward quantizer of a batch in one launch.  Persistent blocks of 256 threads, two per SM.
+// Dynamic shared memory: the search grid (kMbqGridBytes), then the stages.
+template <int K, bool INIT>
+__global__ void __launch_bounds__(kMbqEncodeThreads, kMbqBlocksPerSm) mbq_encode_kernel(const MbqArgs a) {
+  grid_dependency_handshake();
+  extern __shared__ __align__(128) uint8_t s_dyn[];
+  __shared__ MbqEncodeShared<K> sh;
+  const int tid = threadIdx.x, lane = tid & 31;
+  uint4* cells = reinterpret_cast<uint4*>(s_dyn);
+  uint8_t* stages = s_dyn + kMbqGridBytes;
+
+  // first of all the block's first two tiles are asked for: they arrive while the tables are built
+  if (tid == 0) {
+    const uint64_t full_tiles = a.n / kMbqGroupTile;
+    mbarrier_init(smem_address(&sh.bar[0]), 1);
+    mbarrier_init(smem_address(&sh.bar[1]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    sh.failed = 0u;
+    sh.grid.usable = 0;
+#pragma unroll
+    for (int st = 0; st < kMbqStages; ++st) {
+      const uint64_t tile = blockIdx.x + (uint64_t)st * gridDim.x;
+      sh.tile[st] = tile < full_tiles ? (uint32_t)tile : 0xFFFFFFFFu;
+      if (tile < full_tiles) mbq_request_tile(a, tile, stages + st * kMbqTileBytes, smem_address(&sh.bar[st]));
+    }
+  }
+
+  MbqLookup<K> lk;
+  lk.table = &sh.table;
+  lk.column = smem_address(cells) + 16u * (uint32_t)(lane & (kMbqColumns - 1));
+  lk.scale = 0.0f;
+#pragma unroll
+  for (int j = 0; j < K; ++j) lk.alpha[j] = 0.0f;
+  mbq_block_sums_clear(&sh.sums, tid, kMbqEncodeThreads);
+  if (tid < 10) sh.cnt[tid] = 0;
+  __syncthreads();  // sh.grid.usable = 0 is in place before the tables are built
+  if (INIT) {
+#pragma unroll
+    for (int j = 0; j < K; ++j) lk.alpha[j] = a.ws->alpha_init[j];
+    // window of the exact sums: around the mean magnitude of the data
+    if (tid == 0) sh.sums.window = make_window(lk.alpha[0]);
+  } else {
+    mbq_build_table<K>(a.alpha_prev, &sh.table, sh.level, tid);
+    // (the scratch of the grid builder must not be a stage: copies are landing there)
+    mbq_build_grid<K>(sh.table, sh.level, &sh.grid, cells, tid, kMbqEncodeThreads);
+    // window of the exact sums: around the largest level (the values the levels were fitted to)
+    if (tid == 0) {
+      float amax = 0.0f;
+      for (int c = 0; c < (1 << K); ++c) amax = fmaxf(amax, fabsf(sh.level[c]));
+      sh.sums.window = make_window(amax * 0.125f);
+    }
+  }
+  __syncthreads();
+  lk.scale = sh.grid.scale;
+
+  MbqSums<K> sums;
+  sums.clear();
+  bool ok;
+  if (INIT) ok = mbq_encode_tiles<K, kMbqResidue>(a, lk, &sh, stages, sums);
+  else if (sh.grid.usable) ok = mbq_encode_tiles<K, kMbqGrid>(a, lk, &sh, stages, sums);
+  else ok = mbq_encode_tiles<K, kMbqSearch>(a, lk, &sh, stages, sums);
+
+  if (ok) {
+    // what is left in the accumulators, then the warp's total into the block's wide sums
+    mbq_flush<K>(sums, &sh.sums);
+    mbq_push<K>(sums, &sh.sums, lane);
+    // counts: lanes, then warps
+#pragma unroll
+    for (int j = 0; j < K; ++j) {
+      const uint32_t c = __reduce_add_sync(0xffffffffu, sums.count[j]);
+      if (lane == 0) atomicAdd(&sh.cnt[j], c);
+    }
+    int pair = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = i + 1; j < 4; ++j, ++pair) {
+        if (j >= K) continue;
+        const uint32_t c = __reduce_add_sync(0xffffffffu, sums.differ[pair]);
+        if (lane == 0) atomicAdd(&sh.cnt[4 + pair], c);
+      }
+  }
+  __syncthreads();
+  if (ok) {
+    mbq_block_sums_deliver(&sh.sums, a.ws, tid);
+    if (tid >= 32 && tid < 42) {
+      const int i = tid - 32;
+      const unsigned long long c = sh.cnt[i];
+      if (c) atomicAdd(i < 4 ? &a.ws->count[i] : &a.ws->differ[i - 4], c);
+    }
+  }
+  // The block that gets here last finishes the batch (also after a copy that did not arrive: the status word
+  // says so, the stream is then meaningless, but the workspace is left clean).  No block waits for another.
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) sh.is_last = (atomicAdd(&a.ws->blocks_done, 1u) == gridDim.x - 1) ? 1u : 0u;
+  __syncthreads();
+  if (sh.is_last) {
+    __threadfence();
+    mbq_finalize<K>(a, tid, &sh.final_step);
+  }
+
 }
 
 // Receiver: planes -> codes -> level(c) - m_q.

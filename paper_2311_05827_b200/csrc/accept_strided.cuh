@@ -10,6 +10,7 @@
 // vectorised tensor: the per-chunk constants come from the records the range pass left in the
 // workspace (accept_wide.cuh), so this path always runs as range pass + constants + encode.
 #pragma once
+#include "accept_async.cuh"
 #include "accept_wide.cuh"
 
 namespace accept {
@@ -43,51 +44,6 @@ constexpr int kStridedRowBytes = kStridedOctetsPerBlock * 32;
 constexpr int kStridedRowBlockPitch = 8 * kStridedRowBytes + 32;
 constexpr int kStridedTileBytes = 4 * kStridedRowBlockPitch;
 constexpr int kStridedSmemBytes = kStridedTileBytes + 16;  // + two mbarriers
-
-__device__ __forceinline__ uint32_t smem_address(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbarrier_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbarrier_expect_bytes(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_copy_to_shared(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-// How long a wait for an asynchronous copy may last.  A copy lands within microseconds; the limit only has
-// to outlast the time a kernel may sit descheduled on a GPU that is time-sliced between processes (the
-// timer keeps running meanwhile), which is a matter of milliseconds.
-#ifdef ACCEPT_TEST_COPY_STALL
-// Tests-only build: every stage announces 16 bytes more than its copies deliver, so all copies land but no
-// phase ever completes; the waits run out (after 2 ms) and the kernel must report it and leave cleanly.
-constexpr unsigned long long kCopyWaitNs = 2000000ull;
-constexpr uint32_t kCopyAnnounceExtra = 16u;
-#else
-constexpr unsigned long long kCopyWaitNs = 200000000ull;
-constexpr uint32_t kCopyAnnounceExtra = 0u;
-#endif
-
-// Waits for the phase of the given parity; gives up after kCopyWaitNs.
-__device__ __forceinline__ bool mbarrier_wait(uint32_t bar, uint32_t parity) {
-  unsigned long long t0 = 0;
-  for (uint32_t it = 0;; ++it) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-    if (done) return true;
-    if ((it & 63u) == 63u) {
-      unsigned long long now;
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-      if (t0 == 0) t0 = now;
-      else if (now - t0 > kCopyWaitNs) return false;
-    }
-  }
-}
 
 // Transposes a thread's 8 rows x 8 features of codes and stores the words of its eight features.
 template <int K, int LAYOUT>

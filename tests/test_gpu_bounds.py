@@ -118,3 +118,32 @@ def test_bounded_copy_wait_runs_out_and_the_gpu_stays_usable(k, layout):
     # the ordinary library, same process, same GPU: the same call is bit-exact
     test_gpu_strided.check(x, chunk, stride, k, RANGE_ABSMAX, ROUND_NEAREST, layout)
     test_gpu_parity.check_roundtrip(x[:4096 * 7 + 5], 4096, 4, RANGE_ABSMAX, ROUND_STOCHASTIC, LAYOUT_INTERLEAVED, seed=1)
+
+
+def test_bounded_copy_wait_of_the_forward_quantizer_runs_out_cleanly():
+    """The staged encode pass of the forward quantizer under the same stalled copies: the status word reports it,
+    the workspace is left clean (the block that ends last still closes the batch), and the ordinary library
+    then codes the same tensor bit for bit like the oracle, on the very workspace the failed call used."""
+    import paper_2311_05827_b200 as A
+    n, k = 8192 * 40 + 123, 3
+    x = workloads.random_tensor(n, 5, "relu")
+    alpha_prev = np.array([0.9, 0.5, 0.27], dtype=np.float32)
+    p = A.MbqParams(n, k, 2, False)
+    d_x = torch.from_numpy(x).cuda()
+    d_prev = torch.from_numpy(alpha_prev).cuda()
+    d_next = torch.zeros(k, dtype=torch.float32, device="cuda")
+    g_stream = gpu_util.guarded_stream(A, torch, p)
+    g_ws = gpu_util.guarded_workspace(A, torch, p)
+    d_ws = g_ws.view(torch.int32)
+    with gpu_util.library_variant("stall"):
+        A.accept_mbq_compress(p, d_x, d_prev, d_next, g_stream.bytes, d_ws)
+        assert A.accept_last_device_status(d_ws) & A.DEV_COPY_TIMEOUT
+        g_stream.check("stream")
+        g_ws.check("workspace")
+    assert not bool(d_ws.view(torch.uint8)[32:].any()), "sums, counters or tickets left behind"
+    d_ws.zero_()  # the caller clears the status word
+    A.accept_mbq_compress(p, d_x, d_prev, d_next, g_stream.bytes, d_ws)
+    assert A.accept_last_device_status(d_ws) == 0
+    ref, ref_alpha = oracle.mbq_compress(x, k, 2, False, alpha_prev)
+    assert np.array_equal(g_stream.bytes.cpu().numpy(), ref)
+    assert np.array_equal(d_next.cpu().numpy().view(np.uint32), ref_alpha.view(np.uint32))
