@@ -93,9 +93,12 @@ typedef enum { ACCEPT_LAYOUT_INTERLEAVED = 0, ACCEPT_LAYOUT_BITPLANE = 1 } accep
  *                Group index G = g*F + f, words G*k .. G*k+k-1 of the payload, element
  *                (row b, feature f) at position t = b % 32 of its group; rows past the last are zero
  *                bits; payload = 4*k*ceil(rows/32)*F bytes.  Ranges stay per chunk of consecutive
- *                values.  Needs F % 8 == 0, n_elems % F == 0, 32-byte aligned tensors, and not
- *                (k = 8 with BITPLANE); runs as range pass + constants + encode (workspace: 16
- *                bytes per chunk more, as for chunk_elems > 32768).  Header word 7 carries F.
+ *                values.  Needs n_elems % F == 0 and a 32-byte aligned input; any F >= 1 (the
+ *                paper's smallest outputs need not have 8 | w*h*c).  With F % 8 == 0 (and not k = 8
+ *                with BITPLANE) a thread codes eight features of eight rows with 32-byte loads;
+ *                every other shape takes one feature per thread, slower but for any F.  Runs as
+ *                range pass + constants + encode (workspace: 16 bytes per chunk more, as for
+ *                chunk_elems > 32768).  Header word 7 carries F.
  *   seed, rng_offset  STOCHASTIC only.  Element i draws
  *                  U_i = (g >> 8) * 2^-24,
  *                  g   = h * M[ctr & 3] (mod 2^32),  M = {1, 0x9E3779B1, 0x85EBCA77, 0xC2B2AE3D},

@@ -308,6 +308,55 @@ cudaError_t launch_strided_decode_for(const accept_params* p, const CodecArgs& a
   }
 }
 
+// The octet-per-thread kernels need rows that start on 32-byte boundaries and have no eight-plane form; every
+// other shape goes through the feature-per-thread kernels.
+bool strided_any_shape(const accept_params* p) {
+  return p->group_stride % 8 != 0 || (p->k == 8 && p->layout == ACCEPT_LAYOUT_BITPLANE);
+}
+
+dim3 strided_any_grid(const accept_params* p) {
+  const unsigned gx = (p->group_stride + accept::kStridedAnyBlock - 1) / accept::kStridedAnyBlock;
+  const unsigned gy = (unsigned)((p->n_elems / p->group_stride + 31) / 32);
+  return dim3(gx, gy, 1);
+}
+
+template <int K, int LAYOUT, int RANGE>
+cudaError_t launch_strided_encode_any(int round, const CodecArgs& a, const accept::ChunkRecord* rec, dim3 grid, cudaStream_t s) {
+  if (round == accept::kNearest)
+    return launch_overlapped(accept::strided_encode_any_kernel<K, LAYOUT, RANGE, accept::kNearest>, grid, accept::kStridedAnyBlock, s, a, rec);
+  return launch_overlapped(accept::strided_encode_any_kernel<K, LAYOUT, RANGE, accept::kStochastic>, grid, accept::kStridedAnyBlock, s, a, rec);
+}
+
+template <int RANGE>
+cudaError_t launch_strided_encode_any_for(const accept_params* p, const CodecArgs& a, const accept::ChunkRecord* rec, dim3 grid,
+                                          cudaStream_t s) {
+  const bool bp = p->layout == ACCEPT_LAYOUT_BITPLANE;
+  switch (p->k) {
+    case 2: return bp ? launch_strided_encode_any<2, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
+                      : launch_strided_encode_any<2, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s);
+    case 3: return launch_strided_encode_any<3, accept::kBitplane, RANGE>(p->round, a, rec, grid, s);
+    case 4: return bp ? launch_strided_encode_any<4, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
+                      : launch_strided_encode_any<4, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s);
+    default: return bp ? launch_strided_encode_any<8, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
+                       : launch_strided_encode_any<8, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s);
+  }
+}
+
+template <int RANGE>
+cudaError_t launch_strided_decode_any_for(const accept_params* p, const CodecArgs& a, dim3 grid, cudaStream_t s) {
+  const bool bp = p->layout == ACCEPT_LAYOUT_BITPLANE;
+  const unsigned block = accept::kStridedAnyBlock;
+  switch (p->k) {
+    case 2: return bp ? launch_overlapped(accept::strided_decode_any_kernel<2, accept::kBitplane, RANGE>, grid, block, s, a)
+                      : launch_overlapped(accept::strided_decode_any_kernel<2, accept::kInterleaved, RANGE>, grid, block, s, a);
+    case 3: return launch_overlapped(accept::strided_decode_any_kernel<3, accept::kBitplane, RANGE>, grid, block, s, a);
+    case 4: return bp ? launch_overlapped(accept::strided_decode_any_kernel<4, accept::kBitplane, RANGE>, grid, block, s, a)
+                      : launch_overlapped(accept::strided_decode_any_kernel<4, accept::kInterleaved, RANGE>, grid, block, s, a);
+    default: return bp ? launch_overlapped(accept::strided_decode_any_kernel<8, accept::kBitplane, RANGE>, grid, block, s, a)
+                       : launch_overlapped(accept::strided_decode_any_kernel<8, accept::kInterleaved, RANGE>, grid, block, s, a);
+  }
+}
+
 dim3 strided_grid(const accept_params* p) {
   const unsigned gx = (p->group_stride / 8 + accept::kStridedOctetsPerBlock - 1) / accept::kStridedOctetsPerBlock;
   const unsigned gy = (unsigned)((p->n_elems / p->group_stride + 31) / 32);
@@ -320,14 +369,17 @@ accept_status launch_strided(const accept_params* p, const CodecArgs& a, uint8_t
   const uint64_t n_oct = (p->n_elems + 7) / 8;
   const unsigned range_grid = (unsigned)((n_oct + 4 * 256 - 1) / (4 * 256));
   const unsigned fin_grid = (unsigned)((a.n_chunks + 255) / 256);
+  const bool any = strided_any_shape(p);
   if (p->range == ACCEPT_RANGE_ABSMAX) {
     ACCEPT_LAUNCH(launch_overlapped(accept::wide_range_kernel<accept::kAbsMax, 4>, dim3(range_grid), 256, s, a, rec));
     ACCEPT_LAUNCH(launch_overlapped(accept::wide_finalize_kernel<accept::kAbsMax>, dim3(fin_grid), 256, s, a, rec));
-    ACCEPT_LAUNCH(launch_strided_encode_for<accept::kAbsMax>(p, a, rec, strided_grid(p), s));
+    if (any) ACCEPT_LAUNCH(launch_strided_encode_any_for<accept::kAbsMax>(p, a, rec, strided_any_grid(p), s));
+    else ACCEPT_LAUNCH(launch_strided_encode_for<accept::kAbsMax>(p, a, rec, strided_grid(p), s));
   } else {
     ACCEPT_LAUNCH(launch_overlapped(accept::wide_range_kernel<accept::kMinMax, 4>, dim3(range_grid), 256, s, a, rec));
     ACCEPT_LAUNCH(launch_overlapped(accept::wide_finalize_kernel<accept::kMinMax>, dim3(fin_grid), 256, s, a, rec));
-    ACCEPT_LAUNCH(launch_strided_encode_for<accept::kMinMax>(p, a, rec, strided_grid(p), s));
+    if (any) ACCEPT_LAUNCH(launch_strided_encode_any_for<accept::kMinMax>(p, a, rec, strided_any_grid(p), s));
+    else ACCEPT_LAUNCH(launch_strided_encode_for<accept::kMinMax>(p, a, rec, strided_grid(p), s));
   }
   return ACCEPT_OK;
 }
@@ -438,8 +490,7 @@ accept_status accept_check_params(const accept_params* p) {
   if (!(p->k == 2 || p->k == 3 || p->k == 4 || p->k == 8)) return ACCEPT_ERR_BAD_K;
   if (p->k == 3 && p->layout != ACCEPT_LAYOUT_BITPLANE) return ACCEPT_ERR_BAD_K;
   if (p->group_stride != 0) {
-    if (p->group_stride % 8 != 0 || p->n_elems % p->group_stride != 0) return ACCEPT_ERR_BAD_SIZE;
-    if (p->k == 8 && p->layout == ACCEPT_LAYOUT_BITPLANE) return ACCEPT_ERR_BAD_K;
+    if (p->n_elems % p->group_stride != 0) return ACCEPT_ERR_BAD_SIZE;
     if ((p->n_elems / p->group_stride + 31) / 32 > 65535) return ACCEPT_ERR_BAD_SIZE;  // batch groups ride on grid.y
   }
   // one block per chunk / per 4096 elements must fit the grid's x dimension
@@ -516,8 +567,13 @@ accept_status accept_decompress(const accept_params* p, const void* d_stream, si
   ACCEPT_BOUNDS(static_cast<cudaStream_t>(cuda_stream), bounds_list.add(d_stream, accept_compressed_size(p), false);
                 bounds_list.add(d_xhat, 4 * p->n_elems, true); bounds_list.add(d_ws, 16, true));
   if (is_strided(p)) {
-    if (!is_aligned(d_xhat, 32)) return ACCEPT_ERR_MISALIGNED;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (strided_any_shape(p)) {
+      if (p->range == ACCEPT_RANGE_ABSMAX) ACCEPT_LAUNCH(launch_strided_decode_any_for<accept::kAbsMax>(p, a, strided_any_grid(p), s));
+      else ACCEPT_LAUNCH(launch_strided_decode_any_for<accept::kMinMax>(p, a, strided_any_grid(p), s));
+      return ACCEPT_OK;
+    }
+    if (!is_aligned(d_xhat, 32)) return ACCEPT_ERR_MISALIGNED;
     if (p->range == ACCEPT_RANGE_ABSMAX) ACCEPT_LAUNCH(launch_strided_decode_for<accept::kAbsMax>(p, a, strided_grid(p), s));
     else ACCEPT_LAUNCH(launch_strided_decode_for<accept::kMinMax>(p, a, strided_grid(p), s));
     return ACCEPT_OK;

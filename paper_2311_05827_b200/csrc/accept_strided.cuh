@@ -413,4 +413,96 @@ __global__ void __launch_bounds__(256) strided_decode_kernel(const CodecArgs a) 
   }
 }
 
+// ----------------------------------------------------------------------------- any shape
+//
+// Batch groups for any number of values per sample (rows then start at any multiple of four bytes, so there
+// are no 32-byte row loads) and for eight bit planes: a thread owns ONE feature and walks down the 32 rows of
+// a batch group, so consecutive lanes read consecutive floats of a row (128 bytes per warp instruction,
+// whatever the alignment) and a thread ends up with all 32 codes of its group: the k words are formed in the
+// thread's own registers and written as one run of k words per lane.  Per element: the chunk's constants from
+// the record (neighbouring lanes nearly always share it), one quantizer step, k bit insertions.
+
+constexpr int kStridedAnyBlock = 256;  // features per block
+
+template <int K, int LAYOUT, int RANGE, int ROUND>
+__global__ void __launch_bounds__(kStridedAnyBlock) strided_encode_any_kernel(const CodecArgs a, const ChunkRecord* rec) {
+  grid_dependency_handshake();
+  const int tid = threadIdx.x;
+  if (blockIdx.x == 0 && blockIdx.y == 0 && tid < 8) {
+    st_c(a.header + tid, header_word(a, tid));
+    if ((a.n_chunks & 1) && tid < 2) st_c(reinterpret_cast<uint32_t*>(a.meta + a.n_chunks) + tid, 0u);
+  }
+  const uint32_t F = a.group_stride;
+  const uint64_t n_rows = a.n / F;
+  const uint32_t f = blockIdx.x * kStridedAnyBlock + tid;
+  if (f >= F) return;
+  const uint64_t g = blockIdx.y;
+  const Rng rng{(uint32_t)a.seed, (uint32_t)(a.seed >> 32)};
+  uint32_t word[K];
+#pragma unroll
+  for (int j = 0; j < K; ++j) word[j] = 0u;
+#pragma unroll 4
+  for (int r = 0; r < 32; ++r) {
+    const uint64_t row = g * 32 + r;
+    if (row >= n_rows) break;  // rows past the last are zero bits
+    const uint64_t i = row * F + f;
+    float v = ldg_c(a.x + i);
+    const Scale sc = scale_from_record(rec + chunk_of(a, i));
+    if (sc.nonfinite) v = 0.0f;
+    uint32_t h = 0;
+    if (ROUND == kStochastic) h = rng.word(a.rng_offset + i);
+    const uint32_t u = quantize_code<K, RANGE, ROUND>(v, sc, h);
+    if (LAYOUT == kBitplane) {
+#pragma unroll
+      for (int j = 0; j < K; ++j) word[j] |= ((u >> j) & 1u) << r;
+    } else {
+      // the code of row r sits at bits [K r, K r + K) of the group's K words: inside one word, since K divides 32
+      constexpr int per_word = 32 / K;
+#pragma unroll
+      for (int j = 0; j < K; ++j)
+        if (r / per_word == j) word[j] |= u << (K * (r % per_word));
+    }
+  }
+  uint32_t* out = a.payload + (g * F + f) * K;
+#pragma unroll
+  for (int j = 0; j < K; ++j) st_c(out + j, word[j]);
+}
+
+template <int K, int LAYOUT, int RANGE>
+__global__ void __launch_bounds__(kStridedAnyBlock) strided_decode_any_kernel(const CodecArgs a) {
+  grid_dependency_handshake();
+  const int tid = threadIdx.x;
+  if (blockIdx.x == 0 && blockIdx.y == 0 && tid < 8) {
+    const uint32_t mask = (tid == 6) ? 0xFFFF00FFu : 0xFFFFFFFFu;
+    if ((a.header[tid] & mask) != (header_word(a, tid) & mask)) atomicOr(a.status, kDevBadHeader);
+  }
+  const uint32_t F = a.group_stride;
+  const uint64_t n_rows = a.n / F;
+  const uint32_t f = blockIdx.x * kStridedAnyBlock + tid;
+  if (f >= F) return;
+  const uint64_t g = blockIdx.y;
+  const uint32_t* in = a.payload + (g * F + f) * K;
+  uint32_t word[K];
+#pragma unroll
+  for (int j = 0; j < K; ++j) word[j] = ldg_c(in + j);
+#pragma unroll 4
+  for (int r = 0; r < 32; ++r) {
+    const uint64_t row = g * 32 + r;
+    if (row >= n_rows) break;
+    const uint64_t i = row * F + f;
+    uint32_t u = 0;
+    if (LAYOUT == kBitplane) {
+#pragma unroll
+      for (int j = 0; j < K; ++j) u |= ((word[j] >> r) & 1u) << j;
+    } else {
+      constexpr int per_word = 32 / K;
+#pragma unroll
+      for (int j = 0; j < K; ++j)
+        if (r / per_word == j) u = (word[j] >> (K * (r % per_word))) & ((1u << K) - 1u);
+    }
+    const float2 so = ldg_c(a.meta + chunk_of(a, i));
+    st_c(a.xhat + i, dequantize_code<K, RANGE>(u, so.x, so.y));
+  }
+}
+
 }  // namespace accept

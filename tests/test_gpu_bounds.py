@@ -56,7 +56,7 @@ def test_every_launch_path_stays_inside_its_buffers():
         assert _report()[:2] == (0, 0), "consecutive layout"
         # pack groups along the batch dimension
         for k, range_, round_, layout in test_gpu_strided.modes():
-            for rows, stride, chunk in [(64, 24, 64 * 24), (40, 16, 96), (33, 2056, 4096), (70, 520, 1024)]:
+            for rows, stride, chunk in [(64, 24, 64 * 24), (40, 16, 96), (33, 2056, 4096), (70, 520, 1024), (33, 7, 64), (65, 2060, 4096)]:
                 x = workloads.random_tensor(rows * stride, rows + k, "normal")
                 test_gpu_strided.check(x, chunk, stride, k, range_, round_, layout, seed=21, rng_offset=5)
         assert _report()[:2] == (0, 0), "batch groups"

@@ -16,7 +16,7 @@ torch = pytest.importorskip("torch")
 def modes():
     out = []
     for layout in (LAYOUT_INTERLEAVED, LAYOUT_BITPLANE):
-        for k in ((2, 4, 8) if layout == LAYOUT_INTERLEAVED else (2, 3, 4)):
+        for k in ((2, 4, 8) if layout == LAYOUT_INTERLEAVED else (2, 3, 4, 8)):
             for range_ in (RANGE_ABSMAX, RANGE_MINMAX):
                 for round_ in (ROUND_NEAREST, ROUND_STOCHASTIC):
                     out.append((k, range_, round_, layout))
@@ -69,6 +69,22 @@ def test_strided_parity(mode, rows, stride, chunk):
     check(x, chunk, stride, k, range_, round_, layout, seed=21, rng_offset=5)
 
 
+@pytest.mark.parametrize("mode", modes())
+@pytest.mark.parametrize("rows,stride,chunk", [
+    (70, 1, 32),             # one value per sample: the groups are runs of the only column
+    (33, 7, 64),             # rows start at any multiple of four bytes
+    (96, 12, 96 * 12),       # one range for the whole tensor
+    (40, 50, 512),
+    (65, 2060, 4096),        # the 2056 + 4 case: more than one block of features, ragged last block
+])
+def test_strided_parity_any_values_per_sample(mode, rows, stride, chunk):
+    """Values per sample that are not a multiple of eight (Sec. 4.3.1's smaller outputs need not be): the
+    feature-per-thread kernels, every mode, eight bit planes included."""
+    k, range_, round_, layout = mode
+    x = workloads.random_tensor(rows * stride, rows + stride + k, "normal")
+    check(x, chunk, stride, k, range_, round_, layout, seed=33, rng_offset=2 ** 32 - 1000)
+
+
 @pytest.mark.parametrize("i", range(24))
 def test_strided_parity_random_configurations(i):
     """Seeded random (batch rows, values per sample, chunk, mode, seed, counter offset): rows that do not fill
@@ -77,6 +93,8 @@ def test_strided_parity_random_configurations(i):
     rng = np.random.default_rng([20231106, i])
     rows = int(rng.choice([1, 2, 31, 32, 33, int(rng.integers(1, 200))]))
     stride = 8 * int(rng.choice([1, 3, 63, 64, 65, int(rng.integers(1, 1200))]))
+    if i % 3 == 2:
+        stride += int(rng.integers(1, 8))  # not a multiple of eight: the feature-per-thread kernels
     n = rows * stride
     chunk = int(rng.choice([32, 96, 1024, 4096, 32 * int(rng.integers(1, 2000)), (n + 31) // 32 * 32]))
     k, range_, round_, layout = modes()[int(rng.integers(0, len(modes())))]
@@ -101,7 +119,7 @@ def test_strided_nonfinite_and_bad_arguments():
     x = workloads.random_tensor(64 * 64, 2, "normal")
     x[70] = np.nan
     check(x, 1024, 64, 4, RANGE_ABSMAX, ROUND_NEAREST, LAYOUT_BITPLANE)
-    assert A.accept_check_params(A.Params(64 * 64, 1024, 4, group_stride=12)) == 9     # not a multiple of 8
+    assert A.accept_check_params(A.Params(64 * 63, 1024, 4, group_stride=63)) == 0      # any number of values per sample
     assert A.accept_check_params(A.Params(64 * 64 + 8, 1024, 4, group_stride=64)) == 9  # n not a multiple of F
-    assert A.accept_check_params(A.Params(64 * 64, 1024, 8, layout=LAYOUT_BITPLANE, group_stride=64)) == 2
+    assert A.accept_check_params(A.Params(64 * 64, 1024, 8, layout=LAYOUT_BITPLANE, group_stride=64)) == 0
     assert A.accept_workspace_size(A.Params(64 * 64, 1024, 4, group_stride=64)) == 16 + 16 * 4
