@@ -424,8 +424,11 @@ accept_status launch_mbq_compress(const accept::MbqArgs& a, cudaStream_t s) {
   // the search grid and the staged tiles need more dynamic shared memory than a kernel gets without opting in
   // (the attribute is per device: set every time)
   if (a.init) {
-    for (int j = 0; j < K; ++j)
-      ACCEPT_LAUNCH(launch_overlapped(accept::mbq_residue_sum_kernel<K>, dim3(a.n_residue_blocks), 256, s, a, j));
+    const dim3 rgrid(a.n_residue_blocks);
+    ACCEPT_LAUNCH(launch_overlapped(accept::mbq_residue_sum_kernel<K, 0>, rgrid, 256, s, a));
+    ACCEPT_LAUNCH(launch_overlapped(accept::mbq_residue_sum_kernel<K, 1>, rgrid, 256, s, a));
+    if constexpr (K > 2) ACCEPT_LAUNCH(launch_overlapped(accept::mbq_residue_sum_kernel<K, 2>, rgrid, 256, s, a));
+    if constexpr (K > 3) ACCEPT_LAUNCH(launch_overlapped(accept::mbq_residue_sum_kernel<K, 3>, rgrid, 256, s, a));
     auto fn = accept::mbq_encode_kernel<K, true>;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, accept::kMbqEncodeSmemBytes) != cudaSuccess)
       return ACCEPT_ERR_CUDA;

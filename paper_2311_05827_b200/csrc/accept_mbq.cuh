@@ -21,7 +21,7 @@ namespace accept {
 
 constexpr int kMbqRounds = 2;                      // octets per thread and tile of a residue pass
 constexpr int kMbqTile = kMbqRounds * 256 * 8;     // elements per tile of a residue pass
-constexpr int kMbqResidueBlocks = 1184;            // blocks of a residue pass
+constexpr int kMbqResidueBlocks = 148 * 3;         // blocks of a residue pass: three resident per SM, each walks over its tiles
 constexpr int kMbqSums = 5;                        // wide sums in the workspace: basis 0..3, then the sum of x
 constexpr int kMbqFlushTiles = kFlushElems / (kMbqRounds * 8);  // tiles a thread of a residue pass adds between two flushes
 
@@ -323,8 +323,11 @@ __device__ inline void mbq_block_sums_deliver(MbqBlockSums* bs, MbqWorkspace* ws
 // adds the |r_j| of its tiles exactly and hands the sum to the workspace; the block that arrives last
 // rounds the total once, divides by n and leaves the workspace clean for the next pass.  No block waits
 // for another.
-template <int K>
-__global__ void __launch_bounds__(256) mbq_residue_sum_kernel(const MbqArgs a, int j) {
+// J = j, the number of coefficients already known (a template parameter: the residue of a value is then J
+// straight-line steps).
+template <int K, int J>
+__global__ void __launch_bounds__(256) mbq_residue_sum_kernel(const MbqArgs a) {
+  constexpr int j = J;
   grid_dependency_handshake();
   __shared__ MbqBlockSums s_sums;
   __shared__ float s_amax[8];
@@ -364,19 +367,42 @@ __global__ void __launch_bounds__(256) mbq_residue_sum_kernel(const MbqArgs a, i
   double acc = 0.0;
   long long irun = 0;
   int since = 0, flushes = 0;
-  for (uint64_t tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x) {
+  // the octets of the block's next tile are in flight while the current ones are added up
+  auto load_tile = [&](uint64_t tile, float (&v)[kMbqRounds][8]) {
 #pragma unroll
     for (int r = 0; r < kMbqRounds; ++r) {
       const uint64_t oct = tile * (kMbqRounds * 256) + r * 256 + tid;
       if (oct < n_oct) {
-        float v[8], res[8];
-        mbq_ld_octet(a.x, a.n, oct, v);
+        mbq_ld_octet(a.x, a.n, oct, v[r]);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[r][e] = 0.0f;
+      }
+    }
+  };
+  float cur[kMbqRounds][8], nxt[kMbqRounds][8];
+  if (blockIdx.x < a.n_tiles) load_tile(blockIdx.x, cur);
+  for (uint64_t tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x) {
+    const bool more = tile + gridDim.x < a.n_tiles;
+    if (more) load_tile(tile + gridDim.x, nxt);
+#pragma unroll
+    for (int r = 0; r < kMbqRounds; ++r) {
+      const uint64_t oct = tile * (kMbqRounds * 256) + r * 256 + tid;
+      {
+        float res[8];
         WindowCheck chk;
         chk.init();
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          mbq_residue_code<K>(alpha, v[e], j, &res[e]);
-          res[e] = (oct * 8 + e < a.n) ? fabsf(res[e]) : 0.0f;
+          float rr = cur[r][e];
+#pragma unroll
+          for (int i = 0; i < J; ++i) rr = (rr >= 0.0f) ? __fsub_rn(rr, alpha[i]) : __fadd_rn(rr, alpha[i]);
+          res[e] = fabsf(rr);
+        }
+        if (oct * 8 + 8 > a.n) {  // the octet that holds the end of the tensor: nothing past the end
+#pragma unroll
+          for (int e = 0; e < 8; ++e)
+            if (oct * 8 + e >= a.n) res[e] = 0.0f;
         }
 #pragma unroll
         for (int e = 0; e < 8; e += 2) chk.add2(res[e], res[e + 1]);
@@ -391,6 +417,12 @@ __global__ void __launch_bounds__(256) mbq_residue_sum_kernel(const MbqArgs a, i
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc += (double)res[e];
       }
+    }
+    if (more) {
+#pragma unroll
+      for (int r = 0; r < kMbqRounds; ++r)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) cur[r][e] = nxt[r][e];
     }
     if (++since == kMbqFlushTiles) {
       since = 0;
