@@ -14,7 +14,7 @@
  * Readings of points the paper leaves open (each also listed in the design notes):
  *   - one range per chunk of C consecutive values of the vectorised tensor; C >= N is the paper's
  *     per-tensor range ("Backward Quantizer": c = max|g|);
- *   - "dividing by the scaling factor" is computed as a product with inv = L/c rounded toward zero
+ *   - the division by the scaling factor is computed as a product with inv = L/c rounded toward zero
  *     (one division per chunk; rounded down so that |x * inv| <= L as in exact arithmetic); pinned
  *     against true division in the tests;
  *   - nearest rounding is IEEE round-half-to-even;
@@ -98,7 +98,7 @@ double oracle_rng_uniform(uint64_t seed, uint64_t ctr) {
  * meta[0] = s (scaling factor), meta[1] = o (offset).  i0 is the index of x[0] in the whole
  * tensor (the random-number counter).  Returns 1 if the chunk was non-finite.
  */
-/* L / r rounded TOWARD ZERO (inf if the quotient overflows).  "Dividing by the scaling factor" s = r / L
+/* L / r rounded TOWARD ZERO (inf if the quotient overflows).  The division by the scaling factor s = r / L
  * is computed as a product with this reciprocal; in the paper's exact arithmetic |g / s| never exceeds L, and
  * rounding the reciprocal down keeps that true in fp32: r * inv <= L, hence fl(d * inv) <= L for every
  * d <= r, so no value has to be clamped back into the code range.  The round-to-nearest quotient is above
@@ -258,7 +258,7 @@ void oracle_unpack(const uint32_t* payload, uint64_t n, uint32_t C, uint32_t k, 
 
 /* ---------------------------------------------------------------- dequantizer ("Backward Dequantizer") */
 
-/* ABSMAX: g_hat = g_q * s with g_q = u - 2^(k-1) ("subtracting each element by 8" for k = 4).
+/* ABSMAX: g_hat = g_q * s with g_q = u - 2^(k-1) (the shift by 8 is taken back for k = 4).
  * MINMAX: x_hat = u*s + o, product and sum rounded separately. */
 void oracle_dequantize(const uint8_t* codes, const float* meta, uint64_t n, uint32_t C, uint32_t k,
                        int range, float* xhat) {
@@ -347,7 +347,7 @@ int oracle_bitwidth_schedule(int is_backward, int n_lr_changes) {
  * ("Forward Encoder") and the receiver side (Sec. 3.4 "Forward Decoder", "Forward Dequantizer").
  *
  * x_v ~ B_v alpha with B_v in {-1,+1}^(N x k): element i carries k signs b_i0..b_i,k-1, stored as
- * the k-bit code c_i = sum_j [b_ij = +1] << j ("replace all the -1s with 0"), packed as bit planes
+ * the k-bit code c_i = sum_j [b_ij = +1] << j (a sign of -1 is stored as the bit 0), packed as bit planes
  * (plane j = basis j).  The 2^k possible values (the set P of the paper) are
  *     level(c) = (+-alpha_0) + (+-alpha_1) + ... summed in fp32 in the order j = 0..k-1.
  *
@@ -675,9 +675,9 @@ int oracle_mbq_decompress(const void* stream, uint64_t stream_bytes, uint64_t n_
 }
 
 /* ============================================================================================
- * Grouping along the batch dimension (Sec. 3.3: "the bit-wise encoder concatenates the quantized
- * data along the batch size dimension"; "Forward Encoder": consecutive elements along the first
- * dimension share an integer; "Backward Encoder": "combine two tensors along the first dimension").
+ * Grouping along the batch dimension (Sec. 3.3: the encoder works along the batch dimension; "Forward
+ * Encoder": consecutive elements along the first dimension share an integer; "Backward Encoder": codes of
+ * neighbouring samples are combined into one integer).
  *
  * The tensor is n_b x F (F = w*h*c values per sample, group_stride).  A pack group is made of the
  * 32 batch neighbours (rows 32g .. 32g+31) of one feature f instead of 32 consecutive values:

@@ -1,5 +1,5 @@
-// Pack groups along the batch dimension (Sec. 3.3: the encoder "concatenates the quantized data
-// along the batch size dimension"): the tensor is n_b x F, a group is the 32 batch neighbours
+// Pack groups along the batch dimension (Sec. 3.3, "Forward Encoder" / "Backward Encoder": values that share a
+// packed integer are neighbours along the first dimension): the tensor is n_b x F, a group is the 32 batch neighbours
 // (rows 32g..32g+31) of one feature f, group index G = g*F + f, words G*K .. G*K+K-1.
 //
 // A thread owns eight consecutive features (one octet column) and eight rows of one batch group: every
