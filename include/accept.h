@@ -97,8 +97,9 @@ typedef enum { ACCEPT_LAYOUT_INTERLEAVED = 0, ACCEPT_LAYOUT_BITPLANE = 1 } accep
  *                paper's smallest outputs need not have 8 | w*h*c).  With F % 8 == 0 (and not k = 8
  *                with BITPLANE) a thread codes eight features of eight rows with 32-byte loads;
  *                every other shape takes one feature per thread, slower but for any F.  Runs as
- *                range pass + constants + encode (workspace: 16 bytes per chunk more, as for
- *                chunk_elems > 32768).  Header word 7 carries F.
+ *                two launches: ranges, side words and constants of every chunk, then the encoder
+ *                (workspace: 16 bytes per chunk more, as for chunk_elems > 32768; with such chunks
+ *                it is a memset and four launches).  Header word 7 carries F.
  *   seed, rng_offset  STOCHASTIC only.  Element i draws
  *                  U_i = (g >> 8) * 2^-24,
  *                  g   = h * M[ctr & 3] (mod 2^32),  M = {1, 0x9E3779B1, 0x85EBCA77, 0xC2B2AE3D},

@@ -236,6 +236,54 @@ cudaError_t launch_wide_encode_for(const accept_params* p, const CodecArgs& a, c
   }
 }
 
+// Launch shape of the kernels that hold a chunk in registers (the one-launch coder, the constants pass of the
+// batch-group coder): fills the geometry fields of the arguments.  Chunks without such a geometry, the ragged
+// last chunk, and everything when the input is not 32-byte aligned get a block of the any-shape path each.
+struct ChunkLaunch { unsigned grid, block; int rounds; };
+
+ChunkLaunch chunk_launch(const accept_params* p, CodecArgs& a, bool aligned) {
+  const FastGeometry g = fast_geometry(p->chunk_elems);
+  const bool fast = g.rounds != 0 && aligned;
+  unsigned block = accept::kGenericBlock;
+  uint64_t fast_blocks = 0;
+  if (fast) {
+    a.n_fast_chunks = p->n_elems / p->chunk_elems;  // full chunks
+    a.tpc = g.tpc;
+    const bool share = g.tpc <= (uint32_t)accept::kFastBlock && accept::kFastBlock % g.tpc == 0;
+    block = share ? accept::kFastBlock : g.tpc;
+    a.chunks_per_block = share ? accept::kFastBlock / g.tpc : 1;
+    a.tpc_shift = 0;
+    while ((1u << a.tpc_shift) < g.tpc) ++a.tpc_shift;  // exact when share: tpc is then a power of two
+    fast_blocks = (a.n_fast_chunks + a.chunks_per_block - 1) / a.chunks_per_block;
+  } else {
+    a.n_fast_chunks = 0;
+    a.tpc = 32;
+    a.chunks_per_block = 1;
+  }
+  a.fast_blocks = (uint32_t)fast_blocks;
+  const uint64_t grid = fast_blocks + (a.n_chunks - a.n_fast_chunks);
+  return {(unsigned)grid, block, fast ? g.rounds : 2};
+}
+
+// Range pass and constants in one launch (chunks of at most 32768 elements): see chunk_constants_kernel.
+template <int RANGE>
+cudaError_t launch_chunk_constants(const accept_params* p, CodecArgs& a, accept::ChunkRecord* rec, cudaStream_t s) {
+  const ChunkLaunch cl = chunk_launch(p, a, true);
+  const dim3 grid(cl.grid);
+  if (cl.block > 256) {
+    switch (cl.rounds) {
+      case 4: return launch_overlapped(accept::chunk_constants_kernel<RANGE, 4, 1024>, grid, cl.block, s, a, rec);
+      case 2: return launch_overlapped(accept::chunk_constants_kernel<RANGE, 2, 1024>, grid, cl.block, s, a, rec);
+      default: return launch_overlapped(accept::chunk_constants_kernel<RANGE, 1, 1024>, grid, cl.block, s, a, rec);
+    }
+  }
+  switch (cl.rounds) {
+    case 4: return launch_overlapped(accept::chunk_constants_kernel<RANGE, 4, 256>, grid, cl.block, s, a, rec);
+    case 2: return launch_overlapped(accept::chunk_constants_kernel<RANGE, 2, 256>, grid, cl.block, s, a, rec);
+    default: return launch_overlapped(accept::chunk_constants_kernel<RANGE, 1, 256>, grid, cl.block, s, a, rec);
+  }
+}
+
 // rec_bytes = the workspace past its first 16 bytes: one record per chunk, cleared here.
 accept_status launch_wide(const accept_params* p, const CodecArgs& a, uint8_t* rec_bytes, cudaStream_t s) {
   accept::ChunkRecord* rec = reinterpret_cast<accept::ChunkRecord*>(rec_bytes);
@@ -363,21 +411,31 @@ dim3 strided_grid(const accept_params* p) {
   return dim3(gx, gy, 1);
 }
 
-accept_status launch_strided(const accept_params* p, const CodecArgs& a, uint8_t* rec_bytes, cudaStream_t s) {
+accept_status launch_strided(const accept_params* p, CodecArgs a, uint8_t* rec_bytes, cudaStream_t s) {
   accept::ChunkRecord* rec = reinterpret_cast<accept::ChunkRecord*>(rec_bytes);
-  if (cudaMemsetAsync(rec, 0, sizeof(accept::ChunkRecord) * a.n_chunks, s) != cudaSuccess) return ACCEPT_ERR_CUDA;
-  const uint64_t n_oct = (p->n_elems + 7) / 8;
-  const unsigned range_grid = (unsigned)((n_oct + 4 * 256 - 1) / (4 * 256));
-  const unsigned fin_grid = (unsigned)((a.n_chunks + 255) / 256);
+  const bool absmax = p->range == ACCEPT_RANGE_ABSMAX;
+  if (!is_wide(p)) {
+    // a block holds a chunk: ranges, side words and constants in one launch, nothing to clear
+    if (absmax) ACCEPT_LAUNCH(launch_chunk_constants<accept::kAbsMax>(p, a, rec, s));
+    else ACCEPT_LAUNCH(launch_chunk_constants<accept::kMinMax>(p, a, rec, s));
+  } else {
+    if (cudaMemsetAsync(rec, 0, sizeof(accept::ChunkRecord) * a.n_chunks, s) != cudaSuccess) return ACCEPT_ERR_CUDA;
+    const uint64_t n_oct = (p->n_elems + 7) / 8;
+    const unsigned range_grid = (unsigned)((n_oct + 4 * 256 - 1) / (4 * 256));
+    const unsigned fin_grid = (unsigned)((a.n_chunks + 255) / 256);
+    if (absmax) {
+      ACCEPT_LAUNCH(launch_overlapped(accept::wide_range_kernel<accept::kAbsMax, 4>, dim3(range_grid), 256, s, a, rec));
+      ACCEPT_LAUNCH(launch_overlapped(accept::wide_finalize_kernel<accept::kAbsMax>, dim3(fin_grid), 256, s, a, rec));
+    } else {
+      ACCEPT_LAUNCH(launch_overlapped(accept::wide_range_kernel<accept::kMinMax, 4>, dim3(range_grid), 256, s, a, rec));
+      ACCEPT_LAUNCH(launch_overlapped(accept::wide_finalize_kernel<accept::kMinMax>, dim3(fin_grid), 256, s, a, rec));
+    }
+  }
   const bool any = strided_any_shape(p);
-  if (p->range == ACCEPT_RANGE_ABSMAX) {
-    ACCEPT_LAUNCH(launch_overlapped(accept::wide_range_kernel<accept::kAbsMax, 4>, dim3(range_grid), 256, s, a, rec));
-    ACCEPT_LAUNCH(launch_overlapped(accept::wide_finalize_kernel<accept::kAbsMax>, dim3(fin_grid), 256, s, a, rec));
+  if (absmax) {
     if (any) ACCEPT_LAUNCH(launch_strided_encode_any_for<accept::kAbsMax>(p, a, rec, strided_any_grid(p), s));
     else ACCEPT_LAUNCH(launch_strided_encode_for<accept::kAbsMax>(p, a, rec, strided_grid(p), s));
   } else {
-    ACCEPT_LAUNCH(launch_overlapped(accept::wide_range_kernel<accept::kMinMax, 4>, dim3(range_grid), 256, s, a, rec));
-    ACCEPT_LAUNCH(launch_overlapped(accept::wide_finalize_kernel<accept::kMinMax>, dim3(fin_grid), 256, s, a, rec));
     if (any) ACCEPT_LAUNCH(launch_strided_encode_any_for<accept::kMinMax>(p, a, rec, strided_any_grid(p), s));
     else ACCEPT_LAUNCH(launch_strided_encode_for<accept::kMinMax>(p, a, rec, strided_grid(p), s));
   }
@@ -536,28 +594,9 @@ accept_status accept_compress(const accept_params* p, const float* d_x, void* d_
     return launch_wide(p, a, static_cast<uint8_t*>(d_ws) + 16, static_cast<cudaStream_t>(cuda_stream));
   }
 
-  const FastGeometry g = fast_geometry(p->chunk_elems);
-  const bool fast = g.rounds != 0 && is_aligned(d_x, 32);
-  unsigned block = accept::kGenericBlock;
-  uint64_t fast_blocks = 0;
-  if (fast) {
-    a.n_fast_chunks = p->n_elems / p->chunk_elems;  // full chunks
-    a.tpc = g.tpc;
-    const bool share = g.tpc <= (uint32_t)accept::kFastBlock && accept::kFastBlock % g.tpc == 0;
-    block = share ? accept::kFastBlock : g.tpc;
-    a.chunks_per_block = share ? accept::kFastBlock / g.tpc : 1;
-    a.tpc_shift = 0;
-    while ((1u << a.tpc_shift) < g.tpc) ++a.tpc_shift;  // exact when share: tpc is then a power of two
-    fast_blocks = (a.n_fast_chunks + a.chunks_per_block - 1) / a.chunks_per_block;
-  } else {
-    a.n_fast_chunks = 0;
-    a.tpc = 32;
-    a.chunks_per_block = 1;
-  }
-  a.fast_blocks = (uint32_t)fast_blocks;
-  const uint64_t grid = fast_blocks + (a.n_chunks - a.n_fast_chunks);
-  KernelFn fn = select_compress(p, fast ? g.rounds : 2, block <= 256);
-  ACCEPT_LAUNCH(launch_overlapped(fn, (unsigned)grid, block, static_cast<cudaStream_t>(cuda_stream), a));
+  const ChunkLaunch cl = chunk_launch(p, a, is_aligned(d_x, 32));
+  KernelFn fn = select_compress(p, cl.rounds, cl.block <= 256);
+  ACCEPT_LAUNCH(launch_overlapped(fn, cl.grid, cl.block, static_cast<cudaStream_t>(cuda_stream), a));
   return ACCEPT_OK;
 }
 

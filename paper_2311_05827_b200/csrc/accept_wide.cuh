@@ -115,6 +115,28 @@ __global__ void __launch_bounds__(256) wide_range_kernel(const CodecArgs a, Chun
   }
 }
 
+// The range of chunk m -> its side words (to the stream) and the encoder's constants (to the record: a = 1
+// if the chunk is non-finite; the same flag is the sign bit of inv, which is never negative otherwise, for
+// readers that fetch only inv and base).
+template <int RANGE>
+__device__ __forceinline__ void store_chunk_constants(const CodecArgs& a, ChunkRecord* rec, uint64_t m, float hi, float lo) {
+  Scale sc;
+  switch (a.k) {
+    case 2: sc = make_scale<2, RANGE>(hi, lo); break;
+    case 3: sc = make_scale<3, RANGE>(hi, lo); break;
+    case 4: sc = make_scale<4, RANGE>(hi, lo); break;
+    default: sc = make_scale<8, RANGE>(hi, lo); break;
+  }
+  st_c(a.meta + m, make_float2(sc.s, sc.o));
+  if (sc.nonfinite) atomicOr(a.status, kDevNonFinite);
+  ChunkRecord constants;
+  constants.a = sc.nonfinite ? 1u : 0u;
+  constants.b = 0u;
+  constants.inv = sc.nonfinite ? -0.0f : sc.inv;
+  constants.base = sc.base;
+  st_c(rec + m, constants);
+}
+
 // Pass 2: one thread per chunk turns the gathered range into the side words (written to the
 // stream) and the encoder's constants (written over the record: a = 1 if the chunk is non-finite;
 // the same flag is the sign bit of inv, which is never negative otherwise, for readers that fetch
@@ -132,21 +154,61 @@ __global__ void __launch_bounds__(256) wide_finalize_kernel(const CodecArgs a, C
     hi = from_sortable_key(gathered.a);
     lo = from_sortable_key(~gathered.b);
   }
-  Scale sc;
-  switch (a.k) {
-    case 2: sc = make_scale<2, RANGE>(hi, lo); break;
-    case 3: sc = make_scale<3, RANGE>(hi, lo); break;
-    case 4: sc = make_scale<4, RANGE>(hi, lo); break;
-    default: sc = make_scale<8, RANGE>(hi, lo); break;
+  store_chunk_constants<RANGE>(a, rec, m, hi, lo);
+}
+
+// Passes 1 and 2 in one launch for chunks that a block can hold in registers (the geometry of the
+// one-launch coder: a chunk of C = 8*R*tpc elements shared by tpc threads): the block reads its chunk(s),
+// reduces the range and writes side words and constants itself -- no atomics, so the records need not be
+// cleared, and no pass of its own for the constants.  Blocks past the register-resident chunks take the
+// remaining chunk(s) (the ragged last one; all of them when C has no such geometry) with a plain loop.
+template <int RANGE, int R, int BLOCK_MAX>
+__global__ void __launch_bounds__(BLOCK_MAX, BLOCK_MAX == 256 ? (R <= 2 ? 6 : 4) : 1)
+    chunk_constants_kernel(const CodecArgs a, ChunkRecord* rec) {
+  __shared__ float s_hi[32], s_lo[32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  grid_dependency_handshake();
+  Range<RANGE> rg;
+  rg.init();
+  if (blockIdx.x >= a.fast_blocks) {
+    const uint64_t m = a.n_fast_chunks + (blockIdx.x - a.fast_blocks);
+    const uint64_t i0 = m * a.chunk;
+    const uint32_t valid = (uint32_t)min((uint64_t)a.chunk, a.n - i0);
+    for (uint32_t i = tid; i < valid; i += blockDim.x) rg.add(ldg_c(a.x + i0 + i));
+    rg.warp_reduce();
+    if (lane == 0) { s_hi[warp] = rg.hi; s_lo[warp] = rg.lo; }
+    __syncthreads();
+    if (tid == 0) {
+      rg.init();
+      for (int w = 0; w < (int)(blockDim.x >> 5); ++w) rg.merge(s_hi[w], s_lo[w]);
+      store_chunk_constants<RANGE>(a, rec, m, rg.hi, rg.lo);
+    }
+    return;
   }
-  st_c(a.meta + m, make_float2(sc.s, sc.o));
-  if (sc.nonfinite) atomicOr(a.status, kDevNonFinite);
-  ChunkRecord constants;
-  constants.a = sc.nonfinite ? 1u : 0u;
-  constants.b = 0u;
-  constants.inv = sc.nonfinite ? -0.0f : sc.inv;
-  constants.base = sc.base;
-  st_c(rec + m, constants);
+  const uint32_t tpc = a.tpc;
+  const uint32_t grp = (a.chunks_per_block > 1) ? (tid >> a.tpc_shift) : 0u, gt = tid - grp * tpc;
+  uint64_t m = (uint64_t)blockIdx.x * a.chunks_per_block + grp;
+  const bool active = m < a.n_fast_chunks;  // a whole group is active or not; warps never straddle groups
+  if (!active) m = a.n_fast_chunks - 1;     // idle groups redo the last chunk's loads, store nothing
+  const uint64_t e0 = m * a.chunk;
+  float v[R][8];
+#pragma unroll
+  for (int r = 0; r < R; ++r) ld_octet(a.x + e0 + 8ull * (r * tpc + gt), v[r]);
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+#pragma unroll
+    for (int e = 0; e < 8; e += 2) rg.add2(v[r][e], v[r][e + 1]);
+  }
+  rg.warp_reduce();
+  if (tpc > 32) {
+    if (lane == 0) { s_hi[warp] = rg.hi; s_lo[warp] = rg.lo; }
+    __syncthreads();
+    const int w0 = (grp * tpc) >> 5, wn = tpc >> 5;
+    rg.init();
+    if (lane < wn) { rg.hi = s_hi[w0 + lane]; rg.lo = s_lo[w0 + lane]; }
+    rg.warp_reduce();
+  }
+  if (gt == 0 && active) store_chunk_constants<RANGE>(a, rec, m, rg.hi, rg.lo);
 }
 
 // Pass 3: quantize + pack with the constants of each octet's chunk.  A tile that lies inside the
