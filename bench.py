@@ -294,6 +294,31 @@ class Codec:
         torch.cuda.current_stream().wait_stream(side)
         return out[0], out[1]
 
+    def copy_graphed(self, launches: int = 64, replays: int = 10) -> float:
+        """ms per plain device copy of the fp32 tensor (4n bytes read, 4n written; a copy node of the graph),
+        captured and replayed like run_graphed over the same rotating buffers: what the GPU itself needs to
+        move a tensor of this size once, for the small tensors whose calls are not bound by bytes."""
+        torch = self.torch
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            self.xhat[0].copy_(self.x[0])
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for i in range(launches):
+                    self.xhat[i % self.copies].copy_(self.x[i % self.copies])
+            graph.replay()
+            side.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(side)
+            for _ in range(replays):
+                graph.replay()
+            e1.record(side)
+            side.synchronize()
+        torch.cuda.current_stream().wait_stream(side)
+        return e0.elapsed_time(e1) / (replays * launches)
+
     def status(self) -> int:
         return self.A.accept_last_device_status(self.ws)
 
@@ -459,7 +484,9 @@ def small_rows(A, torch, peak: float):
     """Tensors of 16 MB and less: the time of a call is set by launching, not by bytes.  Each kernel is
     replayed from a CUDA graph of 64 calls over rotating buffers (cold) next to an EMPTY kernel of the same
     grid launched the same way (same launch attribute, same graph): the floor.  What is left above the
-    floor is set against the time the algorithmic bytes take at the measured copy bandwidth."""
+    floor is set against the time the algorithmic bytes take at the measured copy bandwidth.  Beside them the
+    time of a plain device copy of the same fp32 tensor (a copy node in the same kind of graph), which moves
+    8n bytes where a codec call moves about 4n + kn/8: what a transfer of this size costs without any codec."""
     rows = []
     for name in ("cfg1_act", "cfg2_grad", "cfg5_64KB", "cfg5_1MB", "cfg5_16MB"):
         spec = workloads.TENSORS[name]
@@ -467,6 +494,7 @@ def small_rows(A, torch, peak: float):
         for mode in spec.headline:
             codec = Codec(A, torch, x_host, spec.chunk, mode, spec.seed)
             g_c, g_d = codec.run_graphed()
+            g_copy = codec.copy_graphed()
             blocks = -(-spec.n // 4096)
             floor_c, floor_d = null_graph_ms(A, torch, blocks, 128), null_graph_ms(A, torch, blocks, 256)
             alg = algorithmic_bytes(spec.n, spec.chunk, mode.k)
@@ -474,6 +502,7 @@ def small_rows(A, torch, peak: float):
             rows.append({"workload": name, "mode": mode_name(mode), "kbytes": spec.n * 4 / 1024,
                          "bytes_us_at_measured_copy": bytes_us,
                          "compress_us_graph": 1e3 * g_c, "decompress_us_graph": 1e3 * g_d,
+                         "plain_copy_us_graph": 1e3 * g_copy,
                          "empty_kernel_us_graph": {"blocks": blocks, "threads_128": 1e3 * floor_c, "threads_256": 1e3 * floor_d},
                          "compress_us_above_floor": 1e3 * (g_c - floor_c), "decompress_us_above_floor": 1e3 * (g_d - floor_d),
                          "compress_frac_of_measured": bytes_us / (1e3 * g_c), "decompress_frac_of_measured": bytes_us / (1e3 * g_d)})

@@ -367,63 +367,40 @@ __global__ void __launch_bounds__(256) mbq_residue_sum_kernel(const MbqArgs a) {
   double acc = 0.0;
   long long irun = 0;
   int since = 0, flushes = 0;
-  // the octets of the block's next tile are in flight while the current ones are added up
-  auto load_tile = [&](uint64_t tile, float (&v)[kMbqRounds][8]) {
+  // |r_j| of one octet into the accumulator; `valid` < 8 only for the octet that holds the end of the tensor
+  auto add_octet = [&](const float (&v)[8], int valid) {
+    float res[8];
+    WindowCheck chk;
+    chk.init();
 #pragma unroll
-    for (int r = 0; r < kMbqRounds; ++r) {
-      const uint64_t oct = tile * (kMbqRounds * 256) + r * 256 + tid;
-      if (oct < n_oct) {
-        mbq_ld_octet(a.x, a.n, oct, v[r]);
-      } else {
+    for (int e = 0; e < 8; ++e) {
+      float rr = v[e];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) v[r][e] = 0.0f;
-      }
+      // a step takes alpha_i towards zero from the side the residue is on.  Only |r| is summed here, and the
+      // steps commute with r -> -r, so -0 may go either way: subtracting alpha_i with the residue's sign bit
+      // gives the same |r| as the comparison r >= 0 that assigns the signs in the encode pass.
+      for (int i = 0; i < J; ++i) rr = __fsub_rn(rr, copysignf(alpha[i], rr));
+      res[e] = fabsf(rr);
     }
+    if (valid < 8) {  // nothing past the end
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        if (e >= valid) res[e] = 0.0f;
+    }
+#pragma unroll
+    for (int e = 0; e < 8; e += 2) chk.add2(res[e], res[e + 1]);
+    if (!chk.ok(win)) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        if (!in_window(win, res[e])) {
+          mbq_wide_add_value(&s_sums, a.status, res[e], 1u << SLOT);
+          res[e] = 0.0f;
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc += (double)res[e];
   };
-  float cur[kMbqRounds][8], nxt[kMbqRounds][8];
-  if (blockIdx.x < a.n_tiles) load_tile(blockIdx.x, cur);
-  for (uint64_t tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x) {
-    const bool more = tile + gridDim.x < a.n_tiles;
-    if (more) load_tile(tile + gridDim.x, nxt);
-#pragma unroll
-    for (int r = 0; r < kMbqRounds; ++r) {
-      const uint64_t oct = tile * (kMbqRounds * 256) + r * 256 + tid;
-      {
-        float res[8];
-        WindowCheck chk;
-        chk.init();
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          float rr = cur[r][e];
-#pragma unroll
-          for (int i = 0; i < J; ++i) rr = (rr >= 0.0f) ? __fsub_rn(rr, alpha[i]) : __fadd_rn(rr, alpha[i]);
-          res[e] = fabsf(rr);
-        }
-        if (oct * 8 + 8 > a.n) {  // the octet that holds the end of the tensor: nothing past the end
-#pragma unroll
-          for (int e = 0; e < 8; ++e)
-            if (oct * 8 + e >= a.n) res[e] = 0.0f;
-        }
-#pragma unroll
-        for (int e = 0; e < 8; e += 2) chk.add2(res[e], res[e + 1]);
-        if (!chk.ok(win)) {
-#pragma unroll
-          for (int e = 0; e < 8; ++e)
-            if (!in_window(win, res[e])) {
-              mbq_wide_add_value(&s_sums, a.status, res[e], 1u << SLOT);
-              res[e] = 0.0f;
-            }
-        }
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc += (double)res[e];
-      }
-    }
-    if (more) {
-#pragma unroll
-      for (int r = 0; r < kMbqRounds; ++r)
-#pragma unroll
-        for (int e = 0; e < 8; ++e) cur[r][e] = nxt[r][e];
-    }
+  auto tile_done = [&]() {
     if (++since == kMbqFlushTiles) {
       since = 0;
       irun += __double2ll_rn(acc * win.to_units);
@@ -433,6 +410,47 @@ __global__ void __launch_bounds__(256) mbq_residue_sum_kernel(const MbqArgs a) {
         const long long total = warp_sum_int64(irun);
         if (lane == 0) wide_add_int64(s_sums.wide[SLOT], total, win.pos);
         irun = 0;
+      }
+    }
+  };
+  // Full tiles: no guards, and the octets of the block's next tile are in flight while the current ones are
+  // added up (two sets of registers used in turn).
+  const uint64_t full_tiles = a.n / kMbqTile;
+  auto load_tile = [&](uint64_t tile, float (&v)[kMbqRounds][8]) {
+    const float* src = a.x + tile * kMbqTile + 8u * tid;
+#pragma unroll
+    for (int r = 0; r < kMbqRounds; ++r) ld_octet(src + r * (256 * 8), v[r]);
+  };
+  auto add_tile = [&](const float (&v)[kMbqRounds][8]) {
+#pragma unroll
+    for (int r = 0; r < kMbqRounds; ++r) add_octet(v[r], 8);
+    tile_done();
+  };
+  {
+    float va[kMbqRounds][8], vb[kMbqRounds][8];
+    const uint64_t stride = gridDim.x;
+    uint64_t tile = blockIdx.x;
+    if (tile < full_tiles) load_tile(tile, va);
+    while (tile < full_tiles) {
+      if (tile + stride < full_tiles) load_tile(tile + stride, vb);
+      add_tile(va);
+      tile += stride;
+      if (tile >= full_tiles) break;
+      if (tile + stride < full_tiles) load_tile(tile + stride, va);
+      add_tile(vb);
+      tile += stride;
+    }
+  }
+  // the ragged last tile, by the block whose turn it is
+  if (full_tiles < a.n_tiles && full_tiles % gridDim.x == blockIdx.x) {
+#pragma unroll 1
+    for (int r = 0; r < kMbqRounds; ++r) {
+      const uint64_t oct = full_tiles * (kMbqRounds * 256) + r * 256 + tid;
+      if (oct < n_oct) {
+        float v[8];
+        mbq_ld_octet(a.x, a.n, oct, v);
+        const uint64_t left = a.n - oct * 8;
+        add_octet(v, left >= 8 ? 8 : (int)left);
       }
     }
   }

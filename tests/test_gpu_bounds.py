@@ -103,12 +103,17 @@ def test_bounded_copy_wait_runs_out_and_the_gpu_stays_usable(k, layout):
     rows, stride, chunk = 96, 4096, 4096
     x = workloads.random_tensor(rows * stride, 12, "normal")
     p = A.Params(x.size, chunk, k, RANGE_ABSMAX, ROUND_NEAREST, layout, group_stride=stride)
+    d_x = torch.from_numpy(x).cuda()
     with gpu_util.library_variant("stall"):
         g_stream = gpu_util.guarded_stream(A, torch, p)
         g_ws = gpu_util.guarded_workspace(A, torch, p)
+        # a call of this build that stages nothing first: loading its kernels onto the GPU is not what is timed
+        warm = A.Params(x.size, chunk, k, RANGE_ABSMAX, ROUND_NEAREST, layout)
+        A.accept_compress(warm, d_x, gpu_util.guarded_stream(A, torch, warm).bytes, gpu_util.guarded_workspace(A, torch, warm).view(torch.int32))
+        torch.cuda.synchronize()
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0.record()
-        A.accept_compress(p, torch.from_numpy(x).cuda(), g_stream.bytes, g_ws.view(torch.int32))
+        A.accept_compress(p, d_x, g_stream.bytes, g_ws.view(torch.int32))
         t1.record()
         status = A.accept_last_device_status(g_ws.view(torch.int32))
         assert status == A.DEV_COPY_TIMEOUT

@@ -56,6 +56,26 @@ def check(x, chunk, stride, k, range_, round_, layout, seed=0, rng_offset=0):
     assert A.accept_parse_header(bytes(got[:32])).group_stride == stride
 
 
+@pytest.mark.parametrize("range_", [RANGE_ABSMAX, RANGE_MINMAX])
+@pytest.mark.parametrize("rows,stride,chunk", [
+    (40, 1000, 256),         # one octet per thread, a warp per chunk, four chunks per block; ragged last chunk
+    (40, 1000, 512),         # two octets per thread
+    (40, 1000, 1024),        # four octets per thread, a warp per chunk
+    (40, 1000, 12800),       # two octets per thread, 800 threads per chunk (a block of its own)
+    (48, 2048, 24576),       # four octets per thread, 768 threads per chunk
+    (48, 2048, 32768),       # the largest chunk a block holds: 1024 threads
+    (40, 1000, 4000),        # no register-resident geometry: every chunk goes through the plain loop
+    (40, 1000, 39968),       # more than 32768: ranges by atomics, constants pass (the whole tensor is 40000)
+])
+def test_strided_parity_chunk_geometries(range_, rows, stride, chunk):
+    """The one-launch pass for ranges, side words and constants under every launch shape it has, and the
+    atomics + constants passes that wider chunks take; side words and payload against the oracle."""
+    x = workloads.random_tensor(rows * stride, chunk % 97, "normal")
+    x[5] = 7.5  # not the largest magnitude of its chunk's neighbours by accident
+    check(x, chunk, stride, 4, range_, ROUND_NEAREST, LAYOUT_BITPLANE)
+    check(x, chunk, stride, 8, range_, ROUND_STOCHASTIC, LAYOUT_INTERLEAVED, seed=3, rng_offset=17)
+
+
 @pytest.mark.parametrize("mode", modes())
 @pytest.mark.parametrize("rows,stride,chunk", [
     (64, 24, 64 * 24),       # one range for the whole tensor, two full batch groups
