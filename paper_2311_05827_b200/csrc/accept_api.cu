@@ -311,8 +311,15 @@ constexpr unsigned kStridedEncodeBlocks = 3 * 148;
 
 template <int K, int LAYOUT, int RANGE>
 cudaError_t launch_strided_encode(int round, const CodecArgs& a, const accept::ChunkRecord* rec, dim3 tiles, cudaStream_t s) {
-  if (round != accept::kNearest)  // instruction bound: one tile per block, rows in registers
-    return launch_overlapped(accept::strided_encode_direct_kernel<K, LAYOUT, RANGE, accept::kStochastic>, tiles, 256, s, a, rec);
+  if (round != accept::kNearest) {  // instruction bound: one tile per block, rows in registers
+    // rows and octets start at multiples of eight values: every octet's first counter sits at the same place in its quad
+    switch ((unsigned)(a.rng_offset & 3u)) {
+      case 0: return launch_overlapped(accept::strided_encode_direct_kernel<K, LAYOUT, RANGE, accept::kStochastic, 0>, tiles, 256, s, a, rec);
+      case 1: return launch_overlapped(accept::strided_encode_direct_kernel<K, LAYOUT, RANGE, accept::kStochastic, 1>, tiles, 256, s, a, rec);
+      case 2: return launch_overlapped(accept::strided_encode_direct_kernel<K, LAYOUT, RANGE, accept::kStochastic, 2>, tiles, 256, s, a, rec);
+      default: return launch_overlapped(accept::strided_encode_direct_kernel<K, LAYOUT, RANGE, accept::kStochastic, 3>, tiles, 256, s, a, rec);
+    }
+  }
   // memory bound: persistent blocks with a staged tile, which needs more dynamic shared memory than a
   // kernel gets without opting in (the attribute is per device: set every time)
   auto fn = accept::strided_encode_kernel<K, LAYOUT, RANGE, accept::kNearest>;

@@ -323,21 +323,31 @@ __device__ __forceinline__ uint32_t lane_word_not(uint32_t h_not, uint32_t h_neg
 
 // Stochastic codes of an octet whose first counter sits at position OFF of its quad; quad_lo/key
 // address that quad.
+// (h[p] = hashed word of the p-th quad the octet touches: two quads when OFF = 0, else three)
 template <int K, int RANGE, int OFF>
-__device__ __forceinline__ void quantize_octet_stochastic(const float (&v)[8], const Scale& sc, uint32_t quad_lo,
-                                                          uint32_t key, uint32_t (&b)[8]) {
+__device__ __forceinline__ void quantize_octet_hashed(const float (&v)[8], const Scale& sc, const uint32_t (&h)[3],
+                                                      uint32_t (&b)[8]) {
   constexpr int NQ = (OFF == 0) ? 2 : 3;
   uint32_t h_not[NQ], h_neg[NQ];
 #pragma unroll
   for (int p = 0; p < NQ; ++p) {
-    const uint32_t h = Rng::quad_hash(quad_lo + p, key);
-    h_not[p] = ~h;
-    h_neg[p] = 0u - h;
+    h_not[p] = ~h[p];
+    h_neg[p] = 0u - h[p];
   }
 #pragma unroll
   for (int e = 0; e < 8; ++e)
     b[e] = quantize_stochastic_word_not<K, RANGE>(v[e], sc,
                                                   lane_word_not(h_not[(e + OFF) >> 2], h_neg[(e + OFF) >> 2], (e + OFF) & 3));
+}
+
+template <int K, int RANGE, int OFF>
+__device__ __forceinline__ void quantize_octet_stochastic(const float (&v)[8], const Scale& sc, uint32_t quad_lo,
+                                                          uint32_t key, uint32_t (&b)[8]) {
+  constexpr int NQ = (OFF == 0) ? 2 : 3;
+  uint32_t h[3] = {0u, 0u, 0u};
+#pragma unroll
+  for (int p = 0; p < NQ; ++p) h[p] = Rng::quad_hash(quad_lo + p, key);
+  quantize_octet_hashed<K, RANGE, OFF>(v, sc, h, b);
 }
 
 // Quantizes an octet.  xlo holds the codes of elements 0..3 one per byte, xhi those of 4..7.

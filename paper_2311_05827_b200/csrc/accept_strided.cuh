@@ -253,10 +253,25 @@ __global__ void __launch_bounds__(256, 3) strided_encode_kernel(const CodecArgs 
   }
 }
 
+// Hashed words of three consecutive quads when the low word of the quad index wraps among them (once in
+// 2^34 counters): each quad with the key of its own upper word.  Out of line, everything by value.
+__device__ __noinline__ uint3 strided_quad_hashes_slowly(Rng rng, uint64_t quad) {
+  // (counters wrap at 2^64, so quad indices wrap at 2^62)
+  const uint64_t q1 = (quad + 1) & 0x3FFFFFFFFFFFFFFFull, q2 = (quad + 2) & 0x3FFFFFFFFFFFFFFFull;
+  uint3 h;
+  h.x = Rng::quad_hash((uint32_t)quad, rng.key((uint32_t)(quad >> 32)));
+  h.y = Rng::quad_hash((uint32_t)q1, rng.key((uint32_t)(q1 >> 32)));
+  h.z = Rng::quad_hash((uint32_t)q2, rng.key((uint32_t)(q2 >> 32)));
+  return h;
+}
+
 // The same encoder with its rows loaded straight into registers, one tile per block: under STOCHASTIC
 // rounding the kernel is bound by instruction issue, not by bytes in flight, and the 32 resident warps
 // this form allows (against 24 with a staged tile) are worth more than the staging.
-template <int K, int LAYOUT, int RANGE, int ROUND>
+// OFF = position of every octet's first counter in its quad of counters: rows and octets start at
+// multiples of eight values, so it is rng_offset & 3 for the whole launch and the host picks the
+// instantiation (one copy of the quantizer per row instead of four behind a branch).
+template <int K, int LAYOUT, int RANGE, int ROUND, int OFF>
 __global__ void __launch_bounds__(256, 4) strided_encode_direct_kernel(const CodecArgs a, const ChunkRecord* rec) {
   grid_dependency_handshake();
   const int tid = threadIdx.x, lane = tid & 31, sub = tid & 3;
@@ -271,23 +286,27 @@ __global__ void __launch_bounds__(256, 4) strided_encode_direct_kernel(const Cod
   const uint64_t g = blockIdx.y;
   const uint64_t word0 = (g * F + (uint64_t)fo * 8) * K;  // first word of feature 8*fo of this batch group
   const Rng rng{(uint32_t)a.seed, (uint32_t)(a.seed >> 32)};
+  // key of the quads of this thread's first row; a later row almost always shares the upper word of its quad index
+  const uint64_t row0 = g * 32 + sub * 8;
+  uint32_t key_hi = (uint32_t)((a.rng_offset + row0 * F + (uint64_t)fo * 8) >> 34);
+  uint32_t key = rng.key(key_hi);
 
   uint32_t xlo[8], xhi[8];  // per row: codes of features 0..3 / 4..7
   // four rows at a time: 128 bytes in flight per thread at half the registers, so that more blocks
-  // stay resident (the kernel waits on memory, not on arithmetic)
+  // stay resident
 #pragma unroll
   for (int half = 0; half < 2; ++half) {
     float v[4][8];
     bool in[4];
-    uint4 raw[4];
+    float2 constants[4];  // {inv (its sign bit: the chunk is non-finite), base}
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
-      const uint64_t row = g * 32 + sub * 8 + half * 4 + r;
+      const uint64_t row = row0 + half * 4 + r;
       in[r] = active && row < n_rows;
       if (in[r]) {
         const uint64_t i0 = row * F + (uint64_t)fo * 8;
         ld_octet(a.x + i0, v[r]);
-        raw[r] = ldg_c(reinterpret_cast<const uint4*>(rec + chunk_of(a, i0)));
+        constants[r] = ldg_c(reinterpret_cast<const float2*>(&rec[chunk_of(a, i0)].inv));
       }
     }
 #pragma unroll
@@ -295,19 +314,38 @@ __global__ void __launch_bounds__(256, 4) strided_encode_direct_kernel(const Cod
       const int rr = half * 4 + r;
       xlo[rr] = 0; xhi[rr] = 0;
       if (in[r]) {
-        const uint64_t i0 = (g * 32 + sub * 8 + rr) * F + (uint64_t)fo * 8;
+        const uint64_t i0 = (row0 + rr) * F + (uint64_t)fo * 8;
         Scale sc;
         sc.s = 0.0f; sc.o = 0.0f;
-        sc.inv = fabsf(__uint_as_float(raw[r].z));
-        sc.base = __uint_as_float(raw[r].w);
-        sc.nonfinite = raw[r].x != 0u;
+        sc.inv = fabsf(constants[r].x);
+        sc.base = constants[r].y;
+        sc.nonfinite = (__float_as_uint(constants[r].x) >> 31) != 0u;
         if (sc.nonfinite) {
 #pragma unroll
           for (int e = 0; e < 8; ++e) v[r][e] = 0.0f;
         }
-        RngThread rt;
-        if (ROUND == kStochastic) rt.init(rng, a.rng_offset + i0, 8u);
-        quantize_octet<K, RANGE, ROUND>(v[r], sc, rng, rt, 0u, xlo[rr], xhi[rr]);
+        uint32_t b[8];
+        if (ROUND == kStochastic) {
+          const uint64_t quad = (a.rng_offset + i0) >> 2;
+          const uint32_t quad_lo = (uint32_t)quad, quad_hi = (uint32_t)(quad >> 32);
+          if (quad_hi != key_hi) { key_hi = quad_hi; key = rng.key(quad_hi); }
+          uint32_t h[3];
+          if (quad_lo <= 0xFFFFFFFFu - 4u) {
+#pragma unroll
+            for (int p = 0; p < 3; ++p) h[p] = (p < 2 || OFF != 0) ? Rng::quad_hash(quad_lo + p, key) : 0u;
+          } else {
+            const uint3 t = strided_quad_hashes_slowly(rng, quad);
+            h[0] = t.x; h[1] = t.y; h[2] = t.z;
+          }
+          quantize_octet_hashed<K, RANGE, OFF>(v[r], sc, h, b);
+          xlo[rr] = pack_bytes<3>(b[0], b[1], b[2], b[3]);
+          xhi[rr] = pack_bytes<3>(b[4], b[5], b[6], b[7]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) b[e] = quantize_nearest_word<K, RANGE>(v[r][e], sc);
+          xlo[rr] = pack_bytes<0>(b[0], b[1], b[2], b[3]);
+          xhi[rr] = pack_bytes<0>(b[4], b[5], b[6], b[7]);
+        }
       }
     }
   }

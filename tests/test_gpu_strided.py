@@ -125,6 +125,21 @@ def test_strided_parity_random_configurations(i):
     check(x, chunk, stride, k, range_, round_, layout, seed=seed, rng_offset=offset)
 
 
+@pytest.mark.parametrize("k,layout", [(2, LAYOUT_INTERLEAVED), (3, LAYOUT_BITPLANE), (4, LAYOUT_INTERLEAVED), (8, LAYOUT_INTERLEAVED)])
+@pytest.mark.parametrize("position", [0, 1, 2, 3])
+def test_strided_stochastic_counter_wraps(k, layout, position):
+    """Eq. 7 draws in the octet-per-thread encoder: the counter of every octet's first value sits at `position` of
+    its group of four counters (the host picks the kernel by it); counter ranges that cross 2^34 (the low word of
+    the group index wraps: the key changes inside an octet) and 2^64 (the counter itself wraps)."""
+    rows, stride, chunk = 40, 1536, 1024
+    x = workloads.random_tensor(rows * stride, 77 + position, "normal")
+    n = x.size
+    for offset in (position, 2 ** 34 - n // 2 - 4 + position, 2 ** 64 - n // 3 - 8 + position, 2 ** 34 - 8 + position):
+        assert offset % 4 == position
+        check(x, chunk, stride, k, RANGE_ABSMAX, ROUND_STOCHASTIC, layout, seed=0xC0FFEE + k, rng_offset=offset)
+    check(x, chunk, stride, k, RANGE_MINMAX, ROUND_STOCHASTIC, layout, seed=5, rng_offset=2 ** 34 - n // 2 + position)
+
+
 def test_strided_largest_latent_output_of_the_paper():
     """Batch 128, 8192 values per sample (the 4096 KB output of Sec. 4.3.1), per-tensor range, both encoders."""
     x = workloads.generate("cfg2_grad").reshape(32, -1)
