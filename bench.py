@@ -638,6 +638,8 @@ def run_gpu(args):
 
     if args.sweep and rank == 0:
         out["sweep"] = sweep(A, torch, peak, args)
+    if args.all_modes and rank == 0:
+        out["all_modes"] = sweep_all_modes(A, torch, peak)
 
     if rank == 0 and world == 1 and not (args.no_cpu_baseline or args.kernels_only):
         tc, td, reps = time_oracle(x_host, spec.chunk, mode, spec.seed, budget_s=args.cpu_budget)
@@ -696,6 +698,33 @@ def sweep(A, torch, peak, args):
         if name == "cfg3_act":
             rows.extend(sweep_mbq(A, torch, peak, name, spec, x_host))
             rows.append(sweep_batch_groups(A, torch, peak, name, spec, x_host))
+    return rows
+
+
+def sweep_all_modes(A, torch, peak, name="cfg5_256MB"):
+    """Every layout / k / range statistic / rounding combination the consecutive layouts have (28), at chunk sizes
+    4096 (four warps share a chunk) and 1024 (one warp per chunk), on the 256 MB tensor: isolated loops."""
+    spec = workloads.TENSORS[name]
+    x_host = workloads.generate(name)
+    rows = []
+    for layout in (0, 1):
+        for k in ((2, 4, 8) if layout == 0 else (2, 3, 4, 8)):
+            for range_ in (0, 1):
+                for round_ in (0, 1):
+                    for chunk in (4096, 1024):
+                        mode = workloads.Mode(k, range_, round_, layout)
+                        codec = Codec(A, torch, x_host, chunk, mode, spec.seed)
+                        ms_c, ms_d = codec.run_isolated(20)
+                        assert codec.status() == 0
+                        alg = algorithmic_bytes(spec.n, chunk, k)
+                        rows.append({"workload": name, "mode": mode_name(mode), "chunk": chunk, "compress_ms": ms_c,
+                                     "decompress_ms": ms_d, "compress_frac_measured": alg / ms_c / 1e6 / peak,
+                                     "decompress_frac_measured": alg / ms_d / 1e6 / peak})
+                        print("# %-12s %-34s C=%-5d c %8.4f ms %6.1f%%  d %8.4f ms %6.1f%% (of measured copy bw)" %
+                              (name, mode_name(mode), chunk, ms_c, 100 * rows[-1]["compress_frac_measured"], ms_d,
+                               100 * rows[-1]["decompress_frac_measured"]), file=sys.stderr)
+                        del codec
+                        torch.cuda.empty_cache()
     return rows
 
 
@@ -834,6 +863,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(workloads.TENSORS))
     ap.add_argument("--sweep", action="store_true", help="also time every workload's headline modes")
+    ap.add_argument("--all-modes", action="store_true",
+                    help="also time all 28 modes of the consecutive layouts on the 256 MB tensor, chunks of 4096 and 1024")
     ap.add_argument("--sweep-max-bytes", type=int, default=1 << 30)
     ap.add_argument("--sweep-only", default=None, choices=sorted(workloads.TENSORS), help="restrict the sweep to one tensor")
     ap.add_argument("--no-cpu-baseline", action="store_true")
