@@ -157,6 +157,11 @@ __global__ void __launch_bounds__(256, 3) strided_encode_kernel(const CodecArgs 
   }
   const uint32_t F = a.group_stride;
   const Rng rng{(uint32_t)a.seed, (uint32_t)(a.seed >> 32)};
+  // The eight lanes of a quarter warp read 32 bytes each at {row block 0..3} x {two neighbouring octet columns}; the row
+  // blocks are 32 bytes apart modulo 128, so the 16-byte halves of neighbouring columns would meet on the same banks two by
+  // two.  Odd columns therefore read their upper half first and hold features 4..7 where the others hold 0..3: codes do not
+  // depend on the position (nearest rounding), so the two packed words of a row are exchanged afterwards and nothing else changes.
+  const int swapped = (ROUND == kNearest) ? ((tid >> 2) & 1) : 0;
 
   const uint32_t tile0 = smem_address(s_tile);
   const uint32_t bar[2] = {smem_address(s_tile + kStridedTileBytes), smem_address(s_tile + kStridedTileBytes) + 8u};
@@ -198,7 +203,7 @@ __global__ void __launch_bounds__(256, 3) strided_encode_kernel(const CodecArgs 
         const float4* src = reinterpret_cast<const float4*>(s_tile + sub * kStridedRowBlockPitch +
                                                             (half * 4 + r) * kStridedRowBytes + (tid >> 2) * 32);
         float4 p0 = make_float4(0.f, 0.f, 0.f, 0.f), p1 = p0;
-        if (cur.in[r] && ok) { p0 = src[0]; p1 = src[1]; }
+        if (cur.in[r] && ok) { p0 = src[swapped]; p1 = src[swapped ^ 1]; }
         v[r][0] = p0.x; v[r][1] = p0.y; v[r][2] = p0.z; v[r][3] = p0.w;
         v[r][4] = p1.x; v[r][5] = p1.y; v[r][6] = p1.z; v[r][7] = p1.w;
       }
@@ -235,6 +240,7 @@ __global__ void __launch_bounds__(256, 3) strided_encode_kernel(const CodecArgs 
           RngThread rt;
           if (ROUND == kStochastic) rt.init(rng, a.rng_offset + i0, 8u);
           quantize_octet<K, RANGE, ROUND>(v[r], sc, rng, rt, 0u, xlo[rr], xhi[rr]);
+          if (swapped) { const uint32_t t_lo = xlo[rr]; xlo[rr] = xhi[rr]; xhi[rr] = t_lo; }
         }
       }
       cur = nxt;
@@ -370,8 +376,9 @@ __global__ void __launch_bounds__(256) strided_decode_kernel(const CodecArgs a) 
   // Side words of the block's 32 row segments (512 values each), fetched once per block: with chunks of at
   // least 512 values a segment touches at most two chunks, so 64 threads fetch {first chunk, next chunk} of
   // a row each and everybody reads them from shared memory (instead of eight global loads per thread).
+  // s_bound[r] = the octet column of the tile at which row r's second chunk starts (255: none).
   __shared__ float2 s_so[32][2];
-  __shared__ uint32_t s_first_chunk[32];
+  __shared__ __align__(8) uint8_t s_bound[32];
   const bool staged = a.chunk >= 8u * kStridedOctetsPerBlock;
   if (staged && tid < 64) {
     const int r = tid >> 1, which = tid & 1;
@@ -381,7 +388,10 @@ __global__ void __launch_bounds__(256) strided_decode_kernel(const CodecArgs a) 
       const uint64_t c0 = chunk_of(a, first);
       const uint64_t c = c0 + which < a.n_chunks ? c0 + which : c0;
       s_so[r][which] = ldg_c(a.meta + c);
-      if (which == 0) s_first_chunk[r] = (uint32_t)c0;
+      if (which == 0) {
+        const uint64_t to_next = (c0 + 1) * a.chunk - first;  // a multiple of 8: chunks are multiples of 32, rows and tiles of 8
+        s_bound[r] = to_next < 8u * kStridedOctetsPerBlock ? (uint8_t)(to_next / 8) : (uint8_t)255;
+      }
     }
   }
 
@@ -433,13 +443,22 @@ __global__ void __launch_bounds__(256) strided_decode_kernel(const CodecArgs a) 
     for (int r = 0; r < 4; ++r) xhi[4 + r] = o[r];
   }
   if (staged) __syncthreads();
+  uint2 bounds = make_uint2(0u, 0u);  // the boundaries of this thread's eight rows, a byte each
+  if (staged) bounds = *reinterpret_cast<const uint2*>(&s_bound[sub * 8]);
 #pragma unroll
   for (int r = 0; r < 8; ++r) {
     const uint64_t row = g * 32 + sub * 8 + r;
     if (active && row < n_rows) {
       const uint64_t i0 = row * F + (uint64_t)fo * 8;
-      const uint64_t c = chunk_of(a, i0);
-      const float2 so = staged ? s_so[sub * 8 + r][(uint32_t)c - s_first_chunk[sub * 8 + r]] : ldg_c(a.meta + c);
+      float2 so;
+      if (staged) {
+        // both candidates in one read that depends on nothing; the boundary decides
+        const float4 both = *reinterpret_cast<const float4*>(&s_so[sub * 8 + r][0]);
+        const bool second = (uint32_t)(tid >> 2) >= ((r < 4 ? bounds.x : bounds.y) >> (8 * (r & 3)) & 0xFFu);
+        so = second ? make_float2(both.z, both.w) : make_float2(both.x, both.y);
+      } else {
+        so = ldg_c(a.meta + chunk_of(a, i0));
+      }
       float out[8];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
