@@ -53,27 +53,31 @@ def algorithmic_bytes(n: int, chunk: int, k: int) -> float:
     return n * (4.0 + k / 8.0 + 8.0 / chunk)
 
 
-def kernel_sources_digest() -> str:
-    """Digest of the CUDA sources: ncu counters stored under profiles/ are quoted only for the kernels they
-    were taken from."""
+def kernel_sources_digest(files=None) -> str:
+    """Digest of CUDA sources (all of csrc/, or the named files of it) and of the build recipe: ncu counters stored
+    under profiles/ are quoted only for the kernels they were taken from."""
     import hashlib
     h = hashlib.sha256()
-    csrc = os.path.join(ROOT, "paper_2311_05827_b200", "csrc")
-    for name in sorted(os.listdir(csrc)):
-        if name.endswith((".cu", ".cuh")):
-            with open(os.path.join(csrc, name), "rb") as f:
-                h.update(name.encode() + b"\0" + f.read())
+    pkg = os.path.join(ROOT, "paper_2311_05827_b200")
+    csrc = os.path.join(pkg, "csrc")
+    names = sorted(files) if files else sorted(n for n in os.listdir(csrc) if n.endswith((".cu", ".cuh")))
+    for name in names:
+        with open(os.path.join(csrc, name), "rb") as f:
+            h.update(name.encode() + b"\0" + f.read())
+    with open(os.path.join(pkg, "build.py"), "rb") as f:
+        h.update(b"build.py\0" + f.read())
     return h.hexdigest()[:16]
 
 
 def recorded_traffic(workload: str, entry_point: str):
     """DRAM bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum) from profiles/traffic.json, or
-    None when there is no capture of this kernel on this workload or the sources have changed since."""
+    None when there is no capture of this kernel on this workload or one of the sources the row names (the files
+    the captured kernel is compiled from) has changed since."""
     try:
         with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
             table = json.load(f)
         row = table["captures"][workload][entry_point]
-        if row["sources_digest"] != kernel_sources_digest():
+        if row["sources_digest"] != kernel_sources_digest(row["sources"]):
             return None
         return float(row["dram_bytes_per_launch"])
     except Exception:
@@ -323,7 +327,10 @@ class Codec:
         return self.A.accept_last_device_status(self.ws)
 
 
-def e2e_run(A, torch, x_host, chunk, mode, seed, steps, warmup, lanes=2):
+E2E_LANES = 4  # streams the host-buffer leg alternates between
+
+
+def e2e_run(A, torch, x_host, chunk, mode, seed, steps, warmup, lanes=E2E_LANES):
     """Round trip through the host-buffer entry points: pinned host tensor in, stream to the host,
     stream back to the device, reconstructed tensor to the host; all copies inside the timed region.
     Consecutive steps alternate between `lanes` CUDA streams, each with its own staging buffers, so
@@ -599,7 +606,7 @@ def run_gpu(args):
             row["step_mcycles"] = row["step_us"]["median"] * clocks["sm_mhz"] * 1e-6  # time x median SM clock
 
     # end to end through host buffers
-    e2e_steps = max(2, min(args.steps, 6))
+    e2e_steps = max(4, min(args.steps, 12))
     if args.kernels_only:
         ms_e2e, h2d, d2h = float("nan"), 0, 0
     else:
@@ -628,7 +635,7 @@ def run_gpu(args):
                      "achieved_alone": gbs(alg, iso_c if dominant == "accept_compress" else iso_d),
                      "frac_alone": gbs(alg, iso_c if dominant == "accept_compress" else iso_d) / peak},
         "e2e": {"value": job_throughput(n, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "streams": 2, "steps": e2e_steps},
+                "d2h_bytes_per_step": d2h, "streams": E2E_LANES, "steps": e2e_steps},
         "gpu_launches": launches_timed,
         "clocks": clocks,
         "workloads": rows,

@@ -153,3 +153,34 @@ def test_workload_generator_is_sliceable_and_seeded():
     assert abs(np.abs(g).max() - 0.05) < 1e-6 and 0.0005 < (np.abs(g) == np.float32(0.05)).mean() < 0.002
     h = workloads.generate("cfg4_hidden", 0, 4096 * 4)
     assert np.allclose(h[:4096].std() / h[4096:8192].std(), 1, atol=0.2)
+
+
+def test_recorded_traffic_is_quoted_only_for_unchanged_sources(tmp_path, monkeypatch):
+    """bench.py's roofline.traffic: the stored ncu bytes are returned while the files the captured kernel is
+    compiled from are the captured ones, and None as soon as one of them differs."""
+    import json
+    import bench
+    files = ["accept_api.cu", "accept_device.cuh", "accept_kernels.cuh"]
+    table = {"captures": {"w": {"accept_compress": {"dram_bytes_per_launch": 123.0, "sources": files,
+                                                    "sources_digest": bench.kernel_sources_digest(files)},
+                                "accept_decompress": {"dram_bytes_per_launch": 5.0, "sources": files,
+                                                      "sources_digest": "0" * 16}}}}
+    (tmp_path / "profiles").mkdir()
+    (tmp_path / "profiles" / "traffic.json").write_text(json.dumps(table))
+    real_root = bench.ROOT
+    real_digest = bench.kernel_sources_digest(files)
+    monkeypatch.setattr(bench, "kernel_sources_digest", lambda f=None: real_digest)
+    monkeypatch.setattr(bench, "ROOT", str(tmp_path))
+    assert bench.recorded_traffic("w", "accept_compress") == 123.0
+    assert bench.recorded_traffic("w", "accept_decompress") is None      # another digest: the kernel has changed
+    assert bench.recorded_traffic("w", "accept_mbq_compress") is None    # never captured
+    assert bench.recorded_traffic("other", "accept_compress") is None
+    monkeypatch.setattr(bench, "ROOT", real_root)
+    monkeypatch.undo()
+    # the committed table: rows are well formed (whether they are current is the bench's business)
+    with open(os.path.join(real_root, "profiles", "traffic.json")) as f:
+        committed = json.load(f)
+    for rows in committed["captures"].values():
+        for row in rows.values():
+            assert row["dram_bytes_per_launch"] == row["read"] + row["written"]
+            assert all(os.path.exists(os.path.join(real_root, "paper_2311_05827_b200", "csrc", s)) for s in row["sources"])
