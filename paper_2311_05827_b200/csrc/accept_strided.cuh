@@ -387,7 +387,7 @@ __global__ void __launch_bounds__(256) strided_decode_kernel(const CodecArgs a) 
       const uint64_t first = row * F + (uint64_t)blockIdx.x * kStridedOctetsPerBlock * 8;
       const uint64_t c0 = chunk_of(a, first);
       const uint64_t c = c0 + which < a.n_chunks ? c0 + which : c0;
-      s_so[r][which] = ldg_c(a.meta + c);
+      s_so[(r & 7) * 4 + (r >> 3)][which] = ldg_c(a.meta + c);  // row 8 b + i at slot 4 i + b: see the read below
       if (which == 0) {
         const uint64_t to_next = (c0 + 1) * a.chunk - first;  // a multiple of 8: chunks are multiples of 32, rows and tiles of 8
         s_bound[r] = to_next < 8u * kStridedOctetsPerBlock ? (uint8_t)(to_next / 8) : (uint8_t)255;
@@ -453,7 +453,8 @@ __global__ void __launch_bounds__(256) strided_decode_kernel(const CodecArgs a) 
       float2 so;
       if (staged) {
         // both candidates in one read that depends on nothing; the boundary decides
-        const float4 both = *reinterpret_cast<const float4*>(&s_so[sub * 8 + r][0]);
+        // (the four row blocks of a warp read four neighbouring 16-byte slots: no two on the same banks)
+        const float4 both = *reinterpret_cast<const float4*>(&s_so[r * 4 + sub][0]);
         const bool second = (uint32_t)(tid >> 2) >= ((r < 4 ? bounds.x : bounds.y) >> (8 * (r & 3)) & 0xFFu);
         so = second ? make_float2(both.z, both.w) : make_float2(both.x, both.y);
       } else {
