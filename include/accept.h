@@ -94,8 +94,8 @@ typedef enum { ACCEPT_LAYOUT_INTERLEAVED = 0, ACCEPT_LAYOUT_BITPLANE = 1 } accep
  *                (row b, feature f) at position t = b % 32 of its group; rows past the last are zero
  *                bits; payload = 4*k*ceil(rows/32)*F bytes.  Ranges stay per chunk of consecutive
  *                values.  Needs n_elems % F == 0 and a 32-byte aligned input; any F >= 1 (the
- *                paper's smallest outputs need not have 8 | w*h*c).  With F % 8 == 0 (and not k = 8
- *                with BITPLANE) a thread codes eight features of eight rows with 32-byte loads;
+ *                paper's smallest outputs need not have 8 | w*h*c).  With F % 8 == 0 a thread
+ *                codes eight features of eight rows with 32-byte loads;
  *                every other shape takes one feature per thread, slower but for any F.  Runs as
  *                two launches: ranges, side words and constants of every chunk, then the encoder
  *                (workspace: 16 bytes per chunk more, as for chunk_elems > 32768; with such chunks

@@ -346,7 +346,8 @@ cudaError_t launch_strided_encode_for(const accept_params* p, const CodecArgs& a
     case 3: return launch_strided_encode<3, accept::kBitplane, RANGE>(p->round, a, rec, grid, s);
     case 4: return bp ? launch_strided_encode<4, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
                       : launch_strided_encode<4, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s);
-    default: return launch_strided_encode<8, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s);
+    default: return bp ? launch_strided_encode<8, accept::kBitplane, RANGE>(p->round, a, rec, grid, s)
+                       : launch_strided_encode<8, accept::kInterleaved, RANGE>(p->round, a, rec, grid, s);
   }
 }
 
@@ -359,15 +360,14 @@ cudaError_t launch_strided_decode_for(const accept_params* p, const CodecArgs& a
     case 3: return launch_overlapped(accept::strided_decode_kernel<3, accept::kBitplane, RANGE>, dim3(grid), 256, s, a);
     case 4: return bp ? launch_overlapped(accept::strided_decode_kernel<4, accept::kBitplane, RANGE>, dim3(grid), 256, s, a)
                       : launch_overlapped(accept::strided_decode_kernel<4, accept::kInterleaved, RANGE>, dim3(grid), 256, s, a);
-    default: return launch_overlapped(accept::strided_decode_kernel<8, accept::kInterleaved, RANGE>, dim3(grid), 256, s, a);
+    default: return bp ? launch_overlapped(accept::strided_decode_kernel<8, accept::kBitplane, RANGE>, dim3(grid), 256, s, a)
+                       : launch_overlapped(accept::strided_decode_kernel<8, accept::kInterleaved, RANGE>, dim3(grid), 256, s, a);
   }
 }
 
-// The octet-per-thread kernels need rows that start on 32-byte boundaries and have no eight-plane form; every
-// other shape goes through the feature-per-thread kernels.
-bool strided_any_shape(const accept_params* p) {
-  return p->group_stride % 8 != 0 || (p->k == 8 && p->layout == ACCEPT_LAYOUT_BITPLANE);
-}
+// The octet-per-thread kernels need rows that start on 32-byte boundaries; every other shape goes through the
+// feature-per-thread kernels.
+bool strided_any_shape(const accept_params* p) { return p->group_stride % 8 != 0; }
 
 dim3 strided_any_grid(const accept_params* p) {
   const unsigned gx = (p->group_stride + accept::kStridedAnyBlock - 1) / accept::kStridedAnyBlock;

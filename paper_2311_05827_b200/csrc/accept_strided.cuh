@@ -69,7 +69,17 @@ __device__ __forceinline__ void strided_store_tile(const CodecArgs& a, const uin
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
     uint32_t* group_words = a.payload + word0 + (uint64_t)e * K;
-    if (LAYOUT == kBitplane) {
+    if (LAYOUT == kBitplane && K == 8) {
+      // digits 0..3 and 4..7 as two sets of four planes: lane q ends up with digits q and 4 + q of all 32 rows
+      const uint32_t lo = merge_nibbles(ylo[e] & 0x0F0F0F0Fu, yhi[e] & 0x0F0F0F0Fu);
+      const uint32_t hi = merge_nibbles((ylo[e] >> 4) & 0x0F0F0F0Fu, (yhi[e] >> 4) & 0x0F0F0F0Fu);
+      const uint32_t w0 = quad_transpose(planes_nibbles(lo), lane);
+      const uint32_t w1 = quad_transpose(planes_nibbles(hi), lane);
+      if (active) {
+        st_c(group_words + sub, w0);
+        st_c(group_words + 4 + sub, w1);
+      }
+    } else if (LAYOUT == kBitplane) {
       // byte j = digit j of my eight rows; after the quad transpose lane q holds digit q of all 32 rows
       const uint32_t w = quad_transpose(planes_nibbles(merge_nibbles(ylo[e], yhi[e])), lane);
       if (active && sub < K) st_c(group_words + sub, w);
@@ -399,7 +409,14 @@ __global__ void __launch_bounds__(256) strided_decode_kernel(const CodecArgs a) 
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
     const uint32_t* group_words = a.payload + word0 + (uint64_t)e * K;
-    if (LAYOUT == kBitplane) {
+    if (LAYOUT == kBitplane && K == 8) {
+      uint32_t w0 = 0, w1 = 0;
+      if (active) { w0 = ldg_c(group_words + sub); w1 = ldg_c(group_words + 4 + sub); }
+      const uint32_t lo = planes_nibbles(quad_transpose(w0, lane));  // digits 0..3 of my eight rows
+      const uint32_t hi = planes_nibbles(quad_transpose(w1, lane));  // digits 4..7
+      ylo[e] = (lo & 0x0F0F0F0Fu) | ((hi & 0x0F0F0F0Fu) << 4);
+      yhi[e] = ((lo >> 4) & 0x0F0F0F0Fu) | (hi & 0xF0F0F0F0u);
+    } else if (LAYOUT == kBitplane) {
       uint32_t w = 0;
       if (active && sub < K) w = ldg_c(group_words + sub);
       const uint32_t nib = planes_nibbles(quad_transpose(w, lane));  // digits of my eight rows

@@ -125,7 +125,8 @@ def test_strided_parity_random_configurations(i):
     check(x, chunk, stride, k, range_, round_, layout, seed=seed, rng_offset=offset)
 
 
-@pytest.mark.parametrize("k,layout", [(2, LAYOUT_INTERLEAVED), (3, LAYOUT_BITPLANE), (4, LAYOUT_INTERLEAVED), (8, LAYOUT_INTERLEAVED)])
+@pytest.mark.parametrize("k,layout", [(2, LAYOUT_INTERLEAVED), (3, LAYOUT_BITPLANE), (4, LAYOUT_INTERLEAVED), (8, LAYOUT_INTERLEAVED),
+                                      (8, LAYOUT_BITPLANE)])
 @pytest.mark.parametrize("position", [0, 1, 2, 3])
 def test_strided_stochastic_counter_wraps(k, layout, position):
     """Eq. 7 draws in the octet-per-thread encoder: the counter of every octet's first value sits at `position` of
