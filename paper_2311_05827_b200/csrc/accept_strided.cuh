@@ -499,6 +499,69 @@ __global__ void __launch_bounds__(256) strided_decode_kernel(const CodecArgs a) 
 
 constexpr int kStridedAnyBlock = 256;  // features per block
 
+// The codes of rows 8 B .. 8 B + 7 of a thread's group into the group's words.  Bit planes: the eight codes as
+// nibbles of one word (two words for eight digits), a 4 x 8 bit-matrix transpose, and byte j of the result is
+// digit j of the eight rows: bits 8 B .. 8 B + 7 of word j.  Interleaved: K bits per row at a place fixed by B.
+template <int K, int LAYOUT, int B>
+__device__ __forceinline__ void strided_any_place(const uint32_t (&u)[8], uint32_t (&word)[K]) {
+  if (LAYOUT == kBitplane) {
+    uint32_t lo = 0, hi = 0;  // nibble form: byte b = code b in the low, code 4 + b in the high nibble
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      lo |= ((u[b] & 0xFu) | ((u[4 + b] & 0xFu) << 4)) << (8 * b);
+      if (K > 4) hi |= ((u[b] >> 4) | ((u[4 + b] >> 4) << 4)) << (8 * b);
+    }
+    lo = planes_nibbles(lo);
+    if (K > 4) hi = planes_nibbles(hi);
+#pragma unroll
+    for (int j = 0; j < K; ++j) word[j] |= (((j < 4 ? lo : hi) >> (8 * (j & 3))) & 0xFFu) << (8 * B);
+  } else {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      constexpr int per_word = 32 / K;
+      const int r = 8 * B + q;
+      word[r / per_word] |= u[q] << (K * (r % per_word));
+    }
+  }
+}
+
+template <int K, int LAYOUT, int RANGE, int ROUND, int B>
+__device__ __forceinline__ void strided_any_encode_rows(const CodecArgs& a, const ChunkRecord* rec, const Rng& rng, uint64_t g,
+                                                        uint64_t n_rows, uint32_t f, uint32_t (&word)[K]) {
+  const uint32_t F = a.group_stride;
+  const uint64_t row0 = g * 32 + 8 * B;
+  if (row0 >= n_rows) return;  // rows past the last are zero bits
+  float v[8];
+  float2 constants[8];  // {inv (its sign bit: the chunk is non-finite), base}
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    v[q] = 0.0f;
+    constants[q] = make_float2(0.0f, 0.0f);
+    if (row0 + q < n_rows) {
+      const uint64_t i = (row0 + q) * F + f;
+      v[q] = ldg_c(a.x + i);
+      constants[q] = ldg_c(reinterpret_cast<const float2*>(&rec[chunk_of(a, i)].inv));
+    }
+  }
+  uint32_t u[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    u[q] = 0u;
+    if (row0 + q < n_rows) {
+      Scale sc;
+      sc.s = 0.0f; sc.o = 0.0f;
+      sc.inv = fabsf(constants[q].x);
+      sc.base = constants[q].y;
+      sc.nonfinite = (__float_as_uint(constants[q].x) >> 31) != 0u;
+      const float x = sc.nonfinite ? 0.0f : v[q];
+      uint32_t h = 0;
+      if (ROUND == kStochastic) h = rng.word(a.rng_offset + (row0 + q) * F + f);
+      u[q] = quantize_code<K, RANGE, ROUND>(x, sc, h);
+    }
+  }
+  strided_any_place<K, LAYOUT, B>(u, word);
+}
+
 template <int K, int LAYOUT, int RANGE, int ROUND>
 __global__ void __launch_bounds__(kStridedAnyBlock) strided_encode_any_kernel(const CodecArgs a, const ChunkRecord* rec) {
   grid_dependency_handshake();
@@ -516,31 +579,65 @@ __global__ void __launch_bounds__(kStridedAnyBlock) strided_encode_any_kernel(co
   uint32_t word[K];
 #pragma unroll
   for (int j = 0; j < K; ++j) word[j] = 0u;
-#pragma unroll 4
-  for (int r = 0; r < 32; ++r) {
-    const uint64_t row = g * 32 + r;
-    if (row >= n_rows) break;  // rows past the last are zero bits
-    const uint64_t i = row * F + f;
-    float v = ldg_c(a.x + i);
-    const Scale sc = scale_from_record(rec + chunk_of(a, i));
-    if (sc.nonfinite) v = 0.0f;
-    uint32_t h = 0;
-    if (ROUND == kStochastic) h = rng.word(a.rng_offset + i);
-    const uint32_t u = quantize_code<K, RANGE, ROUND>(v, sc, h);
-    if (LAYOUT == kBitplane) {
-#pragma unroll
-      for (int j = 0; j < K; ++j) word[j] |= ((u >> j) & 1u) << r;
-    } else {
-      // the code of row r sits at bits [K r, K r + K) of the group's K words: inside one word, since K divides 32
-      constexpr int per_word = 32 / K;
-#pragma unroll
-      for (int j = 0; j < K; ++j)
-        if (r / per_word == j) word[j] |= u << (K * (r % per_word));
-    }
-  }
+  // eight rows at a time: their values and constants are requested together, then coded
+  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 0>(a, rec, rng, g, n_rows, f, word);
+  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 1>(a, rec, rng, g, n_rows, f, word);
+  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 2>(a, rec, rng, g, n_rows, f, word);
+  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 3>(a, rec, rng, g, n_rows, f, word);
   uint32_t* out = a.payload + (g * F + f) * K;
 #pragma unroll
   for (int j = 0; j < K; ++j) st_c(out + j, word[j]);
+}
+
+// The inverse of strided_any_place: the codes of rows 8 B .. 8 B + 7 out of the group's words.
+template <int K, int LAYOUT, int B>
+__device__ __forceinline__ void strided_any_take(const uint32_t (&word)[K], uint32_t (&u)[8]) {
+  if (LAYOUT == kBitplane) {
+    uint32_t lo = 0, hi = 0;  // plane form: byte j = digit j of the eight rows
+#pragma unroll
+    for (int j = 0; j < K; ++j) {
+      const uint32_t byte = (word[j] >> (8 * B)) & 0xFFu;
+      if (j < 4) lo |= byte << (8 * j);
+      else hi |= byte << (8 * (j - 4));
+    }
+    lo = planes_nibbles(lo);
+    if (K > 4) hi = planes_nibbles(hi);
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      u[b] = (lo >> (8 * b)) & 0xFu;
+      u[4 + b] = (lo >> (8 * b + 4)) & 0xFu;
+      if (K > 4) {
+        u[b] |= ((hi >> (8 * b)) & 0xFu) << 4;
+        u[4 + b] |= ((hi >> (8 * b + 4)) & 0xFu) << 4;
+      }
+    }
+  } else {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      constexpr int per_word = 32 / K;
+      const int r = 8 * B + q;
+      u[q] = (word[r / per_word] >> (K * (r % per_word))) & ((1u << K) - 1u);
+    }
+  }
+}
+
+template <int K, int LAYOUT, int RANGE, int B>
+__device__ __forceinline__ void strided_any_decode_rows(const CodecArgs& a, uint64_t g, uint64_t n_rows, uint32_t f,
+                                                        const uint32_t (&word)[K]) {
+  const uint32_t F = a.group_stride;
+  const uint64_t row0 = g * 32 + 8 * B;
+  if (row0 >= n_rows) return;
+  float2 so[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    so[q] = make_float2(0.0f, 0.0f);
+    if (row0 + q < n_rows) so[q] = ldg_c(a.meta + chunk_of(a, (row0 + q) * F + f));
+  }
+  uint32_t u[8];
+  strided_any_take<K, LAYOUT, B>(word, u);
+#pragma unroll
+  for (int q = 0; q < 8; ++q)
+    if (row0 + q < n_rows) st_c(a.xhat + (row0 + q) * F + f, dequantize_code<K, RANGE>(u[q], so[q].x, so[q].y));
 }
 
 template <int K, int LAYOUT, int RANGE>
@@ -560,24 +657,10 @@ __global__ void __launch_bounds__(kStridedAnyBlock) strided_decode_any_kernel(co
   uint32_t word[K];
 #pragma unroll
   for (int j = 0; j < K; ++j) word[j] = ldg_c(in + j);
-#pragma unroll 4
-  for (int r = 0; r < 32; ++r) {
-    const uint64_t row = g * 32 + r;
-    if (row >= n_rows) break;
-    const uint64_t i = row * F + f;
-    uint32_t u = 0;
-    if (LAYOUT == kBitplane) {
-#pragma unroll
-      for (int j = 0; j < K; ++j) u |= ((word[j] >> r) & 1u) << j;
-    } else {
-      constexpr int per_word = 32 / K;
-#pragma unroll
-      for (int j = 0; j < K; ++j)
-        if (r / per_word == j) u = (word[j] >> (K * (r % per_word))) & ((1u << K) - 1u);
-    }
-    const float2 so = ldg_c(a.meta + chunk_of(a, i));
-    st_c(a.xhat + i, dequantize_code<K, RANGE>(u, so.x, so.y));
-  }
+  strided_any_decode_rows<K, LAYOUT, RANGE, 0>(a, g, n_rows, f, word);
+  strided_any_decode_rows<K, LAYOUT, RANGE, 1>(a, g, n_rows, f, word);
+  strided_any_decode_rows<K, LAYOUT, RANGE, 2>(a, g, n_rows, f, word);
+  strided_any_decode_rows<K, LAYOUT, RANGE, 3>(a, g, n_rows, f, word);
 }
 
 }  // namespace accept
