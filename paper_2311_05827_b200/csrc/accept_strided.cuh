@@ -525,29 +525,35 @@ __device__ __forceinline__ void strided_any_place(const uint32_t (&u)[8], uint32
   }
 }
 
-template <int K, int LAYOUT, int RANGE, int ROUND, int B>
-__device__ __forceinline__ void strided_any_encode_rows(const CodecArgs& a, const ChunkRecord* rec, const Rng& rng, uint64_t g,
-                                                        uint64_t n_rows, uint32_t f, uint32_t (&word)[K]) {
+// Chunk of element e; POW2: the chunk size is a power of two (decided once per thread, not per element).
+template <bool POW2>
+__device__ __forceinline__ uint64_t strided_any_chunk(const CodecArgs& a, uint64_t e) {
+  return POW2 ? (e >> a.chunk_shift) : (e / a.chunk);
+}
+
+// Rows 8 B .. 8 B + 7 of the thread's group.  FULL: all eight exist (no guards).
+template <int K, int LAYOUT, int RANGE, int ROUND, int B, bool POW2, bool FULL>
+__device__ __forceinline__ void strided_any_encode_eight(const CodecArgs& a, const ChunkRecord* rec, const Rng& rng, uint64_t row0,
+                                                         uint64_t n_rows, uint32_t f, uint32_t (&word)[K]) {
   const uint32_t F = a.group_stride;
-  const uint64_t row0 = g * 32 + 8 * B;
-  if (row0 >= n_rows) return;  // rows past the last are zero bits
+  const uint64_t i0 = row0 * F + f;
   float v[8];
   float2 constants[8];  // {inv (its sign bit: the chunk is non-finite), base}
 #pragma unroll
   for (int q = 0; q < 8; ++q) {
     v[q] = 0.0f;
     constants[q] = make_float2(0.0f, 0.0f);
-    if (row0 + q < n_rows) {
-      const uint64_t i = (row0 + q) * F + f;
+    if (FULL || row0 + q < n_rows) {
+      const uint64_t i = i0 + (uint64_t)q * F;
       v[q] = ldg_c(a.x + i);
-      constants[q] = ldg_c(reinterpret_cast<const float2*>(&rec[chunk_of(a, i)].inv));
+      constants[q] = ldg_c(reinterpret_cast<const float2*>(&rec[strided_any_chunk<POW2>(a, i)].inv));
     }
   }
   uint32_t u[8];
 #pragma unroll
   for (int q = 0; q < 8; ++q) {
     u[q] = 0u;
-    if (row0 + q < n_rows) {
+    if (FULL || row0 + q < n_rows) {
       Scale sc;
       sc.s = 0.0f; sc.o = 0.0f;
       sc.inv = fabsf(constants[q].x);
@@ -555,11 +561,29 @@ __device__ __forceinline__ void strided_any_encode_rows(const CodecArgs& a, cons
       sc.nonfinite = (__float_as_uint(constants[q].x) >> 31) != 0u;
       const float x = sc.nonfinite ? 0.0f : v[q];
       uint32_t h = 0;
-      if (ROUND == kStochastic) h = rng.word(a.rng_offset + (row0 + q) * F + f);
+      if (ROUND == kStochastic) h = rng.word(a.rng_offset + i0 + (uint64_t)q * F);
       u[q] = quantize_code<K, RANGE, ROUND>(x, sc, h);
     }
   }
   strided_any_place<K, LAYOUT, B>(u, word);
+}
+
+template <int K, int LAYOUT, int RANGE, int ROUND, int B, bool POW2>
+__device__ __forceinline__ void strided_any_encode_rows(const CodecArgs& a, const ChunkRecord* rec, const Rng& rng, uint64_t g,
+                                                        uint64_t n_rows, uint32_t f, uint32_t (&word)[K]) {
+  const uint64_t row0 = g * 32 + 8 * B;
+  if (row0 >= n_rows) return;  // rows past the last are zero bits
+  if (row0 + 8 <= n_rows) strided_any_encode_eight<K, LAYOUT, RANGE, ROUND, B, POW2, true>(a, rec, rng, row0, n_rows, f, word);
+  else strided_any_encode_eight<K, LAYOUT, RANGE, ROUND, B, POW2, false>(a, rec, rng, row0, n_rows, f, word);
+}
+
+template <int K, int LAYOUT, int RANGE, int ROUND, bool POW2>
+__device__ __forceinline__ void strided_any_encode_group(const CodecArgs& a, const ChunkRecord* rec, const Rng& rng, uint64_t g,
+                                                         uint64_t n_rows, uint32_t f, uint32_t (&word)[K]) {
+  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 0, POW2>(a, rec, rng, g, n_rows, f, word);
+  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 1, POW2>(a, rec, rng, g, n_rows, f, word);
+  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 2, POW2>(a, rec, rng, g, n_rows, f, word);
+  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 3, POW2>(a, rec, rng, g, n_rows, f, word);
 }
 
 template <int K, int LAYOUT, int RANGE, int ROUND>
@@ -580,13 +604,21 @@ __global__ void __launch_bounds__(kStridedAnyBlock) strided_encode_any_kernel(co
 #pragma unroll
   for (int j = 0; j < K; ++j) word[j] = 0u;
   // eight rows at a time: their values and constants are requested together, then coded
-  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 0>(a, rec, rng, g, n_rows, f, word);
-  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 1>(a, rec, rng, g, n_rows, f, word);
-  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 2>(a, rec, rng, g, n_rows, f, word);
-  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 3>(a, rec, rng, g, n_rows, f, word);
+  if (a.chunk_shift >= 0) strided_any_encode_group<K, LAYOUT, RANGE, ROUND, true>(a, rec, rng, g, n_rows, f, word);
+  else strided_any_encode_group<K, LAYOUT, RANGE, ROUND, false>(a, rec, rng, g, n_rows, f, word);
+  // (the payload starts 16-byte aligned and a group is K words: whole groups move as one access where K allows)
   uint32_t* out = a.payload + (g * F + f) * K;
+  if (K == 4) {
+    st_c(reinterpret_cast<uint4*>(out), make_uint4(word[0], word[1], word[2 % K], word[3 % K]));
+  } else if (K == 8) {
+    st_c(reinterpret_cast<uint4*>(out), make_uint4(word[0], word[1], word[2 % K], word[3 % K]));
+    st_c(reinterpret_cast<uint4*>(out) + 1, make_uint4(word[4 % K], word[5 % K], word[6 % K], word[7 % K]));
+  } else if (K == 2) {
+    st_c(reinterpret_cast<uint2*>(out), make_uint2(word[0], word[1]));
+  } else {
 #pragma unroll
-  for (int j = 0; j < K; ++j) st_c(out + j, word[j]);
+    for (int j = 0; j < K; ++j) st_c(out + j, word[j]);
+  }
 }
 
 // The inverse of strided_any_place: the codes of rows 8 B .. 8 B + 7 out of the group's words.
@@ -621,23 +653,40 @@ __device__ __forceinline__ void strided_any_take(const uint32_t (&word)[K], uint
   }
 }
 
-template <int K, int LAYOUT, int RANGE, int B>
-__device__ __forceinline__ void strided_any_decode_rows(const CodecArgs& a, uint64_t g, uint64_t n_rows, uint32_t f,
-                                                        const uint32_t (&word)[K]) {
+template <int K, int LAYOUT, int RANGE, int B, bool POW2, bool FULL>
+__device__ __forceinline__ void strided_any_decode_eight(const CodecArgs& a, uint64_t row0, uint64_t n_rows, uint32_t f,
+                                                         const uint32_t (&word)[K]) {
   const uint32_t F = a.group_stride;
-  const uint64_t row0 = g * 32 + 8 * B;
-  if (row0 >= n_rows) return;
+  const uint64_t i0 = row0 * F + f;
   float2 so[8];
 #pragma unroll
   for (int q = 0; q < 8; ++q) {
     so[q] = make_float2(0.0f, 0.0f);
-    if (row0 + q < n_rows) so[q] = ldg_c(a.meta + chunk_of(a, (row0 + q) * F + f));
+    if (FULL || row0 + q < n_rows) so[q] = ldg_c(a.meta + strided_any_chunk<POW2>(a, i0 + (uint64_t)q * F));
   }
   uint32_t u[8];
   strided_any_take<K, LAYOUT, B>(word, u);
 #pragma unroll
   for (int q = 0; q < 8; ++q)
-    if (row0 + q < n_rows) st_c(a.xhat + (row0 + q) * F + f, dequantize_code<K, RANGE>(u[q], so[q].x, so[q].y));
+    if (FULL || row0 + q < n_rows) st_c(a.xhat + i0 + (uint64_t)q * F, dequantize_code<K, RANGE>(u[q], so[q].x, so[q].y));
+}
+
+template <int K, int LAYOUT, int RANGE, int B, bool POW2>
+__device__ __forceinline__ void strided_any_decode_rows(const CodecArgs& a, uint64_t g, uint64_t n_rows, uint32_t f,
+                                                        const uint32_t (&word)[K]) {
+  const uint64_t row0 = g * 32 + 8 * B;
+  if (row0 >= n_rows) return;
+  if (row0 + 8 <= n_rows) strided_any_decode_eight<K, LAYOUT, RANGE, B, POW2, true>(a, row0, n_rows, f, word);
+  else strided_any_decode_eight<K, LAYOUT, RANGE, B, POW2, false>(a, row0, n_rows, f, word);
+}
+
+template <int K, int LAYOUT, int RANGE, bool POW2>
+__device__ __forceinline__ void strided_any_decode_group(const CodecArgs& a, uint64_t g, uint64_t n_rows, uint32_t f,
+                                                         const uint32_t (&word)[K]) {
+  strided_any_decode_rows<K, LAYOUT, RANGE, 0, POW2>(a, g, n_rows, f, word);
+  strided_any_decode_rows<K, LAYOUT, RANGE, 1, POW2>(a, g, n_rows, f, word);
+  strided_any_decode_rows<K, LAYOUT, RANGE, 2, POW2>(a, g, n_rows, f, word);
+  strided_any_decode_rows<K, LAYOUT, RANGE, 3, POW2>(a, g, n_rows, f, word);
 }
 
 template <int K, int LAYOUT, int RANGE>
@@ -655,12 +704,22 @@ __global__ void __launch_bounds__(kStridedAnyBlock) strided_decode_any_kernel(co
   const uint64_t g = blockIdx.y;
   const uint32_t* in = a.payload + (g * F + f) * K;
   uint32_t word[K];
+  if (K == 4) {
+    const uint4 w = ldg_c(reinterpret_cast<const uint4*>(in));
+    word[0] = w.x; word[1] = w.y; word[2 % K] = w.z; word[3 % K] = w.w;
+  } else if (K == 8) {
+    const uint4 w = ldg_c(reinterpret_cast<const uint4*>(in)), x = ldg_c(reinterpret_cast<const uint4*>(in) + 1);
+    word[0] = w.x; word[1] = w.y; word[2 % K] = w.z; word[3 % K] = w.w;
+    word[4 % K] = x.x; word[5 % K] = x.y; word[6 % K] = x.z; word[7 % K] = x.w;
+  } else if (K == 2) {
+    const uint2 w = ldg_c(reinterpret_cast<const uint2*>(in));
+    word[0] = w.x; word[1] = w.y;
+  } else {
 #pragma unroll
-  for (int j = 0; j < K; ++j) word[j] = ldg_c(in + j);
-  strided_any_decode_rows<K, LAYOUT, RANGE, 0>(a, g, n_rows, f, word);
-  strided_any_decode_rows<K, LAYOUT, RANGE, 1>(a, g, n_rows, f, word);
-  strided_any_decode_rows<K, LAYOUT, RANGE, 2>(a, g, n_rows, f, word);
-  strided_any_decode_rows<K, LAYOUT, RANGE, 3>(a, g, n_rows, f, word);
+    for (int j = 0; j < K; ++j) word[j] = ldg_c(in + j);
+  }
+  if (a.chunk_shift >= 0) strided_any_decode_group<K, LAYOUT, RANGE, true>(a, g, n_rows, f, word);
+  else strided_any_decode_group<K, LAYOUT, RANGE, false>(a, g, n_rows, f, word);
 }
 
 }  // namespace accept
