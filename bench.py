@@ -705,6 +705,9 @@ def sweep(A, torch, peak, args):
         if name == "cfg3_act":
             rows.extend(sweep_mbq(A, torch, peak, name, spec, x_host))
             rows.append(sweep_batch_groups(A, torch, peak, name, spec, x_host))
+            # eight bit planes, and values per sample that are not a multiple of eight (the feature-per-thread kernels)
+            rows.append(sweep_batch_groups(A, torch, peak, name, spec, x_host, mode=workloads.Mode(8, 0, 0, 1)))
+            rows.append(sweep_batch_groups(A, torch, peak, name, spec, x_host, stride=spec.n // spec.shape[0] - 4))
     return rows
 
 
@@ -735,15 +738,18 @@ def sweep_all_modes(A, torch, peak, name="cfg5_256MB"):
     return rows
 
 
-def sweep_batch_groups(A, torch, peak, name, spec, x_host):
-    """Pack groups along the batch dimension (the paper's grouping): the tensor as batch x (values per sample)."""
-    mode = spec.headline[0]
-    stride = spec.n // spec.shape[0]
-    p = A.Params(spec.n, spec.chunk, mode.k, mode.range, mode.round, mode.layout, spec.seed, 0, group_stride=stride)
+def sweep_batch_groups(A, torch, peak, name, spec, x_host, mode=None, stride=None):
+    """Pack groups along the batch dimension (the paper's grouping): the tensor as batch x (values per sample).
+    stride: values per sample if not the tensor's own (the first batch x stride values are coded then)."""
+    mode = mode or spec.headline[0]
+    stride = stride or spec.n // spec.shape[0]
+    n = spec.shape[0] * stride
+    x_host = x_host[:n]
+    p = A.Params(n, spec.chunk, mode.k, mode.range, mode.round, mode.layout, spec.seed, 0, group_stride=stride)
     copies = 2
     x = [torch.from_numpy(x_host).cuda() for _ in range(copies)]
     st = [A.new_stream_buffer(p) for _ in range(copies)]
-    xh = [torch.empty(spec.n, dtype=torch.float32, device="cuda") for _ in range(copies)]
+    xh = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(copies)]
     ws = A.new_workspace(p)
     times = []
     for fn in (lambda j: A.accept_compress(p, x[j], st[j], ws), lambda j: A.accept_decompress(p, st[j], xh[j], ws)):
@@ -759,12 +765,12 @@ def sweep_batch_groups(A, torch, peak, name, spec, x_host):
         times.append(e0.elapsed_time(e1) / 20)
     assert A.accept_last_device_status(ws) == 0
     ms_c, ms_d = times
-    alg_c, alg_d = spec.n * (8.0 + mode.k / 8.0), spec.n * (4.0 + mode.k / 8.0)
-    row = {"workload": name, "mode": mode_name(mode) + "-batch-groups", "mbytes": spec.n * 4 / 2 ** 20, "copies": copies,
+    alg_c, alg_d = n * (8.0 + mode.k / 8.0), n * (4.0 + mode.k / 8.0)
+    row = {"workload": name, "mode": mode_name(mode) + "-batch-groups", "mbytes": n * 4 / 2 ** 20, "copies": copies,
            "group_stride": stride, "compress_ms": ms_c, "decompress_ms": ms_d, "compress_bytes_per_element": 8.0 + mode.k / 8.0,
            "compress_frac_measured": alg_c / ms_c / 1e6 / peak, "decompress_frac_measured": alg_d / ms_d / 1e6 / peak}
     print("# %-12s %-34s c %8.4f ms %6.1f%%  d %8.4f ms %6.1f%% (of measured copy bw)" %
-          (name, ("k%d-batch-groups-%dx%d" % (mode.k, spec.shape[0], stride))[:34], ms_c, 100 * row["compress_frac_measured"],
+          (name, ("k%d%s-batch-groups-%dx%d" % (mode.k, "bp" if mode.layout else "il", spec.shape[0], stride))[:34], ms_c, 100 * row["compress_frac_measured"],
            ms_d, 100 * row["decompress_frac_measured"]), file=sys.stderr)
     return row
 
