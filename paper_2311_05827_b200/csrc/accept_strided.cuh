@@ -531,10 +531,24 @@ __device__ __forceinline__ uint64_t strided_any_chunk(const CodecArgs& a, uint64
   return POW2 ? (e >> a.chunk_shift) : (e / a.chunk);
 }
 
+// The random word of counter ctr with the key of its upper word kept from one counter to the next (a thread's
+// counters are F apart: the upper 32 bits of the group index change once in 2^34 counters).
+struct StridedAnyKey {
+  uint32_t hi, key;
+};
+__device__ __forceinline__ uint32_t strided_any_word(const Rng& rng, StridedAnyKey& k, uint64_t ctr) {
+  const uint64_t quad = ctr >> 2;
+  const uint32_t hi = (uint32_t)(quad >> 32);
+  if (hi != k.hi) { k.hi = hi; k.key = rng.key(hi); }
+  const uint32_t h = Rng::quad_hash((uint32_t)quad, k.key);
+  const int m = (int)(ctr & 3);
+  return m == 0 ? h : h * (m == 1 ? 0x9E3779B1u : (m == 2 ? 0x85EBCA77u : 0xC2B2AE3Du));
+}
+
 // Rows 8 B .. 8 B + 7 of the thread's group.  FULL: all eight exist (no guards).
 template <int K, int LAYOUT, int RANGE, int ROUND, int B, bool POW2, bool FULL>
-__device__ __forceinline__ void strided_any_encode_eight(const CodecArgs& a, const ChunkRecord* rec, const Rng& rng, uint64_t row0,
-                                                         uint64_t n_rows, uint32_t f, uint32_t (&word)[K]) {
+__device__ __forceinline__ void strided_any_encode_eight(const CodecArgs& a, const ChunkRecord* rec, const Rng& rng, StridedAnyKey& key,
+                                                         uint64_t row0, uint64_t n_rows, uint32_t f, uint32_t (&word)[K]) {
   const uint32_t F = a.group_stride;
   const uint64_t i0 = row0 * F + f;
   float v[8];
@@ -561,7 +575,7 @@ __device__ __forceinline__ void strided_any_encode_eight(const CodecArgs& a, con
       sc.nonfinite = (__float_as_uint(constants[q].x) >> 31) != 0u;
       const float x = sc.nonfinite ? 0.0f : v[q];
       uint32_t h = 0;
-      if (ROUND == kStochastic) h = rng.word(a.rng_offset + i0 + (uint64_t)q * F);
+      if (ROUND == kStochastic) h = strided_any_word(rng, key, a.rng_offset + i0 + (uint64_t)q * F);
       u[q] = quantize_code<K, RANGE, ROUND>(x, sc, h);
     }
   }
@@ -569,21 +583,24 @@ __device__ __forceinline__ void strided_any_encode_eight(const CodecArgs& a, con
 }
 
 template <int K, int LAYOUT, int RANGE, int ROUND, int B, bool POW2>
-__device__ __forceinline__ void strided_any_encode_rows(const CodecArgs& a, const ChunkRecord* rec, const Rng& rng, uint64_t g,
-                                                        uint64_t n_rows, uint32_t f, uint32_t (&word)[K]) {
+__device__ __forceinline__ void strided_any_encode_rows(const CodecArgs& a, const ChunkRecord* rec, const Rng& rng, StridedAnyKey& key,
+                                                        uint64_t g, uint64_t n_rows, uint32_t f, uint32_t (&word)[K]) {
   const uint64_t row0 = g * 32 + 8 * B;
   if (row0 >= n_rows) return;  // rows past the last are zero bits
-  if (row0 + 8 <= n_rows) strided_any_encode_eight<K, LAYOUT, RANGE, ROUND, B, POW2, true>(a, rec, rng, row0, n_rows, f, word);
-  else strided_any_encode_eight<K, LAYOUT, RANGE, ROUND, B, POW2, false>(a, rec, rng, row0, n_rows, f, word);
+  if (row0 + 8 <= n_rows) strided_any_encode_eight<K, LAYOUT, RANGE, ROUND, B, POW2, true>(a, rec, rng, key, row0, n_rows, f, word);
+  else strided_any_encode_eight<K, LAYOUT, RANGE, ROUND, B, POW2, false>(a, rec, rng, key, row0, n_rows, f, word);
 }
 
 template <int K, int LAYOUT, int RANGE, int ROUND, bool POW2>
 __device__ __forceinline__ void strided_any_encode_group(const CodecArgs& a, const ChunkRecord* rec, const Rng& rng, uint64_t g,
                                                          uint64_t n_rows, uint32_t f, uint32_t (&word)[K]) {
-  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 0, POW2>(a, rec, rng, g, n_rows, f, word);
-  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 1, POW2>(a, rec, rng, g, n_rows, f, word);
-  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 2, POW2>(a, rec, rng, g, n_rows, f, word);
-  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 3, POW2>(a, rec, rng, g, n_rows, f, word);
+  StridedAnyKey key;
+  key.hi = (uint32_t)((a.rng_offset + g * 32 * a.group_stride + f) >> 34);
+  key.key = rng.key(key.hi);
+  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 0, POW2>(a, rec, rng, key, g, n_rows, f, word);
+  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 1, POW2>(a, rec, rng, key, g, n_rows, f, word);
+  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 2, POW2>(a, rec, rng, key, g, n_rows, f, word);
+  strided_any_encode_rows<K, LAYOUT, RANGE, ROUND, 3, POW2>(a, rec, rng, key, g, n_rows, f, word);
 }
 
 template <int K, int LAYOUT, int RANGE, int ROUND>
