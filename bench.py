@@ -84,6 +84,24 @@ def recorded_traffic(workload: str, entry_point: str):
         return None
 
 
+def recorded_instructions(workload: str, kernel: str):
+    """Executed thread-instructions per element of an instruction-bound kernel (ncu smsp__inst_executed.sum x 32 / n)
+    from profiles/traffic.json, under the same rule as recorded_traffic; None if not captured or changed since."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            row = json.load(f)["instructions"][workload][kernel]
+        if row["sources_digest"] != kernel_sources_digest(row["sources"]):
+            return None
+        return float(row["thread_instructions_per_element"])
+    except Exception:
+        return None
+
+
+# Issue rate of a B200: 148 SMs x 4 schedulers x one warp instruction of 32 lanes per cycle, at the SM clock.
+def issue_peak_per_second(sm_mhz: float) -> float:
+    return 148 * 4 * 32 * sm_mhz * 1e6
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -824,6 +842,14 @@ def sweep_mbq(A, torch, peak, name, spec, x_host):
         rows.append({"workload": name, "mode": "mbq-k%d" % k, "mbytes": n * 4 / 2 ** 20, "copies": copies,
                      "init_ms": ms_i, "compress_ms": ms_c, "decompress_ms": ms_d,
                      "compress_frac_measured": alg / ms_c / 1e6 / peak, "decompress_frac_measured": alg / ms_d / 1e6 / peak})
+        # the encode pass is bound by instruction issue, not by HBM: its second roofline is the issue rate of the
+        # SMs at the nominal maximum clock, with the instruction count of the ncu capture
+        ipe = recorded_instructions(name, "mbq_encode_kernel<%d>" % k)
+        if ipe is not None:
+            achieved = ipe * n / (ms_c * 1e-3)
+            rows[-1]["compress_roofline_alu"] = {"bound": "alu", "unit": "thread-instructions/s", "achieved": achieved,
+                                                 "peak": issue_peak_per_second(1965.0), "frac": achieved / issue_peak_per_second(1965.0),
+                                                 "thread_instructions_per_element": ipe}
         print("# %-12s %-34s c %8.4f ms %6.1f%%  d %8.4f ms %6.1f%% (of measured copy bw); residue init %.4f ms" %
               (name, "mbq-k%d" % k, ms_c, 100 * rows[-1]["compress_frac_measured"], ms_d,
                100 * rows[-1]["decompress_frac_measured"], ms_i), file=sys.stderr)
