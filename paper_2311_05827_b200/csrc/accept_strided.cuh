@@ -287,14 +287,11 @@ __device__ __noinline__ uint3 strided_quad_hashes_slowly(Rng rng, uint64_t quad)
 // OFF = position of every octet's first counter in its quad of counters: rows and octets start at
 // multiples of eight values, so it is rng_offset & 3 for the whole launch and the host picks the
 // instantiation (one copy of the quantizer per row instead of four behind a branch).
-template <int K, int LAYOUT, int RANGE, int ROUND, int OFF>
-__global__ void __launch_bounds__(256, 4) strided_encode_direct_kernel(const CodecArgs a, const ChunkRecord* rec) {
-  grid_dependency_handshake();
+// FULL: all 32 rows and all 64 feature octets of the block's tile exist and the chunk size is a power of two
+// (decided once per block): no guards, chunk indices by a shift.
+template <int K, int LAYOUT, int RANGE, int ROUND, int OFF, bool FULL>
+__device__ __forceinline__ void strided_encode_direct_tile(const CodecArgs& a, const ChunkRecord* rec) {
   const int tid = threadIdx.x, lane = tid & 31, sub = tid & 3;
-  if (blockIdx.x == 0 && blockIdx.y == 0 && tid < 8) {
-    st_c(a.header + tid, header_word(a, tid));
-    if ((a.n_chunks & 1) && tid < 2) st_c(reinterpret_cast<uint32_t*>(a.meta + a.n_chunks) + tid, 0u);
-  }
   const uint32_t F = a.group_stride;
   const uint64_t n_rows = a.n / F;
   const uint32_t fo = blockIdx.x * kStridedOctetsPerBlock + (tid >> 2);  // feature octet
@@ -318,11 +315,12 @@ __global__ void __launch_bounds__(256, 4) strided_encode_direct_kernel(const Cod
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
       const uint64_t row = row0 + half * 4 + r;
-      in[r] = active && row < n_rows;
+      in[r] = FULL || (active && row < n_rows);
       if (in[r]) {
         const uint64_t i0 = row * F + (uint64_t)fo * 8;
         ld_octet(a.x + i0, v[r]);
-        constants[r] = ldg_c(reinterpret_cast<const float2*>(&rec[chunk_of(a, i0)].inv));
+        const uint64_t m = FULL ? (i0 >> a.chunk_shift) : chunk_of(a, i0);
+        constants[r] = ldg_c(reinterpret_cast<const float2*>(&rec[m].inv));
       }
     }
 #pragma unroll
@@ -366,6 +364,21 @@ __global__ void __launch_bounds__(256, 4) strided_encode_direct_kernel(const Cod
     }
   }
   strided_store_tile<K, LAYOUT>(a, xlo, xhi, word0, active, sub, lane);
+}
+
+template <int K, int LAYOUT, int RANGE, int ROUND, int OFF>
+__global__ void __launch_bounds__(256, 4) strided_encode_direct_kernel(const CodecArgs a, const ChunkRecord* rec) {
+  grid_dependency_handshake();
+  const int tid = threadIdx.x;
+  if (blockIdx.x == 0 && blockIdx.y == 0 && tid < 8) {
+    st_c(a.header + tid, header_word(a, tid));
+    if ((a.n_chunks & 1) && tid < 2) st_c(reinterpret_cast<uint32_t*>(a.meta + a.n_chunks) + tid, 0u);
+  }
+  const uint64_t n_rows = a.n / a.group_stride;
+  const bool full = a.chunk_shift >= 0 && ((uint64_t)blockIdx.y + 1) * 32 <= n_rows &&
+                    ((uint64_t)blockIdx.x + 1) * kStridedOctetsPerBlock * 8 <= a.group_stride;
+  if (full) strided_encode_direct_tile<K, LAYOUT, RANGE, ROUND, OFF, true>(a, rec);
+  else strided_encode_direct_tile<K, LAYOUT, RANGE, ROUND, OFF, false>(a, rec);
 }
 
 template <int K, int LAYOUT, int RANGE>
