@@ -129,6 +129,8 @@ template <int RANGE>
 struct StridedRowConstants {
   float inv[4], base[4];
   bool in[4];
+  // ALLFULL: every tile of the launch has all its rows and octets and the chunk size is a power of two
+  template <bool ALLFULL>
   __device__ __forceinline__ void fetch(const CodecArgs& a, const ChunkRecord* rec, const StridedTiling& t, uint32_t bx,
                                         uint32_t g, int half, int tid) {
     const uint32_t F = a.group_stride;
@@ -138,11 +140,11 @@ struct StridedRowConstants {
     uint64_t i0 = (uint64_t)row0 * F + (uint64_t)fo * 8;
 #pragma unroll
     for (int r = 0; r < 4; ++r, i0 += F) {
-      in[r] = active && row0 + r < t.n_rows;
+      in[r] = ALLFULL || (active && row0 + r < t.n_rows);
       inv[r] = 0.0f;
       base[r] = 0.0f;
       if (in[r]) {
-        const ChunkRecord* c = rec + chunk_of(a, i0);
+        const ChunkRecord* c = rec + (ALLFULL ? (i0 >> a.chunk_shift) : chunk_of(a, i0));
         if (RANGE == kAbsMax) {
           inv[r] = ldg_c(&c->inv);
         } else {
@@ -155,16 +157,10 @@ struct StridedRowConstants {
   }
 };
 
-template <int K, int LAYOUT, int RANGE, int ROUND>
-__global__ void __launch_bounds__(256, 3) strided_encode_kernel(const CodecArgs a, const ChunkRecord* rec,
-                                                                const StridedTiling t) {
-  extern __shared__ __align__(128) uint8_t s_tile[];
-  grid_dependency_handshake();
+template <int K, int LAYOUT, int RANGE, int ROUND, bool ALLFULL>
+__device__ __forceinline__ void strided_encode_tiles(const CodecArgs& a, const ChunkRecord* rec, const StridedTiling& t,
+                                                     uint8_t* s_tile) {
   const int tid = threadIdx.x, lane = tid & 31, sub = tid & 3;
-  if (blockIdx.x == 0 && tid < 8) {
-    st_c(a.header + tid, header_word(a, tid));
-    if ((a.n_chunks & 1) && tid < 2) st_c(reinterpret_cast<uint32_t*>(a.meta + a.n_chunks) + tid, 0u);
-  }
   const uint32_t F = a.group_stride;
   const Rng rng{(uint32_t)a.seed, (uint32_t)(a.seed >> 32)};
   // The eight lanes of a quarter warp read 32 bytes each at {row block 0..3} x {two neighbouring octet columns}; the row
@@ -194,13 +190,13 @@ __global__ void __launch_bounds__(256, 3) strided_encode_kernel(const CodecArgs 
   }
   bool failed = false;
   StridedRowConstants<RANGE> cur, nxt;  // constants are fetched one stage ahead of their use
-  if (g < t.tiles_y) cur.fetch(a, rec, t, bx, g, 0, tid);
+  if (g < t.tiles_y) cur.template fetch<ALLFULL>(a, rec, t, bx, g, 0, tid);
   while (g < t.tiles_y) {
     uint32_t next_bx = bx + t.step_x, next_g = g + t.step_y;
     if (next_bx >= t.tiles_x) { next_bx -= t.tiles_x; ++next_g; }
     const bool has_next = next_g < t.tiles_y;
     const uint32_t fo = bx * kStridedOctetsPerBlock + (tid >> 2);  // feature octet of this thread
-    const bool active = fo < F / 8;                                // inactive lanes still shuffle
+    const bool active = ALLFULL || fo < F / 8;                     // inactive lanes still shuffle
     const uint64_t word0 = ((uint64_t)g * F + (uint64_t)fo * 8) * K;  // first word of feature 8*fo of this batch group
 
     uint32_t xlo[8], xhi[8];  // per row: codes of features 0..3 / 4..7
@@ -213,7 +209,7 @@ __global__ void __launch_bounds__(256, 3) strided_encode_kernel(const CodecArgs 
         const float4* src = reinterpret_cast<const float4*>(s_tile + sub * kStridedRowBlockPitch +
                                                             (half * 4 + r) * kStridedRowBytes + (tid >> 2) * 32);
         float4 p0 = make_float4(0.f, 0.f, 0.f, 0.f), p1 = p0;
-        if (cur.in[r] && ok) { p0 = src[swapped]; p1 = src[swapped ^ 1]; }
+        if ((ALLFULL || cur.in[r]) && ok) { p0 = src[swapped]; p1 = src[swapped ^ 1]; }
         v[r][0] = p0.x; v[r][1] = p0.y; v[r][2] = p0.z; v[r][3] = p0.w;
         v[r][4] = p1.x; v[r][5] = p1.y; v[r][6] = p1.z; v[r][7] = p1.w;
       }
@@ -230,13 +226,13 @@ __global__ void __launch_bounds__(256, 3) strided_encode_kernel(const CodecArgs 
           failed = true;
         }
       }
-      if (half == 0) nxt.fetch(a, rec, t, bx, g, 1, tid);
-      else if (has_next) nxt.fetch(a, rec, t, next_bx, next_g, 0, tid);
+      if (half == 0) nxt.template fetch<ALLFULL>(a, rec, t, bx, g, 1, tid);
+      else if (has_next) nxt.template fetch<ALLFULL>(a, rec, t, next_bx, next_g, 0, tid);
 #pragma unroll
       for (int r = 0; r < 4; ++r) {
         const int rr = half * 4 + r;
         xlo[rr] = 0; xhi[rr] = 0;
-        if (cur.in[r] && !failed) {
+        if ((ALLFULL || cur.in[r]) && !failed) {
           const uint64_t i0 = (uint64_t)(g * 32 + sub * 8 + rr) * F + (uint64_t)fo * 8;
           Scale sc;
           sc.s = 0.0f; sc.o = 0.0f;
@@ -267,6 +263,22 @@ __global__ void __launch_bounds__(256, 3) strided_encode_kernel(const CodecArgs 
     for (int half = 0; half < 2; ++half)
       if (pending[half]) mbarrier_wait(bar[half], parity[half]);
   }
+}
+
+template <int K, int LAYOUT, int RANGE, int ROUND>
+__global__ void __launch_bounds__(256, 3) strided_encode_kernel(const CodecArgs a, const ChunkRecord* rec,
+                                                                const StridedTiling t) {
+  extern __shared__ __align__(128) uint8_t s_tile[];
+  grid_dependency_handshake();
+  const int tid = threadIdx.x;
+  if (blockIdx.x == 0 && tid < 8) {
+    st_c(a.header + tid, header_word(a, tid));
+    if ((a.n_chunks & 1) && tid < 2) st_c(reinterpret_cast<uint32_t*>(a.meta + a.n_chunks) + tid, 0u);
+  }
+  // the same for every block of the launch: no tile with missing rows or octets, chunk indices by a shift
+  const bool all_full = a.chunk_shift >= 0 && t.n_rows % 32 == 0 && (a.group_stride / 8) % kStridedOctetsPerBlock == 0;
+  if (all_full) strided_encode_tiles<K, LAYOUT, RANGE, ROUND, true>(a, rec, t, s_tile);
+  else strided_encode_tiles<K, LAYOUT, RANGE, ROUND, false>(a, rec, t, s_tile);
 }
 
 // Hashed words of three consecutive quads when the low word of the quad index wraps among them (once in
